@@ -1,0 +1,97 @@
+"""Literal scalar-loop writing of the SwitchHead forward pass (fp64, tiny shapes only).
+
+TEST INFRASTRUCTURE ONLY.  A second, independent transcription of the equations of the
+paper's Sec. 2.2, written token by token with Python floats and `math`, so that an index
+or broadcasting slip in the vectorised oracle shows up as a disagreement.  It shares no
+helper with the vectorised oracle.
+
+Per sequence, per head h, per destination token t:
+    y[t] += sum_{e in E_D^h(t)} sigmoid(z_D^h[t,e]) * (sum_{s<=t} A^h[t,s] V^h[s]) W_O^{h,e}
+with V^h[s] = sum_{e in E_S^h(s)} sigmoid(z_S^h[s,e]) * x[s] W_V^{h,e}  and
+     A^h[t,:] = softmax over visible keys of  Q^h[t].K^h[s] / sqrt(d_head)      (Eq. 1).
+"""
+from __future__ import annotations
+
+import math
+
+
+def _sigmoid(z: float) -> float:
+    if z >= 0:
+        return 1.0 / (1.0 + math.exp(-z))
+    ez = math.exp(z)
+    return ez / (1.0 + ez)
+
+
+def _select(z_row, k):
+    """k best experts: repeatedly take the largest remaining logit, lowest index on ties."""
+    chosen = []
+    remaining = list(range(len(z_row)))
+    for _ in range(k):
+        best = remaining[0]
+        for e in remaining[1:]:
+            if z_row[e] > z_row[best]:
+                best = e
+        chosen.append(best)
+        remaining.remove(best)
+    return chosen
+
+
+def _vecmat(v, W):
+    """v [n], W [n][m] -> [m]"""
+    m = len(W[0])
+    out = [0.0] * m
+    for i, vi in enumerate(v):
+        row = W[i]
+        for j in range(m):
+            out[j] += vi * row[j]
+    return out
+
+
+def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=None, causal=True):
+    """Nested lists or arrays in, nested list y [B][T][M] out."""
+    x = [[list(map(float, tok)) for tok in seq] for seq in x]
+    B, T, M = len(x), len(x[0]), len(x[0][0])
+    H, E = len(Wv), len(Wv[0])
+    D = len(Wv[0][0][0])
+    tolist = lambda a: a.tolist() if hasattr(a, "tolist") else a
+    Wq, Wk, Wv, Wo, Ws, Wd = map(tolist, (Wq, Wk, Wv, Wo, Ws, Wd))
+    bias_s = tolist(bias_s) if bias_s is not None else None
+    bias_d = tolist(bias_d) if bias_d is not None else None
+    y = [[[0.0] * M for _ in range(T)] for _ in range(B)]
+    for b in range(B):
+        for h in range(H):
+            Q, K, V, selD = [], [], [], []
+            for t in range(T):
+                xt = x[b][t]
+                Q.append(_vecmat(xt, Wq[h]))
+                K.append(_vecmat(xt, Wk[h]))
+                zs = _vecmat(xt, Ws[h])
+                zd = _vecmat(xt, Wd[h])
+                if bias_s is not None:
+                    zs = [a + c for a, c in zip(zs, bias_s[h])]
+                if bias_d is not None:
+                    zd = [a + c for a, c in zip(zd, bias_d[h])]
+                v = [0.0] * D
+                for e in _select(zs, k):
+                    g = _sigmoid(zs[e])
+                    pe = _vecmat(xt, Wv[h][e])
+                    for d in range(D):
+                        v[d] += g * pe[d]
+                V.append(v)
+                selD.append([(e, _sigmoid(zd[e])) for e in _select(zd, k)])
+            for t in range(T):
+                last = t if causal else T - 1
+                logits = [sum(Q[t][d] * K[s][d] for d in range(D)) / math.sqrt(D)
+                          for s in range(last + 1)]
+                mx = max(logits)
+                w = [math.exp(l - mx) for l in logits]
+                tot = sum(w)
+                a = [0.0] * D
+                for s, ws_ in enumerate(w):
+                    for d in range(D):
+                        a[d] += (ws_ / tot) * V[s][d]
+                for e, g in selD[t]:
+                    contrib = _vecmat(a, Wo[h][e])
+                    for c in range(M):
+                        y[b][t][c] += g * contrib[c]
+    return y

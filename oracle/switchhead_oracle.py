@@ -1,0 +1,191 @@
+"""fp64 CPU oracle for the forward pass of one SwitchHead attention layer.
+
+TEST INFRASTRUCTURE ONLY.  This file is the yardstick the CUDA path is compared with; it
+shares no code with the CUDA path and nothing in the product imports it (only tests/,
+the smoke check and the benchmark's CPU-baseline leg do).
+
+What it computes, following the paper's Sec. 2.2 ("From Dense to SwitchHead"):
+
+  source-side gate        s_S^h = sigmoid(x W_S^h)            (first display eq. of Sec. 2.2)
+  destination-side gate   s_D^h = sigmoid(x W_D^h)            (text after it)
+  selections              E_S^h, E_D^h = arg top-k            (same place)
+  value projection        V^h = sum_{e in E_S^h} s_S^h[e] x W_V^{h,e}
+  dense queries / keys    Q^h = x W_Q^h, K^h = x W_K^h        (SwitchHead keeps one dense
+                                                               Q/K per head, end of Sec. 2.2)
+  attention               A^h = softmax(Q^h K^h^T / sqrt(d_head))     (Eq. 1), causal
+  output                  y = sum_h sum_{e in E_D^h} s_D^h[e] A^h V^h W_O^{h,e}
+                                                              (the MoE output equation)
+
+Readings where the paper is silent (each is listed in the design notes):
+  * top-k is taken on the pre-sigmoid logits (sigmoid is strictly increasing, so the set
+    is the same in exact arithmetic); ties go to the lower expert index; -0.0 == +0.0.
+  * no renormalisation among the selected gates (non-competitive sigmoid gate).
+  * causal mask: key s is visible to query t iff s <= t (language-model setting).
+  * an optional per-expert gate bias b (z = x W + b) exists only for the skew-routed
+    synthetic workload; None reproduces the paper exactly.
+  * batch elements are independent sequences.
+
+All arithmetic is fp64 on the values handed in (already rounded to their storage type);
+no intermediate rounding.  Every stage is returned so that a failing comparison can be
+localised.
+
+Pins (tests/test_oracle_pins.py): E=1 with zero gate weights equals 0.25 x textbook MHA
+(Eq. 2 and Eq. 3 forms, and torch's scaled_dot_product_attention); gate forced to 1 equals
+MHA; k=E equals the dense gate-weighted einsum; top-k equals a brute-force stable sort;
+causality; W_Q=0 gives running means of V; expert-permutation and batch-permutation
+invariance; linearity in W_O; bucket lists are a stable counting sort.
+Absolute output values for realistic trained weights: parity unpinned (the paper prints
+no worked forward-pass example).
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import numpy as np
+
+
+def stable_sigmoid(z: np.ndarray) -> np.ndarray:
+    z = np.asarray(z, dtype=np.float64)
+    out = np.empty_like(z)
+    pos = z >= 0
+    out[pos] = 1.0 / (1.0 + np.exp(-z[pos]))
+    ez = np.exp(z[~pos])
+    out[~pos] = ez / (1.0 + ez)
+    return out
+
+
+def topk_lower_index_wins(z: np.ndarray, k: int) -> np.ndarray:
+    """Indices of the k largest entries of each row of z [n, E]: value descending, and among
+    equal values the lower index first.  Returns [n, k] int32."""
+    z = np.asarray(z, dtype=np.float64) + 0.0      # -0.0 + 0.0 = +0.0: the two zeros tie
+    # stable sort on the negated value keeps equal values in ascending index order
+    order = np.argsort(-z, axis=1, kind="stable")
+    return order[:, :k].astype(np.int32)
+
+
+def gate_and_select(x2d, W, bias, k):
+    """x2d [n, M], W [H, M, E], bias [H, E] or None.
+    Returns logits z [n, H, E], scores s [n, H, E], idx [n, H, k] (rank order), gate [n, H, k]."""
+    n = x2d.shape[0]
+    H, _, E = W.shape
+    z = np.empty((n, H, E))
+    for h in range(H):
+        z[:, h, :] = x2d @ W[h]
+        if bias is not None:
+            z[:, h, :] += bias[h]
+    s = stable_sigmoid(z)
+    idx = np.empty((n, H, k), dtype=np.int32)
+    for h in range(H):
+        idx[:, h, :] = topk_lower_index_wins(z[:, h, :], k)
+    gate = np.take_along_axis(s, idx.astype(np.int64), axis=2)
+    return z, s, idx, gate
+
+
+def bucket_lists(idx: np.ndarray, n_experts: int):
+    """Per (head, expert) lists of the tokens that selected the expert, token-ascending.
+
+    idx [n, H, k].  Returns offsets [H, E+1] (exclusive scan of the counts, per head) and
+    lists [H, n*k] of token ids (bucket e of head h occupies lists[h, offsets[h,e]:offsets[h,e+1]])."""
+    n, H, k = idx.shape
+    offsets = np.zeros((H, n_experts + 1), dtype=np.int32)
+    lists = np.empty((H, n * k), dtype=np.int32)
+    for h in range(H):
+        pos = 0
+        for e in range(n_experts):
+            toks = np.nonzero((idx[:, h, :] == e).any(axis=1))[0]
+            lists[h, pos:pos + toks.size] = toks
+            pos += toks.size
+            offsets[h, e + 1] = pos
+        assert pos == n * k
+    return offsets, lists
+
+
+def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=None,
+                       causal: bool = True, gate_override: Optional[float] = None,
+                       return_stages: bool = True):
+    """Forward pass of one SwitchHead layer in fp64.
+
+    x [B, T, M]; Wq, Wk [H, M, D]; Wv [H, E, M, D]; Wo [H, E, D, M]; Ws, Wd [H, M, E].
+    gate_override: if given, every selected expert's gate is replaced by this constant
+    (used only to pin the E=1 case to plain multi-head attention).
+    Returns a dict with y [B, T, M] and, if return_stages, the intermediate stages."""
+    f = lambda a: None if a is None else np.asarray(a, dtype=np.float64)
+    x, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d = map(f, (x, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d))
+    B, T, M = x.shape
+    H, E, _, D = Wv.shape
+    N = B * T
+    x2d = x.reshape(N, M)
+
+    zS, sS, idxS, gateS = gate_and_select(x2d, Ws, bias_s, k)
+    zD, sD, idxD, gateD = gate_and_select(x2d, Wd, bias_d, k)
+    if gate_override is not None:
+        gateS = np.full_like(gateS, gate_override)
+        gateD = np.full_like(gateD, gate_override)
+
+    Q = np.empty((N, H, D))
+    K = np.empty((N, H, D))
+    V = np.zeros((N, H, D))
+    for h in range(H):
+        Q[:, h, :] = x2d @ Wq[h]
+        K[:, h, :] = x2d @ Wk[h]
+        # value experts: only the rows that selected expert e are projected with it
+        for e in range(E):
+            for j in range(k):
+                rows = np.nonzero(idxS[:, h, j] == e)[0]
+                if rows.size:
+                    V[rows, h, :] += gateS[rows, h, j][:, None] * (x2d[rows] @ Wv[h, e])
+
+    Ahat = np.empty((N, H, D))
+    scale = 1.0 / np.sqrt(D)
+    mask = np.triu(np.ones((T, T), dtype=bool), k=1) if causal else None
+    for b in range(B):
+        sl = slice(b * T, (b + 1) * T)
+        for h in range(H):
+            L = (Q[sl, h, :] @ K[sl, h, :].T) * scale
+            if causal:
+                L = np.where(mask, -np.inf, L)
+            L = L - L.max(axis=1, keepdims=True)
+            P = np.exp(L)
+            A = P / P.sum(axis=1, keepdims=True)
+            Ahat[sl, h, :] = A @ V[sl, h, :]
+
+    y = np.zeros((N, M))
+    for h in range(H):
+        for e in range(E):
+            for j in range(k):
+                rows = np.nonzero(idxD[:, h, j] == e)[0]
+                if rows.size:
+                    y[rows] += gateD[rows, h, j][:, None] * (Ahat[rows, h, :] @ Wo[h, e])
+
+    out = {"y": y.reshape(B, T, M)}
+    if return_stages:
+        offS, listS = bucket_lists(idxS, E)
+        offD, listD = bucket_lists(idxD, E)
+        out.update(zS=zS, zD=zD, sS=sS, sD=sD, idxS=idxS, idxD=idxD, gateS=gateS, gateD=gateD,
+                   Q=Q.reshape(B, T, H, D), K=K.reshape(B, T, H, D), V=V.reshape(B, T, H, D),
+                   Ahat=Ahat.reshape(B, T, H, D), offsetsS=offS, listsS=listS,
+                   offsetsD=offD, listsD=listD)
+    return out
+
+
+def dense_mha_forward(x, Wq, Wk, Wv, Wo, causal: bool = True):
+    """Standard multi-head attention (Eq. 1-2) in the concatenated form: the per-head
+    readouts are concatenated along the feature axis and multiplied by one W_O of shape
+    [H*D, M].  x [B, T, M]; Wq, Wk, Wv [H, M, D]; Wo [H, D, M] (row blocks of W_O)."""
+    x, Wq, Wk, Wv, Wo = (np.asarray(a, dtype=np.float64) for a in (x, Wq, Wk, Wv, Wo))
+    B, T, M = x.shape
+    H, _, D = Wq.shape
+    WO = Wo.reshape(H * D, M)
+    y = np.empty((B, T, M))
+    for b in range(B):
+        cat = np.empty((T, H * D))
+        for h in range(H):
+            Qh, Kh, Vh = x[b] @ Wq[h], x[b] @ Wk[h], x[b] @ Wv[h]
+            L = Qh @ Kh.T / np.sqrt(D)
+            if causal:
+                L = np.where(np.triu(np.ones((T, T), dtype=bool), k=1), -np.inf, L)
+            L = L - L.max(axis=1, keepdims=True)
+            P = np.exp(L)
+            cat[:, h * D:(h + 1) * D] = (P / P.sum(axis=1, keepdims=True)) @ Vh
+        y[b] = cat @ WO
+    return y
