@@ -1,0 +1,142 @@
+/*
+ * switchhead.h - C ABI of the B200 (sm_100a) forward pass of one SwitchHead attention layer.
+ *
+ * The layer (paper Sec. 2.2): for an input x [B, T, d_model] and each of n_heads heads h,
+ *   source gate       s_S^h = sigmoid(x W_S^h),  destination gate  s_D^h = sigmoid(x W_D^h)
+ *   selections        E_S^h(t), E_D^h(t) = arg top-k over the E experts, per token
+ *   values            V^h[t] = sum_{e in E_S^h(t)} s_S^h[t,e] * x[t] W_V^{h,e}
+ *   queries / keys    Q^h = x W_Q^h,  K^h = x W_K^h           (one dense pair per head)
+ *   attention         A^h = softmax(Q^h K^h^T / sqrt(d_head)) (Eq. 1), causal: key s <= query t
+ *   output            y[t] = sum_h sum_{e in E_D^h(t)} s_D^h[t,e] * (A^h V^h)[t] W_O^{h,e}
+ * Top-k is taken on the pre-sigmoid logits; equal logits go to the lower expert index.
+ * Selected gates are not renormalised.  Batch elements are independent sequences.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless the comment says "host".
+ *   - Arrays are dense, row-major, in the layouts stated per argument.
+ *   - `stream` is a cudaStream_t passed as void*; NULL is the default stream.  All device
+ *     work of a call is enqueued on that stream; no call synchronises the device.
+ *   - Functions returning int give SH_OK (0) or a negative SH_ERR_* code; sh_last_error()
+ *     then holds a readable reason (thread-local, host string owned by the library).
+ *   - The library owns only the handle.  x, out, the source weights and the workspace
+ *     belong to the caller.  sh_forward / sh_gate_topk allocate nothing.
+ *   - Inputs must be finite.  There is no CPU fallback: without a CUDA device every
+ *     launching call fails with SH_ERR_CUDA.
+ */
+#ifndef SWITCHHEAD_H_
+#define SWITCHHEAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sh_layer sh_layer;
+
+enum { SH_F32 = 0, SH_BF16 = 1 };
+
+enum {
+  SH_OK = 0,
+  SH_ERR_INVALID_ARG = -1,
+  SH_ERR_UNSUPPORTED = -2,
+  SH_ERR_NOT_CONFIGURED = -3,
+  SH_ERR_WORKSPACE = -4,
+  SH_ERR_CUDA = -5,
+  SH_ERR_TIMEOUT = -6, /* a bounded device-side wait ran out (reported by sh_last_status) */
+  SH_ERR_BOUNDS = -7   /* a device-side index check failed (reported by sh_last_status)  */
+};
+
+/* Identifiers for sh_debug_buffer. */
+enum {
+  SH_BUF_Q = 0,      /* [B, H, T, D]  queries, pre-multiplied by log2(e)/sqrt(D)            */
+  SH_BUF_K = 1,      /* [B, H, T, D]                                                        */
+  SH_BUF_V = 2,      /* [B, H, T, D]  gate-weighted sum of the selected value experts       */
+  SH_BUF_AHAT = 3,   /* [B*T, H, D]   attention read-out (A^h V^h)[t]                        */
+  SH_BUF_IDX = 4,    /* [2, N, H, k]  int32                                                 */
+  SH_BUF_GATE = 5,   /* [2, N, H, k]  fp32                                                  */
+  SH_BUF_OFFSETS = 6,/* [2, H, E+1]   int32                                                 */
+  SH_BUF_LISTS = 7   /* [2, H, N*k]   int32                                                 */
+};
+
+/* Create a layer description.  Host-only, no CUDA call.
+ * Requires 1 <= k <= n_experts <= 32, n_heads >= 1, d_head in {32, 64, 128},
+ * d_model a positive multiple of 64.  Returns NULL on error (see sh_last_error). */
+sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k);
+
+/* Dense multi-head attention comparator (Eq. 1-2) built from the same kernels: every head
+ * has one dense W_V and W_O and there are no gates.  Used only to time a parameter-matched
+ * dense layer beside SwitchHead.  Weights are passed to sh_set_weights with n_experts = 1
+ * and Ws = Wd = NULL.  Returns NULL on error. */
+sh_layer* sh_create_dense(int d_model, int n_heads, int d_head);
+
+/* Fix the storage type and the problem size.  dtype SH_F32: x and weights fp32, all
+ * arithmetic fp32 on CUDA cores.  dtype SH_BF16: x and weights bf16, tensor-core products
+ * with fp32 accumulation, fp16 intermediates (Q, K, V, P, A^h V^h); requires d_head in
+ * {64, 128} and d_model a multiple of 128.  `out` is fp32 in both cases.
+ * batch*seq*n_heads*k must be below 2^31.  Invalidates workspace and weights. */
+int sh_configure(sh_layer* layer, int dtype, int batch, int seq);
+
+/* Bytes of workspace sh_set_workspace needs for the current configuration (0 if not
+ * configured). */
+size_t sh_workspace_bytes(const sh_layer* layer);
+
+/* Hand the layer a caller-owned device buffer of at least sh_workspace_bytes() bytes,
+ * aligned to 256 bytes.  It must stay valid until sh_destroy or the next sh_configure.
+ * Holds repacked weights, intermediates, token lists and the device status word. */
+int sh_set_workspace(sh_layer* layer, void* workspace, size_t bytes);
+
+/* Repack the weights into the workspace (asynchronously on `stream`); the caller may free
+ * or overwrite its copies once the stream has passed this point.  Element type = dtype of
+ * sh_configure.
+ *   Wq, Wk  [H, d_model, d_head]
+ *   Wv      [H, E, d_model, d_head]
+ *   Wo      [H, E, d_head, d_model]
+ *   Ws, Wd  [H, d_model, E]      source-side / destination-side gate weights
+ *   bias_s, bias_d  [H, E] fp32 or NULL: optional additive gate-logit bias, z = x W + b.
+ *                   The paper has no bias (NULL); it exists for skew-routed test workloads. */
+int sh_set_weights(sh_layer* layer, const void* Wq, const void* Wk, const void* Wv,
+                   const void* Wo, const void* Ws, const void* Wd, const float* bias_s,
+                   const float* bias_d, void* stream);
+
+/* The whole forward pass (gates + top-k + bucket sort, Q/K projections, value experts,
+ * causal attention, output experts with the gate-weighted sum) of x [B, T, d_model] into
+ * out [B, T, d_model] fp32.  out is fully overwritten.  Enqueues kernels only. */
+int sh_forward(sh_layer* layer, const void* x, void* out, void* stream);
+
+/* Gate stage alone, with its results exposed (any output pointer may be NULL):
+ *   idx     [2, N, H, k] int32  selected experts; side 0 = source, 1 = destination;
+ *                               in rank order (largest logit first, ties lower index first)
+ *   gate    [2, N, H, k] fp32   sigmoid of the selected logits, same order
+ *   offsets [2, H, E+1]  int32  exclusive scan of the per-expert token counts
+ *   lists   [2, H, N*k]  int32  token ids grouped by expert, ascending within a group:
+ *                               group e of (side, h) is lists[side,h,offsets[e]:offsets[e+1]]
+ * N = batch*seq. */
+int sh_gate_topk(sh_layer* layer, const void* x, int32_t* idx, float* gate, int32_t* offsets,
+                 int32_t* lists, void* stream);
+
+/* Device pointer and size of an intermediate buffer inside the workspace (contents are
+ * those of the last sh_forward / sh_gate_topk once the stream has drained).  Element type:
+ * fp32 for SH_F32, fp16 for SH_BF16 (Q, K, V, AHAT); int32 / fp32 for the gate buffers.
+ * Testing aid: lets a failing output be traced to the stage that produced it. */
+int sh_debug_buffer(sh_layer* layer, int which, void** dev_ptr, size_t* bytes);
+
+/* Reads the device status word (one blocking 4-byte copy on `stream`, which it drains).
+ * 0 if every kernel so far completed normally, else the first SH_ERR_TIMEOUT / SH_ERR_BOUNDS
+ * code recorded by a kernel that gave up a bounded wait or skipped a bad index. */
+int sh_last_status(sh_layer* layer, void* stream);
+
+/* Number of kernel launches the last sh_forward enqueued. */
+int sh_launch_count(const sh_layer* layer);
+
+/* Reason for the last failure on this host thread ("" if none). */
+const char* sh_last_error(void);
+
+/* Free the handle (NULL is allowed).  Does not touch caller-owned device memory. */
+void sh_destroy(sh_layer* layer);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWITCHHEAD_H_ */

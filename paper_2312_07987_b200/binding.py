@@ -1,0 +1,191 @@
+"""ctypes binding of libswitchhead.so: argument marshalling only.
+
+Every step of the forward pass runs in the library's CUDA kernels; torch is used here for
+device memory and streams.  Function names mirror the C ABI (include/switchhead.h).
+There is no CPU fallback: if the library cannot be loaded, importing this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+SH_F32, SH_BF16 = 0, 1
+SH_OK = 0
+ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_NOT_CONFIGURED",
+               -4: "SH_ERR_WORKSPACE", -5: "SH_ERR_CUDA", -6: "SH_ERR_TIMEOUT", -7: "SH_ERR_BOUNDS"}
+BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
+
+EXPORTS = ["sh_create", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
+           "sh_set_weights", "sh_forward", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
+           "sh_launch_count", "sh_last_error", "sh_destroy"]
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = ctypes.CDLL(path)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.sh_create.restype = vp
+    lib.sh_create.argtypes = [i32] * 5
+    lib.sh_create_dense.restype = vp
+    lib.sh_create_dense.argtypes = [i32] * 3
+    lib.sh_configure.restype = i32
+    lib.sh_configure.argtypes = [vp, i32, i32, i32]
+    lib.sh_workspace_bytes.restype = sz
+    lib.sh_workspace_bytes.argtypes = [vp]
+    lib.sh_set_workspace.restype = i32
+    lib.sh_set_workspace.argtypes = [vp, vp, sz]
+    lib.sh_set_weights.restype = i32
+    lib.sh_set_weights.argtypes = [vp] * 10
+    lib.sh_forward.restype = i32
+    lib.sh_forward.argtypes = [vp, vp, vp, vp]
+    lib.sh_gate_topk.restype = i32
+    lib.sh_gate_topk.argtypes = [vp] * 7
+    lib.sh_debug_buffer.restype = i32
+    lib.sh_debug_buffer.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(sz)]
+    lib.sh_last_status.restype = i32
+    lib.sh_last_status.argtypes = [vp, vp]
+    lib.sh_launch_count.restype = i32
+    lib.sh_launch_count.argtypes = [vp]
+    lib.sh_last_error.restype = ctypes.c_char_p
+    lib.sh_last_error.argtypes = []
+    lib.sh_destroy.restype = None
+    lib.sh_destroy.argtypes = [vp]
+    return lib
+
+
+lib = _load()
+
+
+class SwitchHeadError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        msg = lib.sh_last_error().decode()
+        super().__init__(f"{ERROR_NAMES.get(code, code)}: {msg}")
+
+
+def _check(code: int) -> None:
+    if code != SH_OK:
+        raise SwitchHeadError(code)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def sh_last_error() -> str:
+    return lib.sh_last_error().decode()
+
+
+class Layer:
+    """Owns one sh_layer handle plus the torch tensors that back its workspace."""
+
+    def __init__(self, d_model: int, n_heads: int, d_head: int, n_experts: int = 1, k: int = 1,
+                 dense: bool = False):
+        self.dense = dense
+        self.dims = (d_model, n_heads, d_head, n_experts, k)
+        h = lib.sh_create_dense(d_model, n_heads, d_head) if dense else \
+            lib.sh_create(d_model, n_heads, d_head, n_experts, k)
+        if not h:
+            raise SwitchHeadError(-1)
+        self.handle = ctypes.c_void_p(h)
+        self.workspace = None
+        self.dtype = None
+        self.batch = self.seq = 0
+
+    def sh_configure(self, dtype: int, batch: int, seq: int, device="cuda") -> None:
+        _check(lib.sh_configure(self.handle, dtype, batch, seq))
+        self.dtype, self.batch, self.seq = dtype, batch, seq
+        nbytes = lib.sh_workspace_bytes(self.handle)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 255) // 256 * 256
+        _check(lib.sh_set_workspace(self.handle, ctypes.c_void_p(self._ws_ptr), nbytes))
+
+    def sh_set_weights(self, Wq, Wk, Wv, Wo, Ws=None, Wd=None, bias_s=None, bias_d=None) -> None:
+        ts = [Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d]
+        for t in ts:
+            assert t is None or (t.is_cuda and t.is_contiguous())
+        _check(lib.sh_set_weights(self.handle, *[_ptr(t) for t in ts], _stream()))
+        torch.cuda.current_stream().synchronize()   # the source tensors may now be released
+
+    def sh_forward(self, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        assert x.is_cuda and x.is_contiguous()
+        if out is None:
+            out = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+        _check(lib.sh_forward(self.handle, _ptr(x), _ptr(out), _stream()))
+        return out
+
+    def sh_gate_topk(self, x: torch.Tensor):
+        d_model, H, D, E, k = self.dims
+        N = self.batch * self.seq
+        dev = x.device
+        idx = torch.empty((2, N, H, k), dtype=torch.int32, device=dev)
+        gate = torch.empty((2, N, H, k), dtype=torch.float32, device=dev)
+        offsets = torch.empty((2, H, E + 1), dtype=torch.int32, device=dev)
+        lists = torch.empty((2, H, N * k), dtype=torch.int32, device=dev)
+        _check(lib.sh_gate_topk(self.handle, _ptr(x), _ptr(idx), _ptr(gate), _ptr(offsets), _ptr(lists), _stream()))
+        return idx, gate, offsets, lists
+
+    def sh_debug_buffer(self, name: str) -> torch.Tensor:
+        """Copy of an intermediate buffer as a torch tensor (Q, K, V [B,H,T,D]; AHAT [N,H,D])."""
+        p, n = ctypes.c_void_p(), ctypes.c_size_t()
+        _check(lib.sh_debug_buffer(self.handle, BUF[name], ctypes.byref(p), ctypes.byref(n)))
+        off = p.value - self.workspace.data_ptr()
+        raw = self.workspace[off:off + n.value].clone()
+        d_model, H, D, E, k = self.dims
+        if name in ("Q", "K", "V", "AHAT"):
+            t = raw.view(torch.float32 if self.dtype == SH_F32 else torch.float16)
+            return t.view(self.batch, H, self.seq, D) if name != "AHAT" else t.view(self.batch * self.seq, H, D)
+        return raw.view(torch.float32 if name == "GATE" else torch.int32)
+
+    def sh_last_status(self) -> int:
+        return lib.sh_last_status(self.handle, _stream())
+
+    def sh_launch_count(self) -> int:
+        return lib.sh_launch_count(self.handle)
+
+    def close(self) -> None:
+        if self.handle:
+            lib.sh_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def to_device(a: Optional[np.ndarray], dtype: int, device="cuda") -> Optional[torch.Tensor]:
+    """Host array (fp32 values already representable in the storage type) -> device tensor."""
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+    if dtype == SH_BF16:
+        t = t.to(torch.bfloat16)
+    return t.to(device).contiguous()
+
+
+def layer_from_inputs(inp, batch=None, seq=None, device="cuda") -> "Layer":
+    """Create, configure and load a Layer from a LayerInputs record (see inputs.py)."""
+    cfg = inp.cfg
+    B, T = inp.x.shape[0], inp.x.shape[1]
+    L = Layer(cfg.d_model, cfg.n_heads, cfg.d_head, cfg.n_experts, cfg.k)
+    L.sh_configure(cfg.dtype, B, T, device=device)
+    dv = lambda a: to_device(a, cfg.dtype, device)
+    bias = lambda a: None if a is None else torch.from_numpy(a).to(device)
+    L.sh_set_weights(dv(inp.Wq), dv(inp.Wk), dv(inp.Wv), dv(inp.Wo), dv(inp.Ws), dv(inp.Wd),
+                     bias(inp.bias_s), bias(inp.bias_d))
+    return L

@@ -1,0 +1,369 @@
+// Host side of libswitchhead: argument validation, workspace layout, weight repacking and
+// the launch sequence of the forward pass.  Every entry point is documented in
+// include/switchhead.h.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "sh_internal.cuh"
+#include "sh_simt.cuh"
+
+static thread_local char g_err[512] = "";
+
+void sh_set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+#define SH_CUDA_CHECK(expr)                                                          \
+  do {                                                                               \
+    cudaError_t _e = (expr);                                                         \
+    if (_e != cudaSuccess) {                                                         \
+      sh_set_error("%s failed: %s", #expr, cudaGetErrorString(_e));                  \
+      return SH_ERR_CUDA;                                                            \
+    }                                                                                \
+  } while (0)
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static size_t elem_bytes_in(int dtype) { return dtype == SH_F32 ? 4 : 2; }
+static size_t elem_bytes_mid(int dtype) { return dtype == SH_F32 ? 4 : 2; }
+
+static void layout_workspace(sh_layer* L) {
+  const ShDims& d = L->d;
+  const size_t in = elem_bytes_in(L->dtype), mid = elem_bytes_mid(L->dtype);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 1024);
+    return o;
+  };
+  ShWorkspace& o = L->o;
+  const size_t HD = (size_t)d.H * d.D;
+  const size_t nproj = L->dense ? 3 : 2;
+  o.status = take(256);
+  o.wqk = take(nproj * HD * d.M * in);
+  o.wgate = take((size_t)d.G * d.M * in);
+  o.gbias = take((size_t)d.G * 4);
+  o.wv = take(L->dense ? 16 : HD * d.E * d.M * in);
+  o.wo = take(HD * d.E * d.M * mid);
+  o.q = take((size_t)d.N * HD * mid);
+  o.k = take((size_t)d.N * HD * mid);
+  o.v = take((size_t)d.N * HD * mid);
+  o.ahat = take((size_t)d.N * HD * mid);
+  const size_t slots = (size_t)2 * d.N * d.H * d.k;
+  o.idx = take(slots * 4);
+  o.gate = take(slots * 4);
+  o.blockcnt = take((size_t)d.nblk * d.G * 4);
+  o.blockoff = take((size_t)d.nblk * d.G * 4);
+  o.offsets = take((size_t)2 * d.H * (d.E + 1) * 4);
+  o.lists = take(slots * 4);
+  o.lgate = take(slots * 4);
+  o.tiles = take((size_t)2 * d.max_tiles * sizeof(ShTile));
+  o.ntiles = take(256);
+  o.total = off;
+}
+
+static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_experts, int k, bool dense) {
+  g_err[0] = 0;
+  if (d_model <= 0 || d_model % 64 != 0) { sh_set_error("d_model must be a positive multiple of 64 (got %d)", d_model); return nullptr; }
+  if (n_heads < 1) { sh_set_error("n_heads must be >= 1 (got %d)", n_heads); return nullptr; }
+  if (d_head != 32 && d_head != 64 && d_head != 128) { sh_set_error("d_head must be 32, 64 or 128 (got %d)", d_head); return nullptr; }
+  if (n_experts < 1 || n_experts > 32) { sh_set_error("n_experts must be in 1..32 (got %d)", n_experts); return nullptr; }
+  if (k < 1 || k > n_experts) { sh_set_error("k must be in 1..n_experts (got k=%d, n_experts=%d)", k, n_experts); return nullptr; }
+  sh_layer* L = new (std::nothrow) sh_layer();
+  if (!L) { sh_set_error("out of host memory"); return nullptr; }
+  L->d.M = d_model; L->d.H = n_heads; L->d.D = d_head; L->d.E = n_experts; L->d.k = k;
+  L->d.G = 2 * n_heads * n_experts;
+  L->dense = dense;
+  return L;
+}
+
+extern "C" sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k) {
+  return create_common(d_model, n_heads, d_head, n_experts, k, false);
+}
+
+extern "C" sh_layer* sh_create_dense(int d_model, int n_heads, int d_head) {
+  return create_common(d_model, n_heads, d_head, 1, 1, true);
+}
+
+extern "C" int sh_configure(sh_layer* L, int dtype, int batch, int seq) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (dtype != SH_F32 && dtype != SH_BF16) { sh_set_error("dtype must be SH_F32 or SH_BF16 (got %d)", dtype); return SH_ERR_INVALID_ARG; }
+  if (batch < 1 || seq < 1) { sh_set_error("batch and seq must be >= 1 (got %d, %d)", batch, seq); return SH_ERR_INVALID_ARG; }
+  const ShDims& d0 = L->d;
+  if (dtype == SH_BF16 && (d0.D < 64 || d0.M % 128 != 0)) {
+    sh_set_error("bf16 path needs d_head in {64,128} and d_model %% 128 == 0 (got d_head=%d, d_model=%d)", d0.D, d0.M);
+    return SH_ERR_UNSUPPORTED;
+  }
+  const long long slots = (long long)batch * seq * d0.H * d0.k;
+  if (slots >= (1ll << 31) || (long long)batch * seq * d0.M >= (1ll << 40)) {
+    sh_set_error("problem too large: batch*seq*n_heads*k = %lld must be below 2^31", slots);
+    return SH_ERR_UNSUPPORTED;
+  }
+  L->dtype = dtype;
+  L->d.B = batch; L->d.T = seq; L->d.N = batch * seq;
+  L->d.nblk = (L->d.N + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
+  L->d.max_tiles = (int)((slots + SH_TILE_ROWS - 1) / SH_TILE_ROWS) + d0.H * d0.E;
+  L->ws = nullptr; L->ws_bytes = 0; L->weights_set = false;
+  sh_tc_release(L);
+  layout_workspace(L);
+  return SH_OK;
+}
+
+extern "C" size_t sh_workspace_bytes(const sh_layer* L) {
+  if (!L || L->dtype < 0) return 0;
+  return L->o.total;
+}
+
+extern "C" int sh_set_workspace(sh_layer* L, void* workspace, size_t bytes) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0) { sh_set_error("sh_configure has not been called"); return SH_ERR_NOT_CONFIGURED; }
+  if (!workspace) { sh_set_error("workspace is NULL"); return SH_ERR_WORKSPACE; }
+  if ((uintptr_t)workspace % 256 != 0) { sh_set_error("workspace must be 256-byte aligned"); return SH_ERR_WORKSPACE; }
+  if (bytes < L->o.total) { sh_set_error("workspace too small: %zu bytes given, %zu needed", bytes, L->o.total); return SH_ERR_WORKSPACE; }
+  L->ws = (char*)workspace; L->ws_bytes = bytes; L->weights_set = false;
+  sh_tc_release(L);
+  return SH_OK;
+}
+
+template <typename TI, typename TO>
+static void repack(const void* in, void* out, int batch, int rows, int cols, long obs, long ors, long oes,
+                   cudaStream_t st) {
+  long total = (long)batch * rows * cols;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 65535 * 4) blocks = 65535 * 4;
+  if (blocks < 1) blocks = 1;
+  sh_repack_kernel<TI, TO><<<blocks, 256, 0, st>>>((const TI*)in, (TO*)out, batch, rows, cols, obs, ors, oes);
+}
+
+template <typename TI, typename TM>
+static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                         const void* Ws, const void* Wd, const float* bias_s, const float* bias_d,
+                         cudaStream_t st) {
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const long HD = (long)d.H * d.D;
+  SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.status, 0, 256, st));
+  // Wq, Wk [H, M, D] -> Wqk[(which*H + h)*D + dd][m]
+  TI* wqk = (TI*)(ws + L->o.wqk);
+  repack<TI, TI>(Wq, wqk, d.H, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
+  repack<TI, TI>(Wk, wqk + HD * d.M, d.H, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
+  if (L->dense) {
+    // Wv [H, 1, M, D] joins the fused projection; Wo [H, 1, D, M] -> Wo_t[m][h*D + dd]
+    repack<TI, TI>(Wv, wqk + 2 * HD * d.M, d.H, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
+    repack<TI, TM>(Wo, ws + L->o.wo, d.H, d.D, d.M, d.D, HD, 1, st);
+  } else {
+    // Ws, Wd [H, M, E] -> Wgate[(side*H + h)*E + e][m]
+    TI* wg = (TI*)(ws + L->o.wgate);
+    repack<TI, TI>(Ws, wg, d.H, d.M, d.E, (long)d.E * d.M, d.M, 1, st);
+    repack<TI, TI>(Wd, wg + (long)d.H * d.E * d.M, d.H, d.M, d.E, (long)d.E * d.M, d.M, 1, st);
+    float* gb = (float*)(ws + L->o.gbias);
+    const size_t hb = (size_t)d.H * d.E * 4;
+    if (bias_s) SH_CUDA_CHECK(cudaMemcpyAsync(gb, bias_s, hb, cudaMemcpyDeviceToDevice, st));
+    else SH_CUDA_CHECK(cudaMemsetAsync(gb, 0, hb, st));
+    if (bias_d) SH_CUDA_CHECK(cudaMemcpyAsync(gb + d.H * d.E, bias_d, hb, cudaMemcpyDeviceToDevice, st));
+    else SH_CUDA_CHECK(cudaMemsetAsync(gb + d.H * d.E, 0, hb, st));
+    // Wv [H, E, M, D] -> [H, E, D, M];  Wo [H, E, D, M] -> [H, E, M, D]
+    repack<TI, TI>(Wv, ws + L->o.wv, d.H * d.E, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
+    repack<TI, TM>(Wo, ws + L->o.wo, d.H * d.E, d.D, d.M, (long)d.D * d.M, d.D, 1, st);
+  }
+  SH_CUDA_CHECK(cudaGetLastError());
+  return SH_OK;
+}
+
+extern "C" int sh_set_weights(sh_layer* L, const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                              const void* Ws, const void* Wd, const float* bias_s, const float* bias_d,
+                              void* stream) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0) { sh_set_error("sh_configure has not been called"); return SH_ERR_NOT_CONFIGURED; }
+  if (!L->ws) { sh_set_error("sh_set_workspace has not been called"); return SH_ERR_WORKSPACE; }
+  if (!Wq || !Wk || !Wv || !Wo) { sh_set_error("Wq, Wk, Wv and Wo must not be NULL"); return SH_ERR_INVALID_ARG; }
+  if (!L->dense && (!Ws || !Wd)) { sh_set_error("Ws and Wd must not be NULL for a SwitchHead layer"); return SH_ERR_INVALID_ARG; }
+  if (L->dense && (Ws || Wd || bias_s || bias_d)) { sh_set_error("a dense layer has no gates: pass NULL for Ws, Wd and the biases"); return SH_ERR_INVALID_ARG; }
+  cudaStream_t st = (cudaStream_t)stream;
+  int rc = (L->dtype == SH_F32)
+               ? set_weights_t<float, float>(L, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d, st)
+               : set_weights_t<__nv_bfloat16, __half>(L, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d, st);
+  if (rc != SH_OK) return rc;
+  if (L->dtype == SH_BF16) {
+    rc = sh_tc_prepare(L);
+    if (rc != SH_OK) return rc;
+  }
+  L->weights_set = true;
+  return SH_OK;
+}
+
+static int check_ready(sh_layer* L) {
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0) { sh_set_error("sh_configure has not been called"); return SH_ERR_NOT_CONFIGURED; }
+  if (!L->ws) { sh_set_error("sh_set_workspace has not been called"); return SH_ERR_WORKSPACE; }
+  if (!L->weights_set) { sh_set_error("sh_set_weights has not been called"); return SH_ERR_NOT_CONFIGURED; }
+  return SH_OK;
+}
+
+// gate + top-k + bucket sort (three launches)
+template <typename TI>
+static int launch_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const size_t hist = (size_t)d.G * 4;
+  sh_gate_topk_kernel<TI><<<d.nblk, 256, hist, st>>>((const TI*)x, (const TI*)(ws + L->o.wgate),
+      (const float*)(ws + L->o.gbias), (int*)(ws + L->o.idx), (float*)(ws + L->o.gate),
+      (int*)(ws + L->o.blockcnt), d);
+  sh_sort_scan_kernel<<<1, 256, (2 * hist + 16), st>>>((const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.blockoff),
+      (int*)(ws + L->o.offsets), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);
+  sh_sort_scatter_kernel<<<d.nblk, SH_TILE_ROWS, 0, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
+      (const int*)(ws + L->o.blockoff), (const int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
+      (float*)(ws + L->o.lgate), d);
+  L->launches += 3;
+  SH_CUDA_CHECK(cudaGetLastError());
+  return SH_OK;
+}
+
+template <typename TI, typename TM>
+static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaStream_t st) {
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const int HD = d.H * d.D;
+  const float qscale = 1.4426950408889634f / sqrtf((float)d.D);
+  if (!L->dense && (stages & SH_STAGE_GATE)) {
+    int rc = launch_gate_sort<TI>(L, x, st);
+    if (rc != SH_OK) return rc;
+  }
+  if (stages & SH_STAGE_QK) {
+  ShGemmArgs g{};
+  g.d = d;
+  // Q, K (and V for the dense comparator)
+  g.A = x; g.lda = d.M; g.Bt = ws + L->o.wqk; g.ldb = d.M; g.K = d.M;
+  g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
+  g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v; g.qscale = qscale;
+  dim3 grid_qk(d.nblk, (g.ncols + 63) / 64);
+  sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_qk, 256, 0, st>>>(g);
+  L->launches += 1;
+  }
+  if (!L->dense && (stages & SH_STAGE_V)) {
+    SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * HD * sizeof(TM), st));
+    ShGemmArgs v{};
+    v.d = d; v.A = x; v.lda = d.M; v.Bt = ws + L->o.wv; v.ldb = d.M; v.K = d.M; v.ncols = d.D;
+    v.lists = (const int*)(ws + L->o.lists); v.lgate = (const float*)(ws + L->o.lgate);
+    v.tiles = (const ShTile*)(ws + L->o.tiles); v.ntiles = (const int*)(ws + L->o.ntiles);
+    v.b_group_stride = (long)d.D * d.M; v.out0 = ws + L->o.v;
+    dim3 grid_v(d.max_tiles, (d.D + 63) / 64);
+    sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_V><<<grid_v, 256, 0, st>>>(v);
+    L->launches += 2;
+  }
+  if (stages & SH_STAGE_ATTN) {
+    const long nq = (long)d.B * d.H * d.T;
+    sh_simt_attention_kernel<TM><<<(unsigned)((nq + 3) / 4), 128, 0, st>>>((const TM*)(ws + L->o.q),
+        (const TM*)(ws + L->o.k), (const TM*)(ws + L->o.v), (TM*)(ws + L->o.ahat), d);
+    L->launches += 1;
+  }
+  if (!(stages & SH_STAGE_O)) {
+  } else if (!L->dense) {
+    SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
+    ShGemmArgs o{};
+    o.d = d; o.A = ws + L->o.ahat; o.lda = HD; o.a_head_stride = d.D; o.Bt = ws + L->o.wo; o.ldb = d.D;
+    o.K = d.D; o.ncols = d.M;
+    const size_t side1 = (size_t)d.H * d.N * d.k;
+    o.lists = (const int*)(ws + L->o.lists) + side1; o.lgate = (const float*)(ws + L->o.lgate) + side1;
+    o.tiles = (const ShTile*)(ws + L->o.tiles) + d.max_tiles; o.ntiles = (const int*)(ws + L->o.ntiles) + 1;
+    o.b_group_stride = (long)d.M * d.D; o.out0 = out;
+    dim3 grid_o(d.max_tiles, (d.M + 63) / 64);
+    sh_simt_gemm_kernel<TM, TM, float, SH_EPI_O><<<grid_o, 256, 0, st>>>(o);
+    L->launches += 2;
+  } else {
+    ShGemmArgs o{};
+    o.d = d; o.A = ws + L->o.ahat; o.lda = HD; o.Bt = ws + L->o.wo; o.ldb = HD; o.K = HD; o.ncols = d.M;
+    o.nrows = d.N; o.out0 = out;
+    dim3 grid_o(d.nblk, (d.M + 63) / 64);
+    sh_simt_gemm_kernel<TM, TM, float, SH_EPI_PLAIN><<<grid_o, 256, 0, st>>>(o);
+    L->launches += 1;
+  }
+  SH_CUDA_CHECK(cudaGetLastError());
+  return SH_OK;
+}
+
+int sh_simt_run_bf16(sh_layer* L, int stages, const void* x, void* out, cudaStream_t st) {
+  return forward_simt<__nv_bfloat16, __half>(L, stages, x, out, st);
+}
+
+extern "C" int sh_forward(sh_layer* L, const void* x, void* out, void* stream) {
+  g_err[0] = 0;
+  int rc = check_ready(L);
+  if (rc != SH_OK) return rc;
+  if (!x || !out) { sh_set_error("x and out must not be NULL"); return SH_ERR_INVALID_ARG; }
+  cudaStream_t st = (cudaStream_t)stream;
+  L->launches = 0;
+  if (L->dtype == SH_F32) return forward_simt<float, float>(L, SH_STAGE_ALL, x, out, st);
+  return sh_tc_forward(L, x, out, st);
+}
+
+extern "C" int sh_gate_topk(sh_layer* L, const void* x, int32_t* idx, float* gate, int32_t* offsets,
+                            int32_t* lists, void* stream) {
+  g_err[0] = 0;
+  int rc = check_ready(L);
+  if (rc != SH_OK) return rc;
+  if (L->dense) { sh_set_error("a dense layer has no gates"); return SH_ERR_UNSUPPORTED; }
+  if (!x) { sh_set_error("x must not be NULL"); return SH_ERR_INVALID_ARG; }
+  cudaStream_t st = (cudaStream_t)stream;
+  L->launches = 0;
+  rc = (L->dtype == SH_F32) ? launch_gate_sort<float>(L, x, st) : sh_tc_gate_sort(L, x, st);
+  if (rc != SH_OK) return rc;
+  const ShDims& d = L->d;
+  const size_t slots = (size_t)2 * d.N * d.H * d.k;
+  if (idx) SH_CUDA_CHECK(cudaMemcpyAsync(idx, L->ws + L->o.idx, slots * 4, cudaMemcpyDeviceToDevice, st));
+  if (gate) SH_CUDA_CHECK(cudaMemcpyAsync(gate, L->ws + L->o.gate, slots * 4, cudaMemcpyDeviceToDevice, st));
+  if (offsets) SH_CUDA_CHECK(cudaMemcpyAsync(offsets, L->ws + L->o.offsets, (size_t)2 * d.H * (d.E + 1) * 4, cudaMemcpyDeviceToDevice, st));
+  if (lists) SH_CUDA_CHECK(cudaMemcpyAsync(lists, L->ws + L->o.lists, slots * 4, cudaMemcpyDeviceToDevice, st));
+  return SH_OK;
+}
+
+extern "C" int sh_debug_buffer(sh_layer* L, int which, void** dev_ptr, size_t* bytes) {
+  g_err[0] = 0;
+  if (!L || !dev_ptr || !bytes) { sh_set_error("NULL argument"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0 || !L->ws) { sh_set_error("layer has no workspace yet"); return SH_ERR_NOT_CONFIGURED; }
+  const ShDims& d = L->d;
+  const size_t mid = elem_bytes_mid(L->dtype), act = (size_t)d.N * d.H * d.D * mid;
+  const size_t slots = (size_t)2 * d.N * d.H * d.k * 4;
+  size_t off, sz;
+  switch (which) {
+    case SH_BUF_Q: off = L->o.q; sz = act; break;
+    case SH_BUF_K: off = L->o.k; sz = act; break;
+    case SH_BUF_V: off = L->o.v; sz = act; break;
+    case SH_BUF_AHAT: off = L->o.ahat; sz = act; break;
+    case SH_BUF_IDX: off = L->o.idx; sz = slots; break;
+    case SH_BUF_GATE: off = L->o.gate; sz = slots; break;
+    case SH_BUF_OFFSETS: off = L->o.offsets; sz = (size_t)2 * d.H * (d.E + 1) * 4; break;
+    case SH_BUF_LISTS: off = L->o.lists; sz = slots; break;
+    default: sh_set_error("unknown buffer id %d", which); return SH_ERR_INVALID_ARG;
+  }
+  *dev_ptr = L->ws + off; *bytes = sz;
+  return SH_OK;
+}
+
+extern "C" int sh_last_status(sh_layer* L, void* stream) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0 || !L->ws) { sh_set_error("layer has no workspace yet"); return SH_ERR_NOT_CONFIGURED; }
+  int v = 0;
+  SH_CUDA_CHECK(cudaMemcpyAsync(&v, L->ws + L->o.status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  SH_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+  return v;
+}
+
+extern "C" int sh_launch_count(const sh_layer* L) { return L ? L->launches : 0; }
+
+extern "C" const char* sh_last_error(void) { return g_err; }
+
+extern "C" void sh_destroy(sh_layer* L) {
+  if (!L) return;
+  sh_tc_release(L);
+  delete L;
+}

@@ -1,0 +1,376 @@
+// CUDA-core (FFMA) kernels: the whole fp32 configuration runs on these; the gate, top-k and
+// bucket-sort kernels also serve the bf16 configuration.
+#pragma once
+#include "sh_internal.cuh"
+
+// ---------------------------------------------------------------------------------------
+// Weight repack: out[b*obs + c*ors + r*oes] = in[b*rows*cols + r*cols + c]  (a batched
+// transpose with free output strides), with type conversion.
+// ---------------------------------------------------------------------------------------
+template <typename TI, typename TO>
+__global__ void sh_repack_kernel(const TI* __restrict__ in, TO* __restrict__ out, int batch, int rows,
+                                 int cols, long obs, long ors, long oes) {
+  long total = (long)batch * rows * cols;
+  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+    int r = (int)(i % rows);
+    long t = i / rows;
+    int c = (int)(t % cols);
+    int b = (int)(t / cols);
+    float v = sh_to_float<TI>(in[((long)b * rows + r) * cols + c]);
+    out[b * obs + c * ors + r * oes] = sh_from_float<TO>(v);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Gate: z = x W (+ b) per (side, head), sigmoid, top-k with lower-index-wins, per-block
+// histogram of the selections (Sec. 2.2: s = sigmoid(x W_S), E = arg top-k).
+// One warp per token; lane e owns expert e's logit during selection.
+// Wg is [G, M] (one row per gate column g = (side*H + h)*E + e).
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const float* __restrict__ gbias,
+                    int* __restrict__ idx, float* __restrict__ gate, int* __restrict__ blockcnt, ShDims d) {
+  extern __shared__ int s_hist[];            // [2*H*E]
+  const int nb = 2 * d.H * d.E;
+  for (int i = threadIdx.x; i < nb; i += blockDim.x) s_hist[i] = 0;
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int tok0 = blockIdx.x * SH_TILE_ROWS;
+  for (int tt = warp; tt < SH_TILE_ROWS; tt += nwarps) {
+    const int t = tok0 + tt;
+    if (t >= d.N) break;
+    const T* xr = x + (size_t)t * d.M;
+    for (int grp = 0; grp < 2 * d.H; ++grp) {
+      float z = 0.f;                         // lane e keeps logit e
+      for (int e0 = 0; e0 < d.E; e0 += 4) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        const T* w0 = Wg + (size_t)(grp * d.E + e0) * d.M;
+        const bool h1 = e0 + 1 < d.E, h2 = e0 + 2 < d.E, h3 = e0 + 3 < d.E;
+        for (int m = lane; m < d.M; m += 32) {
+          float xv = sh_to_float<T>(xr[m]);
+          a0 = fmaf(xv, sh_to_float<T>(w0[m]), a0);
+          if (h1) a1 = fmaf(xv, sh_to_float<T>(w0[d.M + m]), a1);
+          if (h2) a2 = fmaf(xv, sh_to_float<T>(w0[2 * (size_t)d.M + m]), a2);
+          if (h3) a3 = fmaf(xv, sh_to_float<T>(w0[3 * (size_t)d.M + m]), a3);
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) {
+          a0 += __shfl_xor_sync(0xffffffffu, a0, s);
+          a1 += __shfl_xor_sync(0xffffffffu, a1, s);
+          a2 += __shfl_xor_sync(0xffffffffu, a2, s);
+          a3 += __shfl_xor_sync(0xffffffffu, a3, s);
+        }
+        if (lane == e0) z = a0;
+        if (lane == e0 + 1) z = a1;
+        if (lane == e0 + 2) z = a2;
+        if (lane == e0 + 3) z = a3;
+      }
+      if (lane < d.E) z += gbias[grp * d.E + lane];
+      int rank = 0;
+      for (int e = 0; e < d.E; ++e) {
+        float ze = __shfl_sync(0xffffffffu, z, e);
+        rank += (ze > z || (ze == z && e < lane)) ? 1 : 0;
+      }
+      if (lane < d.E && rank < d.k) {
+        const int side = grp / d.H, h = grp % d.H;
+        size_t o = (((size_t)side * d.N + t) * d.H + h) * d.k + rank;
+        idx[o] = lane;
+        gate[o] = 1.f / (1.f + expf(-z));
+        atomicAdd(&s_hist[grp * d.E + lane], 1);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < nb; i += blockDim.x) blockcnt[(size_t)blockIdx.x * nb + i] = s_hist[i];
+}
+
+// ---------------------------------------------------------------------------------------
+// Bucket sort, step 1 (one block): exclusive scan of the per-block histograms over blocks,
+// per-head exclusive scan over experts, and the row-tile table of the grouped GEMMs.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+sh_sort_scan_kernel(const int* __restrict__ blockcnt, int* __restrict__ blockoff, int* __restrict__ offsets,
+                    ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
+  extern __shared__ int s_scan[];            // total[nb], tilebase[nb + 2]
+  const int nb = 2 * d.H * d.E;
+  int* s_total = s_scan;
+  int* s_tbase = s_scan + nb;
+  for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+    int run = 0;
+    for (int blk = 0; blk < d.nblk; ++blk) {
+      int c = blockcnt[(size_t)blk * nb + b];
+      blockoff[(size_t)blk * nb + b] = run;
+      run += c;
+    }
+    s_total[b] = run;
+  }
+  __syncthreads();
+  for (int g = threadIdx.x; g < 2 * d.H; g += blockDim.x) {
+    int run = 0;
+    for (int e = 0; e < d.E; ++e) {
+      offsets[g * (d.E + 1) + e] = run;
+      run += s_total[g * d.E + e];
+    }
+    offsets[g * (d.E + 1) + d.E] = run;
+  }
+  if (threadIdx.x < 2) {                     // tile bases per side
+    const int side = threadIdx.x;
+    int run = 0;
+    for (int b = side * d.H * d.E; b < (side + 1) * d.H * d.E; ++b) {
+      s_tbase[b] = run;
+      run += (s_total[b] + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
+    }
+    ntiles[side] = run;
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+    const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
+    int start = 0;
+    for (int e2 = 0; e2 < e; ++e2) start += s_total[b - e + e2];
+    const int cnt = s_total[b];
+    ShTile* tp = tiles + (size_t)side * d.max_tiles + s_tbase[b];
+    for (int r = 0, i = 0; r < cnt; r += SH_TILE_ROWS, ++i) {
+      ShTile tl;
+      tl.h = h; tl.e = e; tl.row0 = start + r;
+      tl.nrows = min(SH_TILE_ROWS, cnt - r);
+      tp[i] = tl;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Bucket sort, step 2: stable scatter.  Block b owns tokens [b*128, b*128+128); thread =
+// token.  Within a bucket tokens stay in ascending order.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SH_TILE_ROWS)
+sh_sort_scatter_kernel(const int* __restrict__ idx, const float* __restrict__ gate,
+                       const int* __restrict__ blockoff, const int* __restrict__ offsets,
+                       int* __restrict__ lists, float* __restrict__ lgate, ShDims d) {
+  __shared__ int s_wcnt[SH_TILE_ROWS / 32][32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * SH_TILE_ROWS + threadIdx.x;
+  const int nb = 2 * d.H * d.E;
+  const bool live = t < d.N;
+  for (int grp = 0; grp < 2 * d.H; ++grp) {
+    const int side = grp / d.H, h = grp % d.H;
+    const size_t sel = (((size_t)side * d.N + t) * d.H + h) * d.k;
+    unsigned mask = 0;
+    if (live)
+      for (int j = 0; j < d.k; ++j) mask |= 1u << idx[sel + j];
+    __syncthreads();                         // s_wcnt free again
+    for (int e = 0; e < d.E; ++e) {
+      unsigned bal = __ballot_sync(0xffffffffu, (mask >> e) & 1u);
+      if (lane == 0) s_wcnt[warp][e] = __popc(bal);
+    }
+    __syncthreads();
+    for (int e = 0; e < d.E; ++e) {
+      const bool mine = (mask >> e) & 1u;
+      const unsigned bal = __ballot_sync(0xffffffffu, mine);
+      if (mine) {
+        int pos = __popc(bal & ((1u << lane) - 1u));
+        for (int w = 0; w < warp; ++w) pos += s_wcnt[w][e];
+        float g = 0.f;
+        for (int j = 0; j < d.k; ++j)
+          if (idx[sel + j] == e) g = gate[sel + j];
+        const int dst = offsets[grp * (d.E + 1) + e] + blockoff[(size_t)blockIdx.x * nb + grp * d.E + e] + pos;
+        lists[(size_t)grp * d.N * d.k + dst] = t;
+        lgate[(size_t)grp * d.N * d.k + dst] = g;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// CUDA-core GEMM, 128 x 64 x 16 tiles, 256 threads, 8 x 4 outputs per thread.
+//   acc[r, n] = sum_k A[row(r), a_col0 + k] * Bt[b_row0 + n, k]
+// A rows are addressed through an optional row list (token ids); Bt is "K-major": one row
+// of K contiguous values per output column.  The epilogue decides where acc goes.
+// ---------------------------------------------------------------------------------------
+enum { SH_EPI_QKV = 0, SH_EPI_V = 1, SH_EPI_O = 2, SH_EPI_PLAIN = 3 };
+
+struct ShGemmArgs {
+  const void* A; long lda;          // A [*, lda]
+  const void* Bt; long ldb;         // Bt [*, ldb]
+  int K;                            // reduction length
+  int ncols;                        // output columns (per group)
+  int nrows;                        // dense: number of rows; grouped: unused
+  const int* lists;                 // grouped: lists[side] base ([H, N*k]) or nullptr
+  const float* lgate;               // grouped: gates aligned with lists
+  const ShTile* tiles;              // grouped: row-tile table
+  const int* ntiles;                // grouped: number of valid tiles (device)
+  long b_group_stride;              // grouped: elements of Bt per (h*E + e)
+  int a_head_stride;                // grouped O: column offset of head h inside an A row
+  void* out0; void* out1; void* out2;
+  float qscale;
+  ShDims d;
+};
+
+template <typename TA, typename TB, typename TC, int EPI>
+__global__ void __launch_bounds__(256)
+sh_simt_gemm_kernel(ShGemmArgs g) {
+  constexpr int BM = 128, BN = 64, BK = 16;
+  __shared__ float sA[BK][BM + 4];
+  __shared__ float sB[BK][BN + 4];
+  __shared__ int s_row[BM];
+  __shared__ float s_gate[BM];
+  const int tid = threadIdx.x;
+  const ShDims& d = g.d;
+  int h = 0, e = 0, row0, nrows;
+  constexpr bool grouped = (EPI == SH_EPI_V || EPI == SH_EPI_O);
+  if (grouped) {
+    if ((int)blockIdx.x >= *g.ntiles) return;
+    ShTile tl = g.tiles[blockIdx.x];
+    h = tl.h; e = tl.e; row0 = tl.row0; nrows = tl.nrows;
+  } else {
+    row0 = blockIdx.x * BM;
+    nrows = min(BM, g.nrows - row0);
+  }
+  const int col0 = blockIdx.y * BN;
+  if (tid < BM) {
+    int r = -1; float gt = 0.f;
+    if (tid < nrows) {
+      if (grouped) {
+        size_t li = (size_t)h * d.N * d.k + row0 + tid;
+        r = g.lists[li]; gt = g.lgate[li];
+      } else {
+        r = row0 + tid;
+      }
+    }
+    s_row[tid] = r; s_gate[tid] = gt;
+  }
+  __syncthreads();
+  const TA* A = (const TA*)g.A + (EPI == SH_EPI_O ? (long)h * g.a_head_stride : 0);
+  const TB* Bt = (const TB*)g.Bt + (grouped ? (long)(h * d.E + e) * g.b_group_stride : 0);
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  const int tr = tid / 16, tc = tid % 16;   // 16 x 16 thread grid: rows tr*8.., cols tc*4..
+  for (int k0 = 0; k0 < g.K; k0 += BK) {
+    // A tile: 128 rows x 16 k: thread loads row = tid/2, 8 consecutive k
+    {
+      const int r = tid >> 1, kk = (tid & 1) * 8;
+      const int gr = s_row[r];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float v = 0.f;
+        if (gr >= 0 && k0 + kk + i < g.K) v = sh_to_float<TA>(A[(long)gr * g.lda + k0 + kk + i]);
+        sA[kk + i][r] = v;
+      }
+    }
+    {
+      const int n = tid >> 2, kk = (tid & 3) * 4;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float v = 0.f;
+        if (col0 + n < g.ncols && k0 + kk + i < g.K) v = sh_to_float<TB>(Bt[(long)(col0 + n) * g.ldb + k0 + kk + i]);
+        sB[kk + i][n] = v;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[8], b[4];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] = sA[kk][tr * 8 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = sB[kk][tc * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int lr = tr * 8 + i;
+    const int gr = s_row[lr];
+    if (gr < 0) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = col0 + tc * 4 + j;
+      if (n >= g.ncols) continue;
+      const float v = acc[i][j];
+      if (EPI == SH_EPI_QKV) {
+        // column n -> (which, head, dd); row gr -> (b, t); target layout [B, H, T, D]
+        const int HD = d.H * d.D;
+        const int which = n / HD, hh = (n % HD) / d.D, dd = n % d.D;
+        const int b = gr / d.T, t = gr % d.T;
+        TC* dst = (TC*)(which == 0 ? g.out0 : which == 1 ? g.out1 : g.out2);
+        dst[(((size_t)b * d.H + hh) * d.T + t) * d.D + dd] = sh_from_float<TC>(which == 0 ? v * g.qscale : v);
+      } else if (EPI == SH_EPI_V) {
+        const int b = gr / d.T, t = gr % d.T;
+        atomicAdd((TC*)g.out0 + (((size_t)b * d.H + h) * d.T + t) * d.D + n, sh_from_float<TC>(s_gate[lr] * v));
+      } else if (EPI == SH_EPI_O) {
+        atomicAdd((float*)g.out0 + (size_t)gr * d.M + n, s_gate[lr] * v);
+      } else {
+        ((float*)g.out0)[(size_t)gr * g.ncols + n] = v;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// CUDA-core causal attention (Eq. 1 with the autoregressive mask): one warp per query row,
+// keys in chunks of 32 (lane = key), online softmax in base 2 (Q carries log2(e)/sqrt(D)).
+// Q, K, V [B, H, T, D]; Ahat [B*T, H, D].
+// ---------------------------------------------------------------------------------------
+template <typename TM>
+__global__ void __launch_bounds__(128)
+sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, const TM* __restrict__ V,
+                         TM* __restrict__ Ahat, ShDims d) {
+  __shared__ float s_q[4][128];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long qi = (long)blockIdx.x * 4 + warp;          // index over (b, h, t)
+  const long total = (long)d.B * d.H * d.T;
+  if (qi >= total) return;
+  const int t = (int)(qi % d.T);
+  const long bh = qi / d.T;
+  const TM* q = Q + qi * d.D;
+  const TM* Kb = K + bh * d.T * d.D;
+  const TM* Vb = V + bh * d.T * d.D;
+  for (int i = lane; i < d.D; i += 32) s_q[warp][i] = sh_to_float<TM>(q[i]);
+  __syncwarp();
+  float o[4] = {0.f, 0.f, 0.f, 0.f};                    // lane owns d = lane + 32*i
+  float m = -INFINITY, l = 0.f;
+  for (int s0 = 0; s0 <= t; s0 += 32) {
+    const int s = s0 + lane;
+    float sc = -INFINITY;
+    if (s <= t) {
+      const TM* kr = Kb + (long)s * d.D;
+      float a = 0.f;
+      for (int i = 0; i < d.D; ++i) a = fmaf(s_q[warp][i], sh_to_float<TM>(kr[i]), a);
+      sc = a;
+    }
+    float cm = sc;
+#pragma unroll
+    for (int x = 16; x > 0; x >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, x));
+    const float mn = fmaxf(m, cm);
+    const float alpha = exp2f(m - mn);                  // m = -inf first time -> 0
+    const float p = (s <= t) ? exp2f(sc - mn) : 0.f;
+    float ps = p;
+#pragma unroll
+    for (int x = 16; x > 0; x >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, x);
+    l = l * alpha + ps;
+    m = mn;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o[i] *= alpha;
+    const int cnt = min(32, t - s0 + 1);
+    for (int j = 0; j < cnt; ++j) {
+      const float pj = __shfl_sync(0xffffffffu, p, j);
+      const TM* vr = Vb + (long)(s0 + j) * d.D;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (lane + 32 * i < d.D) o[i] = fmaf(pj, sh_to_float<TM>(vr[lane + 32 * i]), o[i]);
+    }
+  }
+  const int b = (int)(bh / d.H), h = (int)(bh % d.H);
+  TM* dst = Ahat + (((long)b * d.T + t) * d.H + h) * d.D;
+  const float inv = 1.f / l;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (lane + 32 * i < d.D) dst[lane + 32 * i] = sh_from_float<TM>(o[i] * inv);
+}

@@ -1,0 +1,75 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C-ABI binding and
+the fp64 oracle on the same seeded inputs, and compare stage by stage."""
+import numpy as np
+import torch
+
+from oracle.switchhead_oracle import switchhead_forward
+from paper_2312_07987_b200 import binding, inputs
+
+# Tolerances.  Outputs: max-abs error relative to the RMS of the oracle output, 1e-4 for the
+# fp32 configuration and 2e-2 for bf16 storage (fp32 accumulation, fp16 intermediates).
+TOL_Y = {inputs.DTYPE_F32: 1e-4, inputs.DTYPE_BF16: 2e-2}
+
+
+def oracle_for(inp, batches=None):
+    x = inp.x if batches is None else inp.x[batches]
+    return switchhead_forward(x, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, inp.cfg.k,
+                              inp.bias_s, inp.bias_d)
+
+
+def rel_rms_err(got, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.abs(np.asarray(got, dtype=np.float64) - ref).max() / np.sqrt((ref ** 2).mean()))
+
+
+def check_selection(idx_gpu, gate_gpu, ref, N):
+    """idx_gpu, gate_gpu [2, N, H, k] (numpy); ref: oracle stages for the same N tokens.
+    The selected SET must match bit-exactly; gates are compared per expert."""
+    for side, (ik, gk) in enumerate((("idxS", "gateS"), ("idxD", "gateD"))):
+        gi = idx_gpu[side].astype(np.int64)
+        order = np.argsort(gi, axis=-1, kind="stable")
+        gi_sorted = np.take_along_axis(gi, order, -1)
+        gg_sorted = np.take_along_axis(gate_gpu[side].astype(np.float64), order, -1)
+        ri = ref[ik].astype(np.int64)
+        rorder = np.argsort(ri, axis=-1, kind="stable")
+        ri_sorted = np.take_along_axis(ri, rorder, -1)
+        rg_sorted = np.take_along_axis(ref[gk], rorder, -1)
+        assert np.array_equal(gi_sorted, ri_sorted), f"side {side}: selected expert sets differ"
+        assert np.abs(gg_sorted - rg_sorted).max() <= 1e-6, f"side {side}: gate values differ"
+
+
+def check_lists(off_gpu, lists_gpu, ref):
+    for side, (ok, lk) in enumerate((("offsetsS", "listsS"), ("offsetsD", "listsD"))):
+        assert np.array_equal(off_gpu[side], ref[ok]), f"side {side}: offsets differ"
+        assert np.array_equal(lists_gpu[side], ref[lk]), f"side {side}: token lists differ"
+
+
+def run_layer(inp, device="cuda"):
+    cfg = inp.cfg
+    layer = binding.layer_from_inputs(inp, device=device)
+    x = binding.to_device(inp.x, cfg.dtype, device)
+    y = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0, "device status word reports a failed kernel"
+    return layer, x, y
+
+
+def check_stages(layer, ref, cfg, batches=None):
+    """Q, K, V, Ahat of the CUDA path against the oracle (fp16 storage on the bf16 path)."""
+    D = cfg.d_head
+    qs = np.log2(np.e) / np.sqrt(D)
+    sel = slice(None) if batches is None else batches
+    rel = 2e-5 if cfg.dtype == inputs.DTYPE_F32 else 2.0 ** -10
+    for name, key, scale in (("Q", "Q", qs), ("K", "K", 1.0), ("V", "V", 1.0)):
+        got = layer.sh_debug_buffer(name).float().cpu().numpy().astype(np.float64)   # [B,H,T,D]
+        got = got.transpose(0, 2, 1, 3)[sel]
+        want = ref[key] * scale
+        tol = rel * np.abs(want) + 3e-4 * np.sqrt((want ** 2).mean())
+        bad = np.abs(got - want) > tol
+        assert not bad.any(), f"{name}: {bad.sum()} elements off, worst {np.abs(got - want).max():.3e}"
+    got = layer.sh_debug_buffer("AHAT").float().cpu().numpy().astype(np.float64)
+    B, T, H, _ = ref["Ahat"].shape
+    got = got.reshape(-1, T, H, D)[sel]
+    want = ref["Ahat"]
+    err = np.abs(got - want).max() / np.sqrt((want ** 2).mean())
+    assert err < (1e-4 if cfg.dtype == inputs.DTYPE_F32 else 1e-2), f"Ahat rel err {err:.3e}"

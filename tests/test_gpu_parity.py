@@ -1,0 +1,125 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the fp64 oracle, element by
+element, on the seeded synthetic workloads and on edge cases."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_07987_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def full_check(inp, check_stage_buffers=True, batches=None):
+    cfg = inp.cfg
+    B, T = inp.x.shape[:2]
+    layer, x, y = pu.run_layer(inp)
+    ref = pu.oracle_for(inp, batches)
+    yb = y.cpu().numpy() if batches is None else y.cpu().numpy()[batches]
+    idx, gate, off, lists = (t.cpu().numpy() for t in layer.sh_gate_topk(x))
+    torch.cuda.synchronize()
+    N = B * T
+    if batches is None:
+        pu.check_selection(idx, gate, ref, N)
+        pu.check_lists(off, lists, ref)
+    else:
+        H, k = cfg.n_heads, cfg.k
+        tok = np.concatenate([np.arange(b * T, (b + 1) * T) for b in batches])
+        pu.check_selection(idx[:, tok], gate[:, tok], ref, tok.size)
+    if check_stage_buffers:
+        y2 = layer.sh_forward(x)          # refresh the intermediates after sh_gate_topk
+        torch.cuda.synchronize()
+        pu.check_stages(layer, ref, cfg, batches)
+    err = pu.rel_rms_err(yb, ref["y"])
+    assert err < pu.TOL_Y[cfg.dtype], f"output max-abs error / rms = {err:.3e}"
+    layer.close()
+    return err
+
+
+def test_tiny_f32_full():
+    full_check(inputs.make_inputs(inputs.CONFIGS["tiny_f32"]))
+
+
+@pytest.mark.parametrize("T,E,k,H,D,M,B", [(1, 4, 2, 2, 32, 128, 1), (2, 1, 1, 1, 32, 64, 3), (17, 5, 5, 2, 64, 128, 2),
+                                             (129, 2, 1, 3, 128, 192, 1), (300, 32, 7, 1, 32, 64, 1)])
+def test_f32_edge_shapes(T, E, k, H, D, M, B):
+    cfg = inputs.LayerConfig("edge", inputs.DTYPE_F32, B, T, M, H, D, E, k, seed=100 + T)
+    full_check(inputs.make_inputs(cfg))
+
+
+def test_f32_gate_bias():
+    cfg = inputs.LayerConfig("edge_bias", inputs.DTYPE_F32, 2, 40, 128, 2, 32, 8, 3, seed=7, zipf_bias=1.2)
+    full_check(inputs.make_inputs(cfg))
+
+
+def test_small_bf16_full():
+    full_check(inputs.make_inputs(inputs.CONFIGS["small_bf16"]))
+
+
+def test_c4_262m_bf16_full():
+    full_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"]))
+
+
+def test_long_ctx_bf16_full_size_sampled_sequences():
+    inp = inputs.make_inputs(inputs.CONFIGS["long_ctx_bf16"])
+    full_check(inp, batches=[1])
+
+
+def test_wide_skew_bf16_full_size_sampled_sequences():
+    inp = inputs.make_inputs(inputs.CONFIGS["wide_skew_bf16"])
+    full_check(inp, batches=[5])
+
+
+@pytest.mark.parametrize("T,B,E,k,H,D", [(1, 2, 4, 2, 2, 64), (100, 3, 5, 3, 2, 64), (129, 1, 4, 4, 1, 128),
+                                           (384, 2, 1, 1, 2, 128), (515, 1, 16, 4, 3, 128)])
+def test_bf16_edge_shapes(T, B, E, k, H, D):
+    cfg = inputs.LayerConfig("edge_bf16", inputs.DTYPE_BF16, B, T, 256, H, D, E, k, seed=200 + T)
+    full_check(inputs.make_inputs(cfg))
+
+
+def test_causality_on_gpu():
+    cfg = inputs.CONFIGS["small_bf16"]
+    inp = inputs.make_inputs(cfg, batch=2)
+    layer, x, y0 = pu.run_layer(inp)
+    t0 = 100
+    x2 = x.clone()
+    x2[:, t0 + 1:] = torch.randn_like(x2[:, t0 + 1:].float()).to(x2.dtype)
+    y1 = layer.sh_forward(x2)
+    torch.cuda.synchronize()
+    a, b = y0[:, :t0 + 1].cpu().numpy(), y1[:, :t0 + 1].cpu().numpy()
+    rms = np.sqrt((a.astype(np.float64) ** 2).mean())
+    assert np.abs(a - b).max() / rms < 1e-3          # only atomics-order noise
+    assert not np.allclose(y0[:, t0 + 1:].cpu().numpy(), y1[:, t0 + 1:].cpu().numpy())
+    layer.close()
+
+
+def test_forward_is_repeatable_and_selection_deterministic():
+    inp = inputs.make_inputs(inputs.CONFIGS["small_bf16"], batch=4)
+    layer, x, y0 = pu.run_layer(inp)
+    r0 = [t.clone() for t in layer.sh_gate_topk(x)]
+    y1 = layer.sh_forward(x)
+    r1 = layer.sh_gate_topk(x)
+    torch.cuda.synchronize()
+    for a, b in zip(r0, r1):
+        assert torch.equal(a, b)
+    rms = y0.double().pow(2).mean().sqrt().item()
+    assert (y0 - y1).abs().max().item() / rms < 1e-3
+    layer.close()
+
+
+def test_dense_comparator_matches_dense_mha_oracle():
+    from oracle.switchhead_oracle import dense_mha_forward
+    from paper_2312_07987_b200 import binding
+    for dtype, M, H, D, B, T, tol in ((inputs.DTYPE_F32, 128, 4, 32, 2, 50, 1e-4), (inputs.DTYPE_BF16, 256, 4, 64, 2, 200, 2e-2)):
+        Wq, Wk, Wv, Wo = inputs.make_dense_mha_weights(M, H, D, seed=5, dtype=dtype)
+        rng = np.random.Generator(np.random.PCG64(6))
+        x = inputs._store(rng.standard_normal((B, T, M)), dtype)
+        ref = dense_mha_forward(x, Wq, Wk, Wv, Wo)
+        L = binding.Layer(M, H, D, dense=True)
+        L.sh_configure(dtype, B, T)
+        dv = lambda a: binding.to_device(a, dtype)
+        L.sh_set_weights(dv(Wq), dv(Wk), dv(Wv[:, None]), dv(Wo[:, None]))
+        y = L.sh_forward(dv(x)).cpu().numpy()
+        assert L.sh_last_status() == 0
+        assert pu.rel_rms_err(y, ref) < tol
+        L.close()
