@@ -1,11 +1,190 @@
-// Tensor-core path of the bf16 configuration (interim: routes to the CUDA-core stages).
-#include "sh_internal.cuh"
+// Tensor-core (tcgen05) path of the bf16 configuration: tensor maps and launch sequence.
+#include <cstdlib>
+#include <new>
 
-int sh_tc_prepare(sh_layer* L) { (void)L; return SH_OK; }
-void sh_tc_release(sh_layer* L) { (void)L; }
-int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
-  return sh_simt_run_bf16(L, SH_STAGE_ALL, x, out, st);
+#include "sh_internal.cuh"
+#include "sh_tc_gemm.cuh"
+
+using namespace shtc;
+
+#define SH_CUDA_CHECK(expr)                                                          \
+  do {                                                                               \
+    cudaError_t _e = (expr);                                                         \
+    if (_e != cudaSuccess) {                                                         \
+      sh_set_error("%s failed: %s", #expr, cudaGetErrorString(_e));                  \
+      return SH_ERR_CUDA;                                                            \
+    }                                                                                \
+  } while (0)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
 }
+
+// 2-D row-major tensor [outer, inner] of 16-bit elements, 128-byte swizzle, box = box_outer
+// rows of box_inner (= 64) elements.
+int sh_tc_encode_2d(CUtensorMap* map, int elem_kind, const void* base, uint64_t inner, uint64_t outer,
+                    uint64_t outer_stride_bytes, uint32_t box_inner, uint32_t box_outer) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { sh_set_error("cuTensorMapEncodeTiled is not available from the driver"); return SH_ERR_CUDA; }
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {outer_stride_bytes};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(map, elem_kind == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { sh_set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return SH_ERR_CUDA; }
+  return SH_OK;
+}
+
+struct TcState {
+  CUtensorMap map_wqk, map_wv, map_wo, map_ahat;
+  int qk_bn, o_bn;
+  int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
+};
+
+constexpr int QK_STAGES = 4;
+
+template <typename K>
+static int set_smem(K kernel, int bytes) {
+  SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  return SH_OK;
+}
+
+void sh_tc_release(sh_layer* L) {
+  if (L && L->tc) {
+    delete (TcState*)L->tc;
+    L->tc = nullptr;
+  }
+}
+
+int sh_tc_prepare(sh_layer* L) {
+  sh_tc_release(L);
+  TcState* S = new (std::nothrow) TcState();
+  if (!S) { sh_set_error("out of host memory"); return SH_ERR_INVALID_ARG; }
+  L->tc = S;
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const int HD = d.H * d.D;
+  const int nproj = L->dense ? 3 : 2;
+  S->qk_bn = 128;
+  S->o_bn = 128;
+  const char* env = getenv("SH_SIMT_STAGES");
+  S->simt_mask = env ? atoi(env) : 0;
+  int rc;
+  if ((rc = sh_tc_encode_2d(&S->map_wqk, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, S->qk_bn))) return rc;
+  if (!L->dense) {
+    if ((rc = sh_tc_encode_2d(&S->map_wv, 0, ws + L->o.wv, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, S->o_bn))) return rc;
+  } else {
+    if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, S->o_bn))) return rc;
+  }
+  if ((rc = sh_tc_encode_2d(&S->map_ahat, 1, ws + L->o.ahat, HD, d.N, (uint64_t)HD * 2, 64, 128))) return rc;
+  return SH_OK;
+}
+
 int sh_tc_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
   return sh_simt_run_bf16(L, SH_STAGE_GATE, x, nullptr, st);
+}
+
+template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16>
+static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, dim3 grid, cudaStream_t st) {
+  auto kern = sh_tc_gemm_kernel<BN, STAGES, MODE, A_BF16, B_BF16>;
+  constexpr int smem = GemmSmem<BN, STAGES>::TOTAL;
+  static bool configured = false;
+  if (!configured) {
+    int rc = set_smem(kern, smem);
+    if (rc != SH_OK) return rc;
+    configured = true;
+  }
+  kern<<<grid, 192, smem, st>>>(mapA, mapB, g);
+  return SH_OK;
+}
+
+int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
+  TcState* S = (TcState*)L->tc;
+  if (!S) { sh_set_error("tensor-core state missing: call sh_set_weights first"); return SH_ERR_NOT_CONFIGURED; }
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const int HD = d.H * d.D;
+  int rc;
+  const int simt = S->simt_mask;
+  int* status = (int*)(ws + L->o.status);
+
+  if (!L->dense) {
+    if ((rc = sh_tc_gate_sort(L, x, st))) return rc;
+  }
+  CUtensorMap map_x;
+  if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
+
+  // ---- Q, K (and V for the dense comparator) ------------------------------------------------
+  if (simt & SH_STAGE_QK) {
+    if ((rc = sh_simt_run_bf16(L, SH_STAGE_QK, x, out, st))) return rc;
+  } else {
+    TcGemmArgs g{};
+    g.d = d; g.K = d.M; g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
+    g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
+    g.qscale = 1.4426950408889634f / sqrtf((float)d.D);
+    g.status = status;
+    dim3 grid(d.nblk, (g.ncols + 127) / 128);
+    if ((rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st))) return rc;
+    L->launches += 1;
+  }
+  // ---- value experts ---------------------------------------------------------------------------
+  if (!L->dense) {
+    if (simt & SH_STAGE_V) {
+      if ((rc = sh_simt_run_bf16(L, SH_STAGE_V, x, out, st))) return rc;
+    } else {
+      SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * HD * 2, st));
+      TcGemmArgs g{};
+      g.d = d; g.K = d.M; g.ncols = d.D;
+      g.A = x; g.lda = d.M;
+      g.lists = (const int*)(ws + L->o.lists); g.lgate = (const float*)(ws + L->o.lgate);
+      g.tiles = (const ShTile*)(ws + L->o.tiles); g.ntiles = (const int*)(ws + L->o.ntiles);
+      g.b_rows_per_group = d.D; g.out0 = ws + L->o.v; g.status = status;
+      dim3 grid(d.max_tiles, 1);
+      if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
+      else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
+      if (rc) return rc;
+      L->launches += 2;
+    }
+  }
+  // ---- attention ---------------------------------------------------------------------------------
+  if ((rc = sh_simt_run_bf16(L, SH_STAGE_ATTN, x, out, st))) return rc;
+  // ---- output experts ----------------------------------------------------------------------------
+  if (simt & SH_STAGE_O) {
+    if ((rc = sh_simt_run_bf16(L, SH_STAGE_O, x, out, st))) return rc;
+  } else if (!L->dense) {
+    SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
+    TcGemmArgs g{};
+    g.d = d; g.K = d.D; g.ncols = d.M;
+    g.A = ws + L->o.ahat; g.lda = HD;
+    const size_t side1 = (size_t)d.H * d.N * d.k;
+    g.lists = (const int*)(ws + L->o.lists) + side1; g.lgate = (const float*)(ws + L->o.lgate) + side1;
+    g.tiles = (const ShTile*)(ws + L->o.tiles) + d.max_tiles; g.ntiles = (const int*)(ws + L->o.ntiles) + 1;
+    g.b_rows_per_group = d.M; g.out0 = out; g.status = status;
+    dim3 grid(d.max_tiles, (d.M + 127) / 128);
+    if ((rc = launch_gemm<128, 3, GEMM_O, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
+    L->launches += 2;
+  } else {
+    TcGemmArgs g{};
+    g.d = d; g.K = HD; g.ncols = d.M; g.nrows = d.N; g.out0 = out; g.status = status;
+    dim3 grid(d.nblk, (d.M + 127) / 128);
+    if ((rc = launch_gemm<128, 4, GEMM_PLAIN, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
+    L->launches += 1;
+  }
+  SH_CUDA_CHECK(cudaGetLastError());
+  return SH_OK;
 }

@@ -1,0 +1,236 @@
+// tcgen05 GEMM kernels of the bf16 configuration: the dense Q/K projection, the grouped
+// value-expert projection and the grouped output-expert projection with its gate-weighted
+// scatter-add epilogue.  One 128 x BN output tile per CTA, accumulator in TMEM, operands
+// staged in 128-byte-swizzled shared memory: B always by TMA, A by TMA (dense rows) or by
+// cp.async row gathers (rows addressed through a per-expert token list).
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
+// warps 2..5 = A-row gatherers during the main loop (grouped modes) and the epilogue.
+#pragma once
+#include "sh_tc_prims.cuh"
+
+namespace shtc {
+
+enum { GEMM_QKV = 0, GEMM_V = 1, GEMM_O = 2, GEMM_PLAIN = 3 };
+
+struct TcGemmArgs {
+  ShDims d;
+  int K;                 // reduction length (multiple of 64)
+  int ncols;             // output columns (per group in grouped modes)
+  int nrows;             // dense modes: rows of A
+  // grouped modes
+  const void* A;         // gathered operand base (bf16 x or fp16 Ahat)
+  long lda;              // elements per A row
+  const int* lists;      // [H, N*k] token ids of this side
+  const float* lgate;    // gates aligned with lists
+  const ShTile* tiles;
+  const int* ntiles;
+  int b_rows_per_group;  // rows of the B tensor map per (h*E + e)
+  void* out0; void* out1; void* out2;
+  float qscale;
+  int* status;
+};
+
+constexpr int GEMM_BM = 128;
+constexpr int GEMM_BK = 64;
+
+template <int BN, int STAGES>
+struct GemmSmem {
+  static constexpr int A_BYTES = GEMM_BM * GEMM_BK * 2;
+  static constexpr int B_BYTES = BN * GEMM_BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int BAR_OFF = STAGES * STAGE_BYTES;
+  static constexpr int TOTAL = BAR_OFF + 256 + 1024;   // + barriers + alignment slack
+};
+
+template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16>
+__global__ void __launch_bounds__(192)
+sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcGemmArgs g) {
+  using SM = GemmSmem<BN, STAGES>;
+  constexpr bool GATHER = (MODE == GEMM_V || MODE == GEMM_O);
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* sgen = smem_raw + (sbase - smem_u32(smem_raw));
+  uint64_t* full_bar = (uint64_t*)(sgen + SM::BAR_OFF);
+  uint64_t* empty_bar = full_bar + STAGES;
+  uint64_t* tmem_full = empty_bar + STAGES;
+  uint32_t* tmem_slot = (uint32_t*)(tmem_full + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const ShDims& d = g.d;
+  int th = 0, te = 0, row0, nrows;
+  if (GATHER) {
+    if ((int)blockIdx.x >= *g.ntiles) return;          // whole CTA leaves before any barrier
+    const ShTile tl = g.tiles[blockIdx.x];
+    th = tl.h; te = tl.e; row0 = tl.row0; nrows = tl.nrows;
+  } else {
+    row0 = blockIdx.x * GEMM_BM;
+    nrows = min(GEMM_BM, g.nrows - row0);
+  }
+  const int col0 = blockIdx.y * BN;
+  const int KB = g.K / GEMM_BK;
+  bool dead = false;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], GATHER ? 129 : 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(tmem_full, 1);
+    fence_barrier_init();
+    tma_prefetch_desc(&mapB);
+    if (!GATHER) tma_prefetch_desc(&mapA);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int brow = (GATHER ? (th * d.E + te) * g.b_rows_per_group : 0) + col0;
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % STAGES;
+        if (!mbar_wait(&empty_bar[s], ((kb / STAGES) & 1) ^ 1, g.status, dead)) break;
+        const uint32_t sa = sbase + s * SM::STAGE_BYTES, sb = sa + SM::A_BYTES;
+        mbar_expect_tx(&full_bar[s], GATHER ? SM::B_BYTES : SM::STAGE_BYTES);
+        if (!GATHER) tma_load_2d(sa, &mapA, &full_bar[s], kb * GEMM_BK, row0);
+        tma_load_2d(sb, &mapB, &full_bar[s], kb * GEMM_BK, brow);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_f16(GEMM_BM, BN, A_BF16, B_BF16, 0);
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % STAGES;
+        if (!mbar_wait(&full_bar[s], (kb / STAGES) & 1, g.status, dead)) break;
+        tc_fence_after();
+        const uint32_t sa = sbase + s * SM::STAGE_BYTES, sb = sa + SM::A_BYTES;
+        const uint64_t adesc = make_desc_k_sw128(sa), bdesc = make_desc_k_sw128(sb);
+#pragma unroll
+        for (int k = 0; k < GEMM_BK / 16; ++k)
+          umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+        umma_commit(&empty_bar[s]);
+      }
+      umma_commit(tmem_full);
+    }
+  } else {
+    const int et = threadIdx.x - 64;                   // 0..127
+    if (GATHER) {
+      // thread -> 16-byte chunk c of rows rb, rb+16, ... (8 threads cover one 128-byte row)
+      const int c = et & 7, rb = et >> 3;
+      const char* src[8];
+      uint32_t ok[8];
+      const int abytes = A_BF16 ? 2 : 2;
+      const long acol = (MODE == GEMM_O) ? (long)th * d.D : 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int r = rb + 16 * i;
+        int tok = 0;
+        ok[i] = 0;
+        if (r < nrows) { tok = g.lists[(size_t)th * d.N * d.k + row0 + r]; ok[i] = 16; }
+        src[i] = (const char*)g.A + ((long)tok * g.lda + acol + c * 8) * abytes;
+      }
+      const uint32_t dsw = (uint32_t)((c ^ (rb & 7)) << 4);
+      int arrived = 0;
+      for (int kb = 0; kb < KB; ++kb) {
+        const int s = kb % STAGES;
+        if (!mbar_wait(&empty_bar[s], ((kb / STAGES) & 1) ^ 1, g.status, dead)) break;
+        const uint32_t sa = sbase + s * SM::STAGE_BYTES;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          cp_async_16(sa + (rb + 16 * i) * 128 + dsw, src[i] + (long)kb * GEMM_BK * abytes, ok[i]);
+        cp_async_commit();
+        if (kb >= 2) {
+          cp_async_wait<2>();
+          fence_proxy_async_smem();
+          mbar_arrive(&full_bar[arrived % STAGES]);
+          ++arrived;
+        }
+      }
+      cp_async_wait<0>();
+      fence_proxy_async_smem();
+      if (!dead)
+        for (; arrived < KB; ++arrived) mbar_arrive(&full_bar[arrived % STAGES]);
+    }
+    // ---- epilogue: thread = accumulator row = TMEM lane --------------------------------------
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const bool live = r < nrows;
+    int tok = 0;
+    float gate = 0.f;
+    if (live) {
+      if (GATHER) {
+        const size_t li = (size_t)th * d.N * d.k + row0 + r;
+        tok = g.lists[li];
+        gate = g.lgate[li];
+      } else {
+        tok = row0 + r;
+      }
+    }
+    if (mbar_wait(tmem_full, 0, g.status, dead)) {
+      tc_fence_after();
+      const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
+      const int bb = tok / d.T, tt = tok % d.T;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(trow + c0, v);
+        tmem_ld_wait();
+        const int n0 = col0 + c0;
+        if (!live || n0 >= g.ncols) continue;
+        if (MODE == GEMM_QKV) {
+          const int HD = d.H * d.D;
+          const int which = n0 / HD, hh = (n0 % HD) / d.D, dd = n0 % d.D;
+          __half* dst = (__half*)(which == 0 ? g.out0 : which == 1 ? g.out1 : g.out2) +
+                        (((size_t)bb * d.H + hh) * d.T + tt) * d.D + dd;
+          const float sc = which == 0 ? g.qscale : 1.f;
+          uint32_t p[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * sc, __uint_as_float(v[2 * i + 1]) * sc);
+            p[i] = *reinterpret_cast<uint32_t*>(&hv);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4*>(dst + 8 * i) = make_uint4(p[4 * i], p[4 * i + 1], p[4 * i + 2], p[4 * i + 3]);
+        } else if (MODE == GEMM_V) {
+          __half* dst = (__half*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D + n0;
+          uint32_t p[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * gate, __uint_as_float(v[2 * i + 1]) * gate);
+            p[i] = *reinterpret_cast<uint32_t*>(&hv);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) red_add_v4_f16x2(dst + 8 * i, p[4 * i], p[4 * i + 1], p[4 * i + 2], p[4 * i + 3]);
+        } else if (MODE == GEMM_O) {
+          float* dst = (float*)g.out0 + (size_t)tok * d.M + n0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            red_add_v4_f32(dst + 4 * i, __uint_as_float(v[4 * i]) * gate, __uint_as_float(v[4 * i + 1]) * gate,
+                           __uint_as_float(v[4 * i + 2]) * gate, __uint_as_float(v[4 * i + 3]) * gate);
+        } else {
+          float* dst = (float*)g.out0 + (size_t)tok * g.ncols + n0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<float4*>(dst + 4 * i) =
+                make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                            __uint_as_float(v[4 * i + 3]));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_d, BN);
+  }
+}
+
+}  // namespace shtc

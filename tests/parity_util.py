@@ -64,12 +64,18 @@ def check_stages(layer, ref, cfg, batches=None):
         got = layer.sh_debug_buffer(name).float().cpu().numpy().astype(np.float64)   # [B,H,T,D]
         got = got.transpose(0, 2, 1, 3)[sel]
         want = ref[key] * scale
-        tol = rel * np.abs(want) + 3e-4 * np.sqrt((want ** 2).mean())
+        # V sums k gate-weighted fp16 contributions, each addition rounding to fp16
+        r = rel * (cfg.k if name == "V" and cfg.dtype != inputs.DTYPE_F32 else 1)
+        tol = r * np.abs(want) + max(3e-4, r) * np.sqrt((want ** 2).mean())
         bad = np.abs(got - want) > tol
         assert not bad.any(), f"{name}: {bad.sum()} elements off, worst {np.abs(got - want).max():.3e}"
     got = layer.sh_debug_buffer("AHAT").float().cpu().numpy().astype(np.float64)
     B, T, H, _ = ref["Ahat"].shape
     got = got.reshape(-1, T, H, D)[sel]
     want = ref["Ahat"]
-    err = np.abs(got - want).max() / np.sqrt((want ** 2).mean())
-    assert err < (1e-4 if cfg.dtype == inputs.DTYPE_F32 else 1e-2), f"Ahat rel err {err:.3e}"
+    # Ahat inherits V's rounding (rows near t = 0 are single V rows) plus its own fp16 store
+    # and the effect of fp16 Q, K on the softmax weights (logit error ~ 2^-11 |q.k|)
+    r = 1e-2 if cfg.dtype != inputs.DTYPE_F32 else 4e-5
+    tol = r * (np.abs(want) + np.sqrt((want ** 2).mean()))
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), f"Ahat: {bad.sum()} elements off, worst {np.abs(got - want).max():.3e}"
