@@ -105,6 +105,12 @@ int sh_set_weights(sh_layer* layer, const void* Wq, const void* Wk, const void* 
  * out [B, T, d_model] fp32.  out is fully overwritten.  Enqueues kernels only. */
 int sh_forward(sh_layer* layer, const void* x, void* out, void* stream);
 
+/* Measurement aid: sh_forward with CUDA events recorded on `stream` at the stage boundaries;
+ * waits for the stream, then writes to the HOST array stage_ms[6] the milliseconds of
+ * {gate + top-k + sort, Q/K projection, value experts, attention, output experts, whole
+ * pass}.  Creates and destroys its events, so unlike sh_forward it must not be stream-captured. */
+int sh_forward_timed(sh_layer* layer, const void* x, void* out, void* stream, float* stage_ms);
+
 /* Gate stage alone, with its results exposed (any output pointer may be NULL):
  *   idx     [2, N, H, k] int32  selected experts; side 0 = source, 1 = destination;
  *                               in rank order (largest logit first, ties lower index first)

@@ -22,7 +22,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
 EXPORTS = ["sh_create", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
-           "sh_set_weights", "sh_forward", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
+           "sh_set_weights", "sh_forward", "sh_forward_timed", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
            "sh_launch_count", "sh_last_error", "sh_destroy"]
 
 
@@ -46,6 +46,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_set_weights.argtypes = [vp] * 10
     lib.sh_forward.restype = i32
     lib.sh_forward.argtypes = [vp, vp, vp, vp]
+    lib.sh_forward_timed.restype = i32
+    lib.sh_forward_timed.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float)]
     lib.sh_gate_topk.restype = i32
     lib.sh_gate_topk.argtypes = [vp] * 7
     lib.sh_debug_buffer.restype = i32
@@ -126,6 +128,12 @@ class Layer:
             out = torch.empty(x.shape, dtype=torch.float32, device=x.device)
         _check(lib.sh_forward(self.handle, _ptr(x), _ptr(out), _stream()))
         return out
+
+    def sh_forward_timed(self, x: torch.Tensor, out: torch.Tensor):
+        """Returns the six stage times in ms: gate+sort, qk, v, attention, o, total."""
+        ms = (ctypes.c_float * 6)()
+        _check(lib.sh_forward_timed(self.handle, _ptr(x), _ptr(out), _stream(), ms))
+        return list(ms)
 
     def sh_gate_topk(self, x: torch.Tensor):
         d_model, H, D, E, k = self.dims

@@ -233,10 +233,13 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   char* ws = L->ws;
   const int HD = d.H * d.D;
   const float qscale = 1.4426950408889634f / sqrtf((float)d.D);
+  const bool all = stages == SH_STAGE_ALL;
+  if (all) sh_mark(L, 0, st);
   if (!L->dense && (stages & SH_STAGE_GATE)) {
     int rc = launch_gate_sort<TI>(L, x, st);
     if (rc != SH_OK) return rc;
   }
+  if (all) sh_mark(L, 1, st);
   if (stages & SH_STAGE_QK) {
   ShGemmArgs g{};
   g.d = d;
@@ -248,6 +251,7 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_qk, 256, 0, st>>>(g);
   L->launches += 1;
   }
+  if (all) sh_mark(L, 2, st);
   if (!L->dense && (stages & SH_STAGE_V)) {
     SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * HD * sizeof(TM), st));
     ShGemmArgs v{};
@@ -259,12 +263,14 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
     sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_V><<<grid_v, 256, 0, st>>>(v);
     L->launches += 2;
   }
+  if (all) sh_mark(L, 3, st);
   if (stages & SH_STAGE_ATTN) {
     const long nq = (long)d.B * d.H * d.T;
     sh_simt_attention_kernel<TM><<<(unsigned)((nq + 3) / 4), 128, 0, st>>>((const TM*)(ws + L->o.q),
         (const TM*)(ws + L->o.k), (const TM*)(ws + L->o.v), (TM*)(ws + L->o.ahat), d);
     L->launches += 1;
   }
+  if (all) sh_mark(L, 4, st);
   if (!(stages & SH_STAGE_O)) {
   } else if (!L->dense) {
     SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
@@ -286,6 +292,7 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
     sh_simt_gemm_kernel<TM, TM, float, SH_EPI_PLAIN><<<grid_o, 256, 0, st>>>(o);
     L->launches += 1;
   }
+  if (all) sh_mark(L, 5, st);
   SH_CUDA_CHECK(cudaGetLastError());
   return SH_OK;
 }
@@ -303,6 +310,27 @@ extern "C" int sh_forward(sh_layer* L, const void* x, void* out, void* stream) {
   L->launches = 0;
   if (L->dtype == SH_F32) return forward_simt<float, float>(L, SH_STAGE_ALL, x, out, st);
   return sh_tc_forward(L, x, out, st);
+}
+
+extern "C" int sh_forward_timed(sh_layer* L, const void* x, void* out, void* stream, float* stage_ms) {
+  g_err[0] = 0;
+  if (!stage_ms) { sh_set_error("stage_ms must not be NULL"); return SH_ERR_INVALID_ARG; }
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  cudaEvent_t ev[6];
+  for (int i = 0; i < 6; ++i) SH_CUDA_CHECK(cudaEventCreate(&ev[i]));
+  L->ev = ev;
+  int rc = sh_forward(L, x, out, stream);
+  L->ev = nullptr;
+  if (rc == SH_OK) {
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) { sh_set_error("stream synchronise failed: %s", cudaGetErrorString(e)); rc = SH_ERR_CUDA; }
+  }
+  if (rc == SH_OK) {
+    for (int i = 0; i < 5; ++i) cudaEventElapsedTime(&stage_ms[i], ev[i], ev[i + 1]);
+    cudaEventElapsedTime(&stage_ms[5], ev[0], ev[5]);
+  }
+  for (int i = 0; i < 6; ++i) cudaEventDestroy(ev[i]);
+  return rc;
 }
 
 extern "C" int sh_gate_topk(sh_layer* L, const void* x, int32_t* idx, float* gate, int32_t* offsets,

@@ -39,6 +39,7 @@ struct sh_layer {
   int launches = 0;
   int sm_count = 0;
   void* tc = nullptr;      // tensor-core path state (tensor maps), owned by the layer
+  cudaEvent_t* ev = nullptr;  // when set (sh_forward_timed): 6 events recorded at the stage boundaries
 };
 
 template <typename T> __device__ __forceinline__ float sh_to_float(T v);
@@ -51,6 +52,12 @@ template <> __device__ __forceinline__ __half sh_from_float<__half>(float v) { r
 template <> __device__ __forceinline__ __nv_bfloat16 sh_from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 void sh_set_error(const char* fmt, ...);
+
+// Stage boundary marker: boundary 0 = start, 1 = after gate+sort, 2 = after Q/K, 3 = after V,
+// 4 = after attention, 5 = after the output projection.
+static inline void sh_mark(sh_layer* L, int boundary, cudaStream_t st) {
+  if (L->ev) cudaEventRecord(L->ev[boundary], st);
+}
 
 enum { SH_STAGE_GATE = 1, SH_STAGE_QK = 2, SH_STAGE_V = 4, SH_STAGE_ATTN = 8, SH_STAGE_O = 16, SH_STAGE_ALL = 31 };
 

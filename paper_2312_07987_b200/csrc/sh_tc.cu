@@ -123,9 +123,11 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   const int simt = S->simt_mask;
   int* status = (int*)(ws + L->o.status);
 
+  sh_mark(L, 0, st);
   if (!L->dense) {
     if ((rc = sh_tc_gate_sort(L, x, st))) return rc;
   }
+  sh_mark(L, 1, st);
   CUtensorMap map_x;
   if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
 
@@ -142,6 +144,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     if ((rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st))) return rc;
     L->launches += 1;
   }
+  sh_mark(L, 2, st);
   // ---- value experts ---------------------------------------------------------------------------
   if (!L->dense) {
     if (simt & SH_STAGE_V) {
@@ -161,8 +164,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       L->launches += 2;
     }
   }
+  sh_mark(L, 3, st);
   // ---- attention ---------------------------------------------------------------------------------
   if ((rc = sh_simt_run_bf16(L, SH_STAGE_ATTN, x, out, st))) return rc;
+  sh_mark(L, 4, st);
   // ---- output experts ----------------------------------------------------------------------------
   if (simt & SH_STAGE_O) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_O, x, out, st))) return rc;
@@ -185,6 +190,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     if ((rc = launch_gemm<128, 4, GEMM_PLAIN, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
     L->launches += 1;
   }
+  sh_mark(L, 5, st);
   SH_CUDA_CHECK(cudaGetLastError());
   return SH_OK;
 }

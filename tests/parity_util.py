@@ -76,6 +76,6 @@ def check_stages(layer, ref, cfg, batches=None):
     # Ahat inherits V's rounding (rows near t = 0 are single V rows) plus its own fp16 store
     # and the effect of fp16 Q, K on the softmax weights (logit error ~ 2^-11 |q.k|)
     r = 1e-2 if cfg.dtype != inputs.DTYPE_F32 else 4e-5
-    tol = r * (np.abs(want) + np.sqrt((want ** 2).mean()))
+    tol = r * (np.abs(want) + 2 * np.sqrt((want ** 2).mean()))
     bad = np.abs(got - want) > tol
     assert not bad.any(), f"Ahat: {bad.sum()} elements off, worst {np.abs(got - want).max():.3e}"
