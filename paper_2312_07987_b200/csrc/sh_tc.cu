@@ -4,6 +4,7 @@
 
 #include "sh_internal.cuh"
 #include "sh_tc_gemm.cuh"
+#include "sh_tc_attn.cuh"
 
 using namespace shtc;
 
@@ -49,7 +50,24 @@ int sh_tc_encode_2d(CUtensorMap* map, int elem_kind, const void* base, uint64_t 
   return SH_OK;
 }
 
+// 3-D tensor [n2, n1, inner] of fp16 (Q, K, V as [B*H, T, D]); box = 128 rows of 64 elements of
+// one (batch, head) slice, so rows past the end of a sequence read as zero.
+static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uint64_t n1, uint64_t n2) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { sh_set_error("cuTensorMapEncodeTiled is not available from the driver"); return SH_ERR_CUDA; }
+  cuuint64_t dims[3] = {inner, n1, n2};
+  cuuint64_t strides[2] = {inner * 2, inner * n1 * 2};
+  cuuint32_t box[3] = {64, 128, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { sh_set_error("cuTensorMapEncodeTiled (3-D) failed with CUresult %d", (int)r); return SH_ERR_CUDA; }
+  return SH_OK;
+}
+
 struct TcState {
+  CUtensorMap map_q, map_k, map_v;
   CUtensorMap map_wqk, map_wv, map_wo, map_ahat;
   int qk_bn, o_bn;
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
@@ -91,6 +109,9 @@ int sh_tc_prepare(sh_layer* L) {
   } else {
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, S->o_bn))) return rc;
   }
+  if ((rc = encode_3d_f16(&S->map_q, ws + L->o.q, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
+  if ((rc = encode_3d_f16(&S->map_k, ws + L->o.k, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
+  if ((rc = encode_3d_f16(&S->map_v, ws + L->o.v, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = sh_tc_encode_2d(&S->map_ahat, 1, ws + L->o.ahat, HD, d.N, (uint64_t)HD * 2, 64, 128))) return rc;
   return SH_OK;
 }
@@ -166,7 +187,23 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   }
   sh_mark(L, 3, st);
   // ---- attention ---------------------------------------------------------------------------------
-  if ((rc = sh_simt_run_bf16(L, SH_STAGE_ATTN, x, out, st))) return rc;
+  if (simt & SH_STAGE_ATTN) {
+    if ((rc = sh_simt_run_bf16(L, SH_STAGE_ATTN, x, out, st))) return rc;
+  } else {
+    TcAttnArgs a{};
+    a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
+    const int nq = (d.T + 127) / 128;
+    const unsigned grid = (unsigned)(nq * d.B * d.H);
+    static bool cfg128 = false, cfg64 = false;
+    if (d.D == 128) {
+      if (!cfg128) { if ((rc = set_smem(sh_tc_attention_kernel<128>, AttnSmem<128>::TOTAL))) return rc; cfg128 = true; }
+      sh_tc_attention_kernel<128><<<grid, 192, AttnSmem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+    } else {
+      if (!cfg64) { if ((rc = set_smem(sh_tc_attention_kernel<64>, AttnSmem<64>::TOTAL))) return rc; cfg64 = true; }
+      sh_tc_attention_kernel<64><<<grid, 192, AttnSmem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+    }
+    L->launches += 1;
+  }
   sh_mark(L, 4, st);
   // ---- output experts ----------------------------------------------------------------------------
   if (simt & SH_STAGE_O) {
