@@ -89,7 +89,7 @@ sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const flo
 // Bucket sort, step 1 (one block): exclusive scan of the per-block histograms over blocks,
 // per-head exclusive scan over experts, and the row-tile table of the grouped GEMMs.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 sh_sort_scan_kernel(const int* __restrict__ blockcnt, int* __restrict__ blockoff, int* __restrict__ offsets,
                     ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
   extern __shared__ int s_scan[];            // total[nb], tilebase[nb + 2]
@@ -143,7 +143,7 @@ sh_sort_scan_kernel(const int* __restrict__ blockcnt, int* __restrict__ blockoff
 // Bucket sort, step 2: stable scatter.  Block b owns tokens [b*128, b*128+128); thread =
 // token.  Within a bucket tokens stay in ascending order.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(SH_TILE_ROWS)
+static __global__ void __launch_bounds__(SH_TILE_ROWS)
 sh_sort_scatter_kernel(const int* __restrict__ idx, const float* __restrict__ gate,
                        const int* __restrict__ blockoff, const int* __restrict__ offsets,
                        int* __restrict__ lists, float* __restrict__ lgate, ShDims d) {

@@ -3,8 +3,10 @@
 #include <new>
 
 #include "sh_internal.cuh"
+#include "sh_simt.cuh"
 #include "sh_tc_gemm.cuh"
 #include "sh_tc_attn.cuh"
+#include "sh_tc_gate.cuh"
 
 using namespace shtc;
 
@@ -68,7 +70,8 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
-  CUtensorMap map_wqk, map_wv, map_wo, map_ahat;
+  CUtensorMap map_wqk, map_wv, map_wo, map_ahat, map_wgate;
+  int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
   int qk_bn, o_bn;
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
 };
@@ -109,6 +112,11 @@ int sh_tc_prepare(sh_layer* L) {
   } else {
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, S->o_bn))) return rc;
   }
+  S->gate_gp = 0;
+  if (!L->dense && (d.G + 15) / 16 * 16 <= 256) {
+    S->gate_gp = (d.G + 15) / 16 * 16;
+    if ((rc = sh_tc_encode_2d(&S->map_wgate, 0, ws + L->o.wgate, d.M, d.G, (uint64_t)d.M * 2, 64, S->gate_gp))) return rc;
+  }
   if ((rc = encode_3d_f16(&S->map_q, ws + L->o.q, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = encode_3d_f16(&S->map_k, ws + L->o.k, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = encode_3d_f16(&S->map_v, ws + L->o.v, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
@@ -116,8 +124,58 @@ int sh_tc_prepare(sh_layer* L) {
   return SH_OK;
 }
 
+constexpr int GATE_STAGES = 4;
+
+static int gate_smem_bytes(int Gp, int G) {
+  const int stage = 128 * 64 * 2 + ((Gp * 128 + 1023) & ~1023);
+  const int pipe = GATE_STAGES * stage, stag = 128 * (Gp + 1) * 4;
+  const int bar_off = ((pipe > stag ? pipe : stag) + 1023) & ~1023;
+  return bar_off + 256 + 3 * G * 4 + 1024;
+}
+
+// Gate + top-k + bucket sort.  With zero_for_forward the fused kernel also clears V and out.
+static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_forward, cudaStream_t st) {
+  TcState* S = (TcState*)L->tc;
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  int rc;
+  if (!S->gate_gp || (S->simt_mask & SH_STAGE_GATE)) {
+    if ((rc = sh_simt_run_bf16(L, SH_STAGE_GATE, x, nullptr, st))) return rc;
+    if (zero_for_forward) {
+      SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * d.H * d.D * 2, st));
+      SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
+      L->launches += 2;
+    }
+    return SH_OK;
+  }
+  CUtensorMap map_x;
+  if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
+  TcGateArgs g{};
+  g.d = d; g.Gp = S->gate_gp; g.gbias = (const float*)(ws + L->o.gbias);
+  g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
+  g.blockcnt = (int*)(ws + L->o.blockcnt); g.blockoff = (int*)(ws + L->o.blockoff);
+  g.offsets = (int*)(ws + L->o.offsets); g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
+  g.done_counter = (unsigned int*)(ws + L->o.status + 64);
+  g.zero_v = zero_for_forward ? (__half*)(ws + L->o.v) : nullptr;
+  g.zero_out = zero_for_forward ? (float*)out : nullptr;
+  g.status = (int*)(ws + L->o.status);
+  const int smem = gate_smem_bytes(S->gate_gp, d.G);
+  static int configured = 0;
+  if (configured < smem) {
+    if ((rc = set_smem(sh_tc_gate_kernel<GATE_STAGES>, smem))) return rc;
+    configured = smem;
+  }
+  sh_tc_gate_kernel<GATE_STAGES><<<d.nblk, 192, smem, st>>>(map_x, S->map_wgate, g);
+  sh_sort_scatter_kernel<<<d.nblk, SH_TILE_ROWS, 0, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
+      (const int*)(ws + L->o.blockoff), (const int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
+      (float*)(ws + L->o.lgate), d);
+  L->launches += 2;
+  return SH_OK;
+}
+
 int sh_tc_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
-  return sh_simt_run_bf16(L, SH_STAGE_GATE, x, nullptr, st);
+  if (!L->tc) { sh_set_error("tensor-core state missing: call sh_set_weights first"); return SH_ERR_NOT_CONFIGURED; }
+  return tc_gate_sort(L, x, nullptr, false, st);
 }
 
 template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16>
@@ -146,7 +204,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
 
   sh_mark(L, 0, st);
   if (!L->dense) {
-    if ((rc = sh_tc_gate_sort(L, x, st))) return rc;
+    if ((rc = tc_gate_sort(L, x, out, true, st))) return rc;
   }
   sh_mark(L, 1, st);
   CUtensorMap map_x;
@@ -171,7 +229,6 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     if (simt & SH_STAGE_V) {
       if ((rc = sh_simt_run_bf16(L, SH_STAGE_V, x, out, st))) return rc;
     } else {
-      SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * HD * 2, st));
       TcGemmArgs g{};
       g.d = d; g.K = d.M; g.ncols = d.D;
       g.A = x; g.lda = d.M;
@@ -182,7 +239,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
       else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
       if (rc) return rc;
-      L->launches += 2;
+      L->launches += 1;
     }
   }
   sh_mark(L, 3, st);
@@ -209,7 +266,6 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   if (simt & SH_STAGE_O) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_O, x, out, st))) return rc;
   } else if (!L->dense) {
-    SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
     TcGemmArgs g{};
     g.d = d; g.K = d.D; g.ncols = d.M;
     g.A = ws + L->o.ahat; g.lda = HD;
@@ -219,7 +275,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     g.b_rows_per_group = d.M; g.out0 = out; g.status = status;
     dim3 grid(d.max_tiles, (d.M + 127) / 128);
     if ((rc = launch_gemm<128, 3, GEMM_O, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
-    L->launches += 2;
+    L->launches += 1;
   } else {
     TcGemmArgs g{};
     g.d = d; g.K = HD; g.ncols = d.M; g.nrows = d.N; g.out0 = out; g.status = status;

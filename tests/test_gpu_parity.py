@@ -19,13 +19,16 @@ def full_check(inp, check_stage_buffers=True, batches=None):
     idx, gate, off, lists = (t.cpu().numpy() for t in layer.sh_gate_topk(x))
     torch.cuda.synchronize()
     N = B * T
+    # fp32 path: fp32 FMA chains.  bf16 path: the logits come from the tensor pipe, whose fp32
+    # accumulation of d_model-term sums is slightly less exact than an FMA chain.
+    gtol = 1e-6 if cfg.dtype == inputs.DTYPE_F32 else 2e-5
     if batches is None:
-        pu.check_selection(idx, gate, ref, N)
+        pu.check_selection(idx, gate, ref, N, gtol)
         pu.check_lists(off, lists, ref)
     else:
         H, k = cfg.n_heads, cfg.k
         tok = np.concatenate([np.arange(b * T, (b + 1) * T) for b in batches])
-        pu.check_selection(idx[:, tok], gate[:, tok], ref, tok.size)
+        pu.check_selection(idx[:, tok], gate[:, tok], ref, tok.size, gtol)
     if check_stage_buffers:
         y2 = layer.sh_forward(x)          # refresh the intermediates after sh_gate_topk
         torch.cuda.synchronize()
