@@ -7,6 +7,7 @@
 #include "sh_tc_gemm.cuh"
 #include "sh_tc_attn.cuh"
 #include "sh_tc_gate.cuh"
+#include "sh_tc_oproj.cuh"
 
 using namespace shtc;
 
@@ -72,7 +73,8 @@ struct TcState {
   CUtensorMap map_q, map_k, map_v;
   CUtensorMap map_wqk, map_wv, map_wo, map_ahat, map_wgate;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
-  int qk_bn, o_bn;
+  int qk_bn, o_bn, qk_variant;
+  int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
 };
 
@@ -100,7 +102,11 @@ int sh_tc_prepare(sh_layer* L) {
   char* ws = L->ws;
   const int HD = d.H * d.D;
   const int nproj = L->dense ? 3 : 2;
-  S->qk_bn = 128;
+  const char* ov = getenv("SH_O_SCATTER");
+  S->o_scatter = ov ? atoi(ov) : 0;
+  const char* qv = getenv("SH_QK_VARIANT");
+  S->qk_variant = qv ? atoi(qv) : 0;
+  S->qk_bn = (S->qk_variant == 2) ? 256 : 128;
   S->o_bn = 128;
   const char* env = getenv("SH_SIMT_STAGES");
   S->simt_mask = env ? atoi(env) : 0;
@@ -157,7 +163,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.offsets = (int*)(ws + L->o.offsets); g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
   g.done_counter = (unsigned int*)(ws + L->o.status + 64);
   g.zero_v = zero_for_forward ? (__half*)(ws + L->o.v) : nullptr;
-  g.zero_out = zero_for_forward ? (float*)out : nullptr;
+  g.zero_out = (zero_for_forward && (S->o_scatter || (S->simt_mask & SH_STAGE_O))) ? (float*)out : nullptr;
   g.status = (int*)(ws + L->o.status);
   const int smem = gate_smem_bytes(S->gate_gp, d.G);
   static int configured = 0;
@@ -219,8 +225,14 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
     g.qscale = 1.4426950408889634f / sqrtf((float)d.D);
     g.status = status;
-    dim3 grid(d.nblk, (g.ncols + 127) / 128);
-    if ((rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st))) return rc;
+    dim3 grid(d.nblk, (g.ncols + S->qk_bn - 1) / S->qk_bn);
+    switch (S->qk_variant) {
+      case 1: rc = launch_gemm<128, 3, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
+      case 2: rc = launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
+      case 3: rc = launch_gemm<128, 6, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
+      default: rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
+    }
+    if (rc) return rc;
     L->launches += 1;
   }
   sh_mark(L, 2, st);
@@ -265,7 +277,8 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   // ---- output experts ----------------------------------------------------------------------------
   if (simt & SH_STAGE_O) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_O, x, out, st))) return rc;
-  } else if (!L->dense) {
+  } else if (!L->dense && S->o_scatter) {
+    // sorted grouped GEMM with a scatter-add epilogue (needs out cleared beforehand)
     TcGemmArgs g{};
     g.d = d; g.K = d.D; g.ncols = d.M;
     g.A = ws + L->o.ahat; g.lda = HD;
@@ -275,6 +288,29 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     g.b_rows_per_group = d.M; g.out0 = out; g.status = status;
     dim3 grid(d.max_tiles, (d.M + 127) / 128);
     if ((rc = launch_gemm<128, 3, GEMM_O, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
+    L->launches += 1;
+  } else if (!L->dense) {
+    TcOprojArgs a{};
+    a.d = d;
+    const size_t side1 = (size_t)d.N * d.H * d.k;
+    a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
+    a.blockcnt = (const int*)(ws + L->o.blockcnt); a.out = (float*)out; a.status = status;
+    const unsigned grid = (unsigned)(d.nblk * (d.M / 128));
+    static int cfg_smem128 = 0, cfg_smem64 = 0;
+    int as = 5, smem = 0;
+    for (; as >= 2; --as) {
+      smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.E, d.k) : OprojSmem<64>::total(as, d.H, d.E, d.k);
+      if (smem <= 227 * 1024) break;
+    }
+    if (as < 2) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
+    a.a_stages = as;
+    if (d.D == 128) {
+      if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
+      sh_tc_oproj_kernel<128><<<grid, 320, smem, st>>>(S->map_ahat, S->map_wo, a);
+    } else {
+      if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
+      sh_tc_oproj_kernel<64><<<grid, 320, smem, st>>>(S->map_ahat, S->map_wo, a);
+    }
     L->launches += 1;
   } else {
     TcGemmArgs g{};

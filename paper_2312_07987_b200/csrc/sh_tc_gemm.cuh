@@ -177,10 +177,16 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
       const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
       const int bb = tok / d.T, tt = tok % d.T;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(trow + c0, v);
+      for (int c00 = 0; c00 < BN; c00 += 64) {
+        // two TMEM loads in flight per wait: the load latency, not its bandwidth, bounds this loop
+        uint32_t vv[64];
+        tmem_ld32(trow + c00, *reinterpret_cast<uint32_t(*)[32]>(&vv[0]));
+        tmem_ld32(trow + c00 + 32, *reinterpret_cast<uint32_t(*)[32]>(&vv[32]));
         tmem_ld_wait();
+#pragma unroll
+        for (int hh2 = 0; hh2 < 2; ++hh2) {
+        const int c0 = c00 + hh2 * 32;
+        uint32_t* v = &vv[hh2 * 32];
         const int n0 = col0 + c0;
         if (!live || n0 >= g.ncols) continue;
         if (MODE == GEMM_QKV) {
@@ -221,6 +227,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
             *reinterpret_cast<float4*>(dst + 4 * i) =
                 make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
                             __uint_as_float(v[4 * i + 3]));
+        }
         }
       }
     }
