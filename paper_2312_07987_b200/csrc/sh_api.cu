@@ -217,12 +217,16 @@ static int launch_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
   sh_gate_topk_kernel<TI><<<d.nblk, 256, hist, st>>>((const TI*)x, (const TI*)(ws + L->o.wgate),
       (const float*)(ws + L->o.gbias), (int*)(ws + L->o.idx), (float*)(ws + L->o.gate),
       (int*)(ws + L->o.blockcnt), d);
-  sh_sort_scan_kernel<<<1, 256, (2 * hist + 16), st>>>((const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.blockoff),
-      (int*)(ws + L->o.offsets), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);
-  sh_sort_scatter_kernel<<<d.nblk, SH_TILE_ROWS, 0, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
-      (const int*)(ws + L->o.blockoff), (const int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
-      (float*)(ws + L->o.lgate), d);
-  L->launches += 3;
+  const size_t ssm = sh_sort_smem_bytes(d);
+  static size_t sort_cfg = 48 * 1024;
+  if (ssm > sort_cfg) {
+    SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+    sort_cfg = ssm;
+  }
+  sh_sort_kernel<<<d.nblk, 256, ssm, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
+      (const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
+      (float*)(ws + L->o.lgate), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);
+  L->launches += 2;
   SH_CUDA_CHECK(cudaGetLastError());
   return SH_OK;
 }

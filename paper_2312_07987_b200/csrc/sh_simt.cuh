@@ -86,99 +86,128 @@ sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const flo
 }
 
 // ---------------------------------------------------------------------------------------
-// Bucket sort, step 1 (one block): exclusive scan of the per-block histograms over blocks,
-// per-head exclusive scan over experts, and the row-tile table of the grouped GEMMs.
+// Bucket sort (one launch).  Block b owns tokens [b*128, b*128+128).  From the per-block
+// selection histograms every block derives, per bucket (side, head, expert): the number of
+// selections in earlier blocks and the bucket total; from the totals the per-head exclusive
+// scan over experts.  It then places its own tokens, in ascending order, behind those of the
+// earlier blocks (a stable counting sort: within a bucket tokens stay ascending).  Block 0
+// also writes the offsets array and the row-tile table of the grouped GEMMs.
+// Dynamic shared memory: 128*H*k*2*8 bytes (the block's idx and gate values, both sides)
+// + (6*G + 8) * 4 bytes.
 // ---------------------------------------------------------------------------------------
 static __global__ void __launch_bounds__(256)
-sh_sort_scan_kernel(const int* __restrict__ blockcnt, int* __restrict__ blockoff, int* __restrict__ offsets,
-                    ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
-  extern __shared__ int s_scan[];            // total[nb], tilebase[nb + 2]
-  const int nb = 2 * d.H * d.E;
-  int* s_total = s_scan;
-  int* s_tbase = s_scan + nb;
-  for (int b = threadIdx.x; b < nb; b += blockDim.x) {
-    int run = 0;
-    for (int blk = 0; blk < d.nblk; ++blk) {
-      int c = blockcnt[(size_t)blk * nb + b];
-      blockoff[(size_t)blk * nb + b] = run;
-      run += c;
+sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, const int* __restrict__ blockcnt,
+               int* __restrict__ offsets, int* __restrict__ lists, float* __restrict__ lgate,
+               ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
+  extern __shared__ int s_sort[];
+  const int nb = d.G;
+  const int per_tok = d.H * d.k;
+  int* s_pre = s_sort;                 // [nb] selections of this bucket in earlier blocks
+  int* s_tot = s_pre + nb;             // [nb] bucket totals
+  int* s_off = s_tot + nb;             // [nb] start of the bucket inside its (side, head) list
+  int* s_tbase = s_off + nb;           // [nb] first tile of the bucket (block 0 only)
+  int* s_wcnt = s_tbase + nb;          // [nb][4] per-warp counts of this block's tokens (warps 0..3)
+  int* s_idx = s_wcnt + 4 * nb;        // [2][128*per_tok]
+  float* s_gt = (float*)(s_idx + 2 * 128 * per_tok);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int blk = blockIdx.x;
+  const int tok0 = blk * SH_TILE_ROWS;
+  const int nrows = min(SH_TILE_ROWS, d.N - tok0);
+  for (int i = tid; i < 2 * nb; i += blockDim.x) s_pre[i] = 0;   // s_pre and s_tot
+  // this block's selections: contiguous per side
+  for (int side = 0; side < 2; ++side) {
+    const size_t base = ((size_t)side * d.N + tok0) * per_tok;
+    for (int i = tid; i < nrows * per_tok; i += blockDim.x) {
+      s_idx[side * 128 * per_tok + i] = idx[base + i];
+      s_gt[side * 128 * per_tok + i] = gate[base + i];
     }
-    s_total[b] = run;
   }
   __syncthreads();
-  for (int g = threadIdx.x; g < 2 * d.H; g += blockDim.x) {
+  for (int i = tid; i < nb * d.nblk; i += blockDim.x) {
+    const int b = i % nb, bk = i / nb;
+    const int c = blockcnt[i];
+    if (c) {
+      atomicAdd(&s_tot[b], c);
+      if (bk < blk) atomicAdd(&s_pre[b], c);
+    }
+  }
+  __syncthreads();
+  for (int g = tid; g < 2 * d.H; g += blockDim.x) {
     int run = 0;
     for (int e = 0; e < d.E; ++e) {
-      offsets[g * (d.E + 1) + e] = run;
-      run += s_total[g * d.E + e];
+      s_off[g * d.E + e] = run;
+      run += s_tot[g * d.E + e];
     }
-    offsets[g * (d.E + 1) + d.E] = run;
   }
-  if (threadIdx.x < 2) {                     // tile bases per side
-    const int side = threadIdx.x;
+  // per-warp counts of this block's tokens, thread = token (warps 0..3)
+  if (tid < SH_TILE_ROWS) {
+    for (int grp = 0; grp < 2 * d.H; ++grp) {
+      const int side = grp / d.H, h = grp % d.H;
+      unsigned mask = 0;
+      if (tid < nrows)
+        for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[side * 128 * per_tok + (tid * d.H + h) * d.k + j];
+      for (int e = 0; e < d.E; ++e) {
+        const unsigned bal = __ballot_sync(0xffffffffu, (mask >> e) & 1u);
+        if (lane == 0) s_wcnt[(grp * d.E + e) * 4 + warp] = __popc(bal);
+      }
+    }
+  }
+  __syncthreads();
+  if (tid < SH_TILE_ROWS) {
+    const int t = tok0 + tid;
+    for (int grp = 0; grp < 2 * d.H; ++grp) {
+      const int side = grp / d.H, h = grp % d.H;
+      const int sel = side * 128 * per_tok + (tid * d.H + h) * d.k;
+      unsigned mask = 0;
+      if (tid < nrows)
+        for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[sel + j];
+      for (int e = 0; e < d.E; ++e) {
+        const bool mine = (mask >> e) & 1u;
+        const unsigned bal = __ballot_sync(0xffffffffu, mine);
+        if (mine) {
+          const int b = grp * d.E + e;
+          int pos = __popc(bal & ((1u << lane) - 1u));
+          for (int w = 0; w < warp; ++w) pos += s_wcnt[b * 4 + w];
+          float gv = 0.f;
+          for (int j = 0; j < d.k; ++j)
+            if (s_idx[sel + j] == e) gv = s_gt[sel + j];
+          const size_t dst = (size_t)grp * d.N * d.k + s_off[b] + s_pre[b] + pos;
+          lists[dst] = t;
+          lgate[dst] = gv;
+        }
+      }
+    }
+  }
+  if (blk != 0) return;
+  for (int g = tid; g < 2 * d.H; g += blockDim.x) {
+    for (int e = 0; e < d.E; ++e) offsets[g * (d.E + 1) + e] = s_off[g * d.E + e];
+    offsets[g * (d.E + 1) + d.E] = s_off[g * d.E + d.E - 1] + s_tot[g * d.E + d.E - 1];
+  }
+  if (tid < 2) {
+    const int side = tid;
     int run = 0;
     for (int b = side * d.H * d.E; b < (side + 1) * d.H * d.E; ++b) {
       s_tbase[b] = run;
-      run += (s_total[b] + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
+      run += (s_tot[b] + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
     }
     ntiles[side] = run;
   }
   __syncthreads();
-  for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+  for (int b = tid; b < nb; b += blockDim.x) {
     const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
-    int start = 0;
-    for (int e2 = 0; e2 < e; ++e2) start += s_total[b - e + e2];
-    const int cnt = s_total[b];
+    const int cnt = s_tot[b];
     ShTile* tp = tiles + (size_t)side * d.max_tiles + s_tbase[b];
     for (int r = 0, i = 0; r < cnt; r += SH_TILE_ROWS, ++i) {
       ShTile tl;
-      tl.h = h; tl.e = e; tl.row0 = start + r;
+      tl.h = h; tl.e = e; tl.row0 = s_off[b] + r;
       tl.nrows = min(SH_TILE_ROWS, cnt - r);
       tp[i] = tl;
     }
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// Bucket sort, step 2: stable scatter.  Block b owns tokens [b*128, b*128+128); thread =
-// token.  Within a bucket tokens stay in ascending order.
-// ---------------------------------------------------------------------------------------
-static __global__ void __launch_bounds__(SH_TILE_ROWS)
-sh_sort_scatter_kernel(const int* __restrict__ idx, const float* __restrict__ gate,
-                       const int* __restrict__ blockoff, const int* __restrict__ offsets,
-                       int* __restrict__ lists, float* __restrict__ lgate, ShDims d) {
-  __shared__ int s_wcnt[SH_TILE_ROWS / 32][32];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x * SH_TILE_ROWS + threadIdx.x;
-  const int nb = 2 * d.H * d.E;
-  const bool live = t < d.N;
-  for (int grp = 0; grp < 2 * d.H; ++grp) {
-    const int side = grp / d.H, h = grp % d.H;
-    const size_t sel = (((size_t)side * d.N + t) * d.H + h) * d.k;
-    unsigned mask = 0;
-    if (live)
-      for (int j = 0; j < d.k; ++j) mask |= 1u << idx[sel + j];
-    __syncthreads();                         // s_wcnt free again
-    for (int e = 0; e < d.E; ++e) {
-      unsigned bal = __ballot_sync(0xffffffffu, (mask >> e) & 1u);
-      if (lane == 0) s_wcnt[warp][e] = __popc(bal);
-    }
-    __syncthreads();
-    for (int e = 0; e < d.E; ++e) {
-      const bool mine = (mask >> e) & 1u;
-      const unsigned bal = __ballot_sync(0xffffffffu, mine);
-      if (mine) {
-        int pos = __popc(bal & ((1u << lane) - 1u));
-        for (int w = 0; w < warp; ++w) pos += s_wcnt[w][e];
-        float g = 0.f;
-        for (int j = 0; j < d.k; ++j)
-          if (idx[sel + j] == e) g = gate[sel + j];
-        const int dst = offsets[grp * (d.E + 1) + e] + blockoff[(size_t)blockIdx.x * nb + grp * d.E + e] + pos;
-        lists[(size_t)grp * d.N * d.k + dst] = t;
-        lgate[(size_t)grp * d.N * d.k + dst] = g;
-      }
-    }
-  }
+static inline size_t sh_sort_smem_bytes(const ShDims& d) {
+  return (size_t)(8 * d.G + 8) * 4 + (size_t)2 * 128 * d.H * d.k * 8;
 }
 
 // ---------------------------------------------------------------------------------------

@@ -159,9 +159,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   TcGateArgs g{};
   g.d = d; g.Gp = S->gate_gp; g.gbias = (const float*)(ws + L->o.gbias);
   g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
-  g.blockcnt = (int*)(ws + L->o.blockcnt); g.blockoff = (int*)(ws + L->o.blockoff);
-  g.offsets = (int*)(ws + L->o.offsets); g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
-  g.done_counter = (unsigned int*)(ws + L->o.status + 64);
+  g.blockcnt = (int*)(ws + L->o.blockcnt);
   g.zero_v = zero_for_forward ? (__half*)(ws + L->o.v) : nullptr;
   g.zero_out = (zero_for_forward && (S->o_scatter || (S->simt_mask & SH_STAGE_O))) ? (float*)out : nullptr;
   g.status = (int*)(ws + L->o.status);
@@ -172,9 +170,15 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
     configured = smem;
   }
   sh_tc_gate_kernel<GATE_STAGES><<<d.nblk, 192, smem, st>>>(map_x, S->map_wgate, g);
-  sh_sort_scatter_kernel<<<d.nblk, SH_TILE_ROWS, 0, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
-      (const int*)(ws + L->o.blockoff), (const int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
-      (float*)(ws + L->o.lgate), d);
+  const size_t ssm = sh_sort_smem_bytes(d);
+  static size_t sort_cfg = 48 * 1024;
+  if (ssm > sort_cfg) {
+    SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+    sort_cfg = ssm;
+  }
+  sh_sort_kernel<<<d.nblk, 256, ssm, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
+      (const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
+      (float*)(ws + L->o.lgate), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);
   L->launches += 2;
   return SH_OK;
 }

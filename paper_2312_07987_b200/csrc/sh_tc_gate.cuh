@@ -4,8 +4,7 @@
 // (side, head) group (strictly-greater scan, so the lower index wins ties), applies the
 // sigmoid, writes idx / gate and adds to the CTA's selection histogram.  While the main loop
 // runs, the otherwise idle epilogue warps clear the V and out rows of the CTA's tokens (both
-// are accumulated into later).  The last CTA to finish turns the per-CTA histograms into
-// block offsets, per-head expert offsets and the row-tile table of the grouped GEMMs.
+// are accumulated into later).
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
 // warps 2..5 = zero-fill, then selection epilogue.
@@ -19,8 +18,7 @@ struct TcGateArgs {
   int Gp;                    // G rounded up to a multiple of 16 (UMMA N)
   const float* gbias;        // [G]
   int* idx; float* gate;     // [2, N, H, k]
-  int* blockcnt; int* blockoff; int* offsets; ShTile* tiles; int* ntiles;
-  unsigned int* done_counter;
+  int* blockcnt;             // [nblk, G] per-CTA selection histogram
   __half* zero_v;            // [B, H, T, D] or nullptr
   float* zero_out;           // [N, M] or nullptr
   int* status;
@@ -42,10 +40,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* tmem_full = empty_bar + STAGES;
   uint32_t* tmem_slot = (uint32_t*)(tmem_full + 1);
-  int* s_flag = (int*)(tmem_slot + 1);
   int* s_hist = (int*)(sgen + bar_off + 256);           // [G]
-  int* s_total = s_hist + d.G;                          // [G]   (last CTA only)
-  int* s_tbase = s_total + d.G;                         // [G]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row0 = blockIdx.x * 128;
@@ -104,15 +99,14 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       for (long i = et; i < total; i += 128) base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (g.zero_v) {
-      const int c16 = d.D / 8;                          // 16-byte chunks per (token, head) row
-      const long total = (long)nrows * d.H * c16;
-      for (long i = et; i < total; i += 128) {
-        const int ch = (int)(i % c16);
-        const long th = i / c16;
-        const int hh = (int)(th % d.H);
-        const int tok = row0 + (int)(th / d.H);
+      const int sh = d.D == 128 ? 4 : 3;                // 16-byte chunks per (token, head) row: D / 8
+      const int ch = et & ((1 << sh) - 1);
+      for (int tl = et >> sh; tl < nrows; tl += 128 >> sh) {
+        const int tok = row0 + tl;
         const int bb = tok / d.T, tt = tok % d.T;
-        *reinterpret_cast<uint4*>(g.zero_v + (((size_t)bb * d.H + hh) * d.T + tt) * d.D + ch * 8) = make_uint4(0, 0, 0, 0);
+        __half* p = g.zero_v + ((size_t)bb * d.H * d.T + tt) * d.D + ch * 8;
+        for (int hh = 0; hh < d.H; ++hh)
+          *reinterpret_cast<uint4*>(p + (size_t)hh * d.T * d.D) = make_uint4(0, 0, 0, 0);
       }
     }
     // ---- selection epilogue: thread = token = TMEM lane ---------------------------------------
@@ -122,17 +116,25 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     if (mbar_wait(tmem_full, 0, g.status, dead)) {
       tc_fence_after();
       const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
-      for (int c0 = 0; c0 < Gp; c0 += 16) {             // logits row -> shared memory (pipeline buffers are idle now)
-        uint32_t v[16];
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-            : "r"(trow + c0)
-            : "memory");
+      // logits row -> shared memory (the pipeline buffers are idle now); up to four TMEM loads
+      // are issued per wait because the load latency, not its bandwidth, bounds this loop
+      for (int c0 = 0; c0 < Gp; c0 += 64) {
+        uint32_t v[64];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (c0 + 16 * u < Gp) {
+            uint32_t* w = &v[16 * u];
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]),
+                  "=r"(w[8]), "=r"(w[9]), "=r"(w[10]), "=r"(w[11]), "=r"(w[12]), "=r"(w[13]), "=r"(w[14]), "=r"(w[15])
+                : "r"(trow + c0 + 16 * u)
+                : "memory");
+          }
+        }
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 64; ++i)
           if (c0 + i < d.G) srow[c0 + i] = __uint_as_float(v[i]) + g.gbias[c0 + i];
       }
       const int t = row0 + r;
@@ -165,67 +167,8 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     tc_fence_after();
     tmem_dealloc(tmem_d, tmem_cols);
   }
-  // ---- publish the histogram; the last CTA builds offsets and the tile table -----------------
-  const int nb = d.G;
-  for (int i = threadIdx.x; i < nb; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * nb + i] = s_hist[i];
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const unsigned prev = atomicAdd(g.done_counter, 1u);
-    *s_flag = (prev == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!*s_flag) return;
-  __threadfence();
-  // warp per bucket: exclusive scan over the CTAs' counts
-  for (int b = warp; b < nb; b += 6) {
-    int run = 0;
-    for (int blk0 = 0; blk0 < d.nblk; blk0 += 32) {
-      const int blk = blk0 + lane;
-      const int c = blk < d.nblk ? __ldcg(&g.blockcnt[(size_t)blk * nb + b]) : 0;
-      int inc = c;
-#pragma unroll
-      for (int s = 1; s < 32; s <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, inc, s);
-        if (lane >= s) inc += n;
-      }
-      if (blk < d.nblk) g.blockoff[(size_t)blk * nb + b] = run + inc - c;
-      run += __shfl_sync(0xffffffffu, inc, 31);
-    }
-    if (lane == 0) s_total[b] = run;
-  }
-  __syncthreads();
-  for (int grp = threadIdx.x; grp < 2 * d.H; grp += blockDim.x) {
-    int run = 0;
-    for (int e = 0; e < d.E; ++e) {
-      g.offsets[grp * (d.E + 1) + e] = run;
-      run += s_total[grp * d.E + e];
-    }
-    g.offsets[grp * (d.E + 1) + d.E] = run;
-  }
-  if (threadIdx.x < 2) {
-    const int side = threadIdx.x;
-    int run = 0;
-    for (int b = side * d.H * d.E; b < (side + 1) * d.H * d.E; ++b) {
-      s_tbase[b] = run;
-      run += (s_total[b] + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
-    }
-    g.ntiles[side] = run;
-  }
-  __syncthreads();
-  for (int b = threadIdx.x; b < nb; b += blockDim.x) {
-    const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
-    int start = 0;
-    for (int e2 = 0; e2 < e; ++e2) start += s_total[b - e + e2];
-    const int cnt = s_total[b];
-    ShTile* tp = g.tiles + (size_t)side * d.max_tiles + s_tbase[b];
-    for (int rr = 0, i = 0; rr < cnt; rr += SH_TILE_ROWS, ++i) {
-      ShTile tl;
-      tl.h = h; tl.e = e; tl.row0 = start + rr; tl.nrows = min(SH_TILE_ROWS, cnt - rr);
-      tp[i] = tl;
-    }
-  }
-  if (threadIdx.x == 0) *g.done_counter = 0;            // ready for the next forward pass
+  // ---- publish this CTA's selection histogram (the sort kernel scans them) ------------------
+  for (int i = threadIdx.x; i < d.G; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
 }
 
 }  // namespace shtc
