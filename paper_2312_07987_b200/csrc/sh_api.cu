@@ -223,7 +223,7 @@ static int launch_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
     SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
     sort_cfg = ssm;
   }
-  sh_sort_kernel<<<d.nblk, 256, ssm, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
+  sh_sort_kernel<<<d.nblk, sh_sort_threads(d), ssm, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
       (const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
       (float*)(ws + L->o.lgate), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);
   L->launches += 2;

@@ -95,7 +95,9 @@ sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const flo
 // Dynamic shared memory: 128*H*k*2*8 bytes (the block's idx and gate values, both sides)
 // + (6*G + 8) * 4 bytes.
 // ---------------------------------------------------------------------------------------
-static __global__ void __launch_bounds__(256)
+// Threads: 128 * GS, thread = (token tid % 128, group slice tid / 128); slice gs handles the
+// (side, head) groups gs, gs + GS, ...
+static __global__ void __launch_bounds__(1024)
 sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, const int* __restrict__ blockcnt,
                int* __restrict__ offsets, int* __restrict__ lists, float* __restrict__ lgate,
                ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
@@ -106,16 +108,17 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
   int* s_tot = s_pre + nb;             // [nb] bucket totals
   int* s_off = s_tot + nb;             // [nb] start of the bucket inside its (side, head) list
   int* s_tbase = s_off + nb;           // [nb] first tile of the bucket (block 0 only)
-  int* s_wcnt = s_tbase + nb;          // [nb][4] per-warp counts of this block's tokens (warps 0..3)
+  int* s_wcnt = s_tbase + nb;          // [nb][4] per-warp counts of this block's tokens
   int* s_idx = s_wcnt + 4 * nb;        // [2][128*per_tok]
   float* s_gt = (float*)(s_idx + 2 * 128 * per_tok);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int tl = tid & 127, gs = tid >> 7, GS = blockDim.x >> 7;
+  const int twarp = tl >> 5;           // warp index among the 4 warps of a slice
   const int blk = blockIdx.x;
   const int tok0 = blk * SH_TILE_ROWS;
   const int nrows = min(SH_TILE_ROWS, d.N - tok0);
   for (int i = tid; i < 2 * nb; i += blockDim.x) s_pre[i] = 0;   // s_pre and s_tot
-  // this block's selections: contiguous per side
-  for (int side = 0; side < 2; ++side) {
+  for (int side = 0; side < 2; ++side) {                          // this block's selections
     const size_t base = ((size_t)side * d.N + tok0) * per_tok;
     for (int i = tid; i < nrows * per_tok; i += blockDim.x) {
       s_idx[side * 128 * per_tok + i] = idx[base + i];
@@ -123,12 +126,20 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     }
   }
   __syncthreads();
-  for (int i = tid; i < nb * d.nblk; i += blockDim.x) {
-    const int b = i % nb, bk = i / nb;
-    const int c = blockcnt[i];
-    if (c) {
-      atomicAdd(&s_tot[b], c);
-      if (bk < blk) atomicAdd(&s_pre[b], c);
+  {
+    // bucket b = tid % nb; the thread sums the blocks part, part + parts, ... in registers
+    const int parts = max(1, (int)blockDim.x / nb);
+    for (int b = tid % nb + (tid / nb / parts) * nb; b < nb; b += blockDim.x) {  // executes once unless nb > blockDim
+      const int part = (tid / nb) % parts;
+      int tot = 0, pre = 0;
+#pragma unroll 4
+      for (int bk = part; bk < d.nblk; bk += parts) {
+        const int c = blockcnt[(size_t)bk * nb + b];
+        tot += c;
+        pre += bk < blk ? c : 0;
+      }
+      if (tot) atomicAdd(&s_tot[b], tot);
+      if (pre) atomicAdd(&s_pre[b], pre);
     }
   }
   __syncthreads();
@@ -139,27 +150,24 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
       run += s_tot[g * d.E + e];
     }
   }
-  // per-warp counts of this block's tokens, thread = token (warps 0..3)
-  if (tid < SH_TILE_ROWS) {
-    for (int grp = 0; grp < 2 * d.H; ++grp) {
-      const int side = grp / d.H, h = grp % d.H;
-      unsigned mask = 0;
-      if (tid < nrows)
-        for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[side * 128 * per_tok + (tid * d.H + h) * d.k + j];
-      for (int e = 0; e < d.E; ++e) {
-        const unsigned bal = __ballot_sync(0xffffffffu, (mask >> e) & 1u);
-        if (lane == 0) s_wcnt[(grp * d.E + e) * 4 + warp] = __popc(bal);
-      }
+  for (int grp = gs; grp < 2 * d.H; grp += GS) {                  // per-warp counts of this block's tokens
+    const int side = grp / d.H, h = grp % d.H;
+    unsigned mask = 0;
+    if (tl < nrows)
+      for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[side * 128 * per_tok + (tl * d.H + h) * d.k + j];
+    for (int e = 0; e < d.E; ++e) {
+      const unsigned bal = __ballot_sync(0xffffffffu, (mask >> e) & 1u);
+      if (lane == 0) s_wcnt[(grp * d.E + e) * 4 + twarp] = __popc(bal);
     }
   }
   __syncthreads();
-  if (tid < SH_TILE_ROWS) {
-    const int t = tok0 + tid;
-    for (int grp = 0; grp < 2 * d.H; ++grp) {
+  {
+    const int t = tok0 + tl;
+    for (int grp = gs; grp < 2 * d.H; grp += GS) {
       const int side = grp / d.H, h = grp % d.H;
-      const int sel = side * 128 * per_tok + (tid * d.H + h) * d.k;
+      const int sel = side * 128 * per_tok + (tl * d.H + h) * d.k;
       unsigned mask = 0;
-      if (tid < nrows)
+      if (tl < nrows)
         for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[sel + j];
       for (int e = 0; e < d.E; ++e) {
         const bool mine = (mask >> e) & 1u;
@@ -167,7 +175,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
         if (mine) {
           const int b = grp * d.E + e;
           int pos = __popc(bal & ((1u << lane) - 1u));
-          for (int w = 0; w < warp; ++w) pos += s_wcnt[b * 4 + w];
+          for (int w = 0; w < twarp; ++w) pos += s_wcnt[b * 4 + w];
           float gv = 0.f;
           for (int j = 0; j < d.k; ++j)
             if (s_idx[sel + j] == e) gv = s_gt[sel + j];
@@ -193,17 +201,24 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     ntiles[side] = run;
   }
   __syncthreads();
-  for (int b = tid; b < nb; b += blockDim.x) {
+  for (int i = tid; i < nb * 32; i += blockDim.x) {               // 32 threads share a bucket's tiles
+    const int b = i >> 5;
     const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
     const int cnt = s_tot[b];
     ShTile* tp = tiles + (size_t)side * d.max_tiles + s_tbase[b];
-    for (int r = 0, i = 0; r < cnt; r += SH_TILE_ROWS, ++i) {
-      ShTile tl;
-      tl.h = h; tl.e = e; tl.row0 = s_off[b] + r;
-      tl.nrows = min(SH_TILE_ROWS, cnt - r);
-      tp[i] = tl;
+    for (int ti = i & 31; ti * SH_TILE_ROWS < cnt; ti += 32) {
+      ShTile tl2;
+      tl2.h = h; tl2.e = e; tl2.row0 = s_off[b] + ti * SH_TILE_ROWS;
+      tl2.nrows = min(SH_TILE_ROWS, cnt - ti * SH_TILE_ROWS);
+      tp[ti] = tl2;
     }
   }
+}
+
+static inline int sh_sort_threads(const ShDims& d) {
+  int gs = 2 * d.H;
+  if (gs > 8) gs = 8;
+  return 128 * gs;
 }
 
 static inline size_t sh_sort_smem_bytes(const ShDims& d) {
