@@ -27,7 +27,7 @@ EXPORTS = ["sh_create", "sh_create_dense", "sh_configure", "sh_workspace_bytes",
 
 
 def _load() -> ctypes.CDLL:
-    path = _build.LIB_PATH
+    path = os.environ.get("SWITCHHEAD_LIB") or _build.LIB_PATH     # a custom build of the library
     if not os.path.exists(path):
         path = _build.build()
     lib = ctypes.CDLL(path)

@@ -129,14 +129,15 @@ sh_tc_attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc_f16(128, 128, 0, 0, 0);
       constexpr uint32_t idesc_pv = make_idesc_f16(128, D, 0, 0, 1);
+      const uint32_t q_lo = desc_lo_k(sbase + SM::Q_OFF), k_lo0 = desc_lo_k(sbase + SM::K_OFF);
+      const uint32_t p_lo = desc_lo_k(sbase + SM::P_OFF), v_lo0 = desc_lo_mn(sbase + SM::V_OFF, BLK);
       auto issue_s = [&](int j) {
         const int s = j & 1;
-        const uint32_t qa = sbase + SM::Q_OFF, ka = sbase + SM::K_OFF + s * SM::KV_BYTES;
+        const uint32_t k_lo = k_lo0 + s * (SM::KV_BYTES >> 4);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint64_t ad = make_desc_k_sw128(qa + (k / 4) * BLK) + 2 * (k % 4);
-          const uint64_t bd = make_desc_k_sw128(ka + (k / 4) * BLK) + 2 * (k % 4);
-          umma_f16(tmem + s * 128, ad, bd, idesc_s, k != 0);
+          const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+          umma_f16(tmem + s * 128, desc_pack(q_lo + koff), desc_pack(k_lo + koff), idesc_s, k != 0);
         }
         umma_commit(&k_empty[s]);
         umma_commit(&s_full[s]);
@@ -158,12 +159,11 @@ sh_tc_attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
         if (!mbar_wait(&v_full[s], (j >> 1) & 1, g.status, dead)) break;
         if (!mbar_wait(p_full, j & 1, g.status, dead)) break;
         tc_fence_after();
-        const uint32_t pa = sbase + SM::P_OFF, va = sbase + SM::V_OFF + s * SM::KV_BYTES;
+        const uint32_t v_lo = v_lo0 + s * (SM::KV_BYTES >> 4);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {                       // 128 keys in steps of 16
-          const uint64_t ad = make_desc_k_sw128(pa + (k / 4) * BLK) + 2 * (k % 4);
-          const uint64_t bd = make_desc_mn_sw128(va + k * 2048, BLK);
-          umma_f16(tmem_o, ad, bd, idesc_pv, (j | k) != 0);
+          const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+          umma_f16(tmem_o, desc_pack(p_lo + koff), desc_pack(v_lo + k * (2048 >> 4)), idesc_pv, (j | k) != 0);
         }
         umma_commit(&v_empty[s]);
         umma_commit(pv_done);

@@ -105,16 +105,18 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_f16(GEMM_BM, BN, A_BF16, B_BF16, 0);
+      const uint32_t a_lo0 = desc_lo_k(sbase), b_lo0 = desc_lo_k(sbase + SM::A_BYTES);
+      int s = 0;
+      uint32_t par = 0;
       for (int kb = 0; kb < KB; ++kb) {
-        const int s = kb % STAGES;
-        if (!mbar_wait(&full_bar[s], (kb / STAGES) & 1, g.status, dead)) break;
+        if (!mbar_wait(&full_bar[s], par, g.status, dead)) break;
         tc_fence_after();
-        const uint32_t sa = sbase + s * SM::STAGE_BYTES, sb = sa + SM::A_BYTES;
-        const uint64_t adesc = make_desc_k_sw128(sa), bdesc = make_desc_k_sw128(sb);
+        const uint32_t a_lo = a_lo0 + s * (SM::STAGE_BYTES >> 4), b_lo = b_lo0 + s * (SM::STAGE_BYTES >> 4);
 #pragma unroll
         for (int k = 0; k < GEMM_BK / 16; ++k)
-          umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+          umma_f16(tmem_d, desc_pack(a_lo + 2 * k), desc_pack(b_lo + 2 * k), idesc, (kb | k) != 0);
         umma_commit(&empty_bar[s]);
+        if (++s == STAGES) { s = 0; par ^= 1; }
       }
       umma_commit(tmem_full);
     }

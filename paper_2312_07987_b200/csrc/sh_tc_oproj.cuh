@@ -100,7 +100,8 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
 
   if (warp == 0) {
     if (lane == 0) {
-      int it = 0;
+      int s = 0;
+      uint32_t e_par = 1;                                   // parity of a_empty[s] for the current ring pass
       for (int h = 0; h < d.H; ++h) {
         const int bs = h & 1;
         if (!mbar_wait(&b_empty[bs], ((h >> 1) & 1) ^ 1, g.status, dead)) break;
@@ -110,14 +111,13 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
           tma_load_2d(sbase + b_off + bs * SM::B_BYTES + c * BLK, &mapAhat, &b_full[bs], h * D + c * 64, row0);
         for (int e = 0; e < d.E && !dead; ++e) {
           if (s_cnt[h * d.E + e] == 0) continue;
-          const int s = it % AS;
-          if (!mbar_wait(&a_empty[s], ((it / AS) & 1) ^ 1, g.status, dead)) break;
+          if (!mbar_wait(&a_empty[s], e_par, g.status, dead)) break;
           mbar_expect_tx(&a_full[s], SM::A_BYTES);
 #pragma unroll
           for (int c = 0; c < DB; ++c)
             tma_load_2d(sbase + a_off + s * SM::A_BYTES + c * BLK, &mapWo, &a_full[s], c * 64,
                         (h * d.E + e) * d.M + fc * 128);
-          ++it;
+          if (++s == AS) { s = 0; e_par ^= 1; }
         }
         if (dead) break;
       }
@@ -125,26 +125,30 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_f16(128, 128, 0, 0, 0);
-      int it = 0;
+      const uint32_t a_lo0 = desc_lo_k(sbase + a_off), b_lo0 = desc_lo_k(sbase + b_off);
+      int it = 0, s = 0;
+      uint32_t a_par = 0;                                   // parity of a_full[s] for the current ring pass
       for (int h = 0; h < d.H && !dead; ++h) {
         const int bs = h & 1;
         if (!mbar_wait(&b_full[bs], (h >> 1) & 1, g.status, dead)) break;
+        const uint32_t b_lo = b_lo0 + bs * (SM::B_BYTES >> 4);
         for (int e = 0; e < d.E; ++e) {
           if (s_cnt[h * d.E + e] == 0) continue;
-          const int s = it % AS, buf = it & 3;
-          if (!mbar_wait(&a_full[s], (it / AS) & 1, g.status, dead)) break;
+          const int buf = it & 3;
+          if (!mbar_wait(&a_full[s], a_par, g.status, dead)) break;
           if (!mbar_wait(&d_empty[buf], ((it >> 2) & 1) ^ 1, g.status, dead)) break;
           tc_fence_after();
-          const uint32_t wa = sbase + a_off + s * SM::A_BYTES, ta = sbase + b_off + bs * SM::B_BYTES;
+          const uint32_t a_lo = a_lo0 + s * (SM::A_BYTES >> 4);
+          const uint32_t td = tmem + buf * 128;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
-            const uint64_t ad = make_desc_k_sw128(wa + (k / 4) * BLK) + 2 * (k % 4);
-            const uint64_t bd = make_desc_k_sw128(ta + (k / 4) * BLK) + 2 * (k % 4);
-            umma_f16(tmem + buf * 128, ad, bd, idesc, k != 0);
+            const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+            umma_f16(td, desc_pack(a_lo + koff), desc_pack(b_lo + koff), idesc, k != 0);
           }
           umma_commit(&a_empty[s]);
           umma_commit(&d_full[buf]);
           ++it;
+          if (++s == AS) { s = 0; a_par ^= 1; }
         }
         umma_commit(&b_empty[bs]);
       }

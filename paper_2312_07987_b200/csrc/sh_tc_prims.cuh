@@ -156,6 +156,16 @@ __device__ __forceinline__ uint64_t make_desc_mn_sw128(uint32_t saddr, uint32_t 
   d |= (uint64_t)2 << 61;
   return d;
 }
+// The UMMA-issuing thread is a single thread on the critical path, so descriptors are kept as
+// a constant high word plus a 32-bit low word that only needs integer adds: +2 per 16-element
+// K step inside a 128-byte row, +(bytes >> 4) to move to another tile or 64-element block.
+constexpr uint32_t DESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128B swizzle
+__device__ __forceinline__ uint32_t desc_lo_k(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mn(uint32_t saddr, uint32_t mn_chunk_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | (((mn_chunk_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t desc_pack(uint32_t lo) { return ((uint64_t)DESC_HI_SW128 << 32) | lo; }
+
 // Instruction descriptor of kind::f16: fp32 accumulator; a_bf16 / b_bf16 choose bf16 (1) or
 // fp16 (0) operands; b_mn_major = 1 when B is stored MN-major.
 __host__ __device__ constexpr uint32_t make_idesc_f16(int m, int n, int a_bf16, int b_bf16, int b_mn_major) {
