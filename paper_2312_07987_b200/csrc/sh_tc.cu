@@ -298,22 +298,28 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     a.d = d;
     const size_t side1 = (size_t)d.N * d.H * d.k;
     a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
-    a.blockcnt = (const int*)(ws + L->o.blockcnt); a.out = (float*)out; a.status = status;
-    const unsigned grid = (unsigned)(d.nblk * (d.M / 128));
+    a.out = (float*)out; a.status = status;
+    a.nwork = d.nblk * (d.M / 128);
+    if (L->sm_count == 0) {
+      int dev = 0;
+      SH_CUDA_CHECK(cudaGetDevice(&dev));
+      SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
     static int cfg_smem128 = 0, cfg_smem64 = 0;
-    int as = 5, smem = 0;
-    for (; as >= 2; --as) {
-      smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.E, d.k) : OprojSmem<64>::total(as, d.H, d.E, d.k);
+    int as = 2, smem = 0;
+    for (; as >= 1; --as) {
+      smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.k) : OprojSmem<64>::total(as, d.H, d.k);
       if (smem <= 227 * 1024) break;
     }
-    if (as < 2) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
+    if (as < 1) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
     a.a_stages = as;
     if (d.D == 128) {
       if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
-      sh_tc_oproj_kernel<128><<<grid, 320, smem, st>>>(S->map_ahat, S->map_wo, a);
+      sh_tc_oproj_kernel<128><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo, a);
     } else {
       if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
-      sh_tc_oproj_kernel<64><<<grid, 320, smem, st>>>(S->map_ahat, S->map_wo, a);
+      sh_tc_oproj_kernel<64><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo, a);
     }
     L->launches += 1;
   } else {

@@ -1,20 +1,26 @@
 // Output-expert projection with the gate-weighted sum kept on chip (the MoE output equation
 // of Sec. 2.2):  y[t] = sum_h sum_{e in E_D^h(t)} s_D^h[t,e] * Ahat^h[t] W_O^{h,e}.
 //
-// One CTA owns 128 consecutive tokens and 128 output features.  For every head h the tokens'
-// Ahat^h rows are one TMA tile (token order, no gather); for every expert e that at least one
-// token of the tile selected, one UMMA chain computes Z = W_O^{h,e}[features, :] Ahat^h[tokens, :]^T
-// (features on the TMEM lanes, tokens on the columns).  Each epilogue thread owns one feature
-// and keeps y[token, feature] for all 128 tokens in registers:  acc[t] += g_e[t] * Z[feature, t],
-// where g_e[t] is the destination gate of expert e for token t, or 0 if t did not select e.
-// The sum over experts and heads therefore never leaves the SM, out is written exactly once
-// (no atomics, no clearing, run-to-run deterministic).  The price is that unselected tokens
-// ride along in the UMMA (E/k times the useful FLOP of this stage).
+// Work unit = 128 consecutive tokens x 128 output features; a persistent CTA (one per SM)
+// walks work units blockIdx.x, blockIdx.x + gridDim.x, ...  For every head h the tokens'
+// Ahat^h rows are one TMA tile (token order, no gather); for every expert e one UMMA chain
+// computes Z = Ahat^h[tokens, :] W_O^{h,e}[:, features] (tokens on the TMEM lanes, features
+// on the columns).  Each epilogue thread owns one token and 64 of the features and keeps
+// y[token, feature] in registers:  acc[f] += g * Z[token, f], where g is the token's
+// destination gate for expert e, or 0 if it did not select e - a per-thread scalar, so the
+// epilogue is pure FFMA.  The sum over experts and heads therefore never leaves the SM and
+// out is written exactly once (no atomics, no clearing, run-to-run deterministic).  The price
+// is that unselected tokens ride along in the UMMA (E/k times the useful FLOP of this stage).
 //
-// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
-// warps 2..9 = epilogue (thread = one feature = TMEM lane, and one half of the tile's tokens;
-// two warps share a lane quarter so that twice as many TMEM loads are in flight).
-// TMEM: four 128-column buffers.
+// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer for the
+// even pipeline items, warp 10 = UMMA issuer for the odd items (two issuing threads, each
+// owning one TMEM buffer, so that one thread's barrier round trips hide behind the other's
+// UMMAs), warps 2..9 = epilogue (thread = one token = TMEM lane, and one half of the 128
+// features; two warps share a lane quarter).
+// Two experts of a head form one pipeline item (one weight stage of two tiles, one 256-column
+// TMEM buffer), so that every barrier round trip of the single UMMA-issuing thread is backed
+// by 1024 tensor-pipe cycles of work.  All rings run on across work units, so the producer
+// and the UMMA issuer work ahead into the next unit while the epilogue stores the last one.
 #pragma once
 #include "sh_tc_prims.cuh"
 
@@ -24,75 +30,63 @@ struct TcOprojArgs {
   ShDims d;
   const int* idx;        // destination side: [N, H, k]
   const float* gate;     // destination side: [N, H, k]
-  const int* blockcnt;   // [nblk, G] per-tile selection counts (bucket = (side*H + h)*E + e)
   float* out;            // [N, M]
-  int a_stages;
+  int a_stages;          // stages of TWO weight tiles
+  int nwork;             // nblk * (M / 128)
   int* status;
 };
 
 template <int D>
 struct OprojSmem {
-  static constexpr int A_BYTES = 128 * D * 2;            // weights tile: 128 features x D
+  static constexpr int A_BYTES = 128 * D * 2;            // one weight tile: 128 features x D
   static constexpr int B_BYTES = 128 * D * 2;            // Ahat tile: 128 tokens x D
-  static int total(int a_stages, int H, int E, int k) {
-    return a_stages * A_BYTES + 2 * B_BYTES + 128 * H * k * 8 + E * 128 * 4 + H * E * 4 + 512 + 1024;
+  static int total(int a_stages, int H, int k) {
+    return a_stages * 2 * A_BYTES + 2 * B_BYTES + 128 * H * k * 8 + 512 + 1024;
   }
 };
 
 template <int D>
-__global__ void __launch_bounds__(320)
+__global__ void __launch_bounds__(352, 1)
 sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g) {
   using SM = OprojSmem<D>;
   constexpr int DB = D / 64;
   constexpr uint32_t BLK = 128 * 128;
-  constexpr int MAX_A = 5;
+  constexpr int MAX_A = 3;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* sgen = smem_raw + (sbase - smem_u32(smem_raw));
   const ShDims& d = g.d;
   const int AS = g.a_stages;
-  const int HE = d.H * d.E;
-  const uint32_t a_off = 0, b_off = AS * SM::A_BYTES, misc_off = b_off + 2 * SM::B_BYTES;
-  int* s_idx = (int*)(sgen + misc_off);                       // [128, H, k]
+  const uint32_t a_off = 0, b_off = AS * 2 * SM::A_BYTES, misc_off = b_off + 2 * SM::B_BYTES;
+  int* s_idx = (int*)(sgen + misc_off);                       // [128, H, k] selections of the current tokens
   float* s_gt = (float*)(s_idx + 128 * d.H * d.k);            // [128, H, k]
-  float* s_g = s_gt + 128 * d.H * d.k;                        // [E, 128] gates of the current head
-  int* s_cnt = (int*)(s_g + d.E * 128);                       // [H*E]
-  uint64_t* bars = (uint64_t*)(((uintptr_t)(s_cnt + HE) + 15) & ~(uintptr_t)15);
+  uint64_t* bars = (uint64_t*)(((uintptr_t)(s_gt + 128 * d.H * d.k) + 15) & ~(uintptr_t)15);
   uint64_t* a_full = bars;               // [MAX_A]
   uint64_t* a_empty = bars + MAX_A;      // [MAX_A]
   uint64_t* b_full = bars + 2 * MAX_A;   // [2]
   uint64_t* b_empty = b_full + 2;        // [2]
-  uint64_t* d_full = b_empty + 2;        // [4]
-  uint64_t* d_empty = d_full + 4;        // [4]
-  uint32_t* tmem_slot = (uint32_t*)(d_empty + 4);
+  uint64_t* d_full = b_empty + 2;        // [2]
+  uint64_t* d_empty = d_full + 2;        // [2]
+  uint64_t* sel_free = d_empty + 2;      // epilogue threads are done with the selections copy
+  uint64_t* sel_ready = sel_free + 1;    // the selections copy of the current work unit is complete
+  uint32_t* tmem_slot = (uint32_t*)(sel_ready + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nfc = d.M / 128;
-  const int tt = blockIdx.x / nfc, fc = blockIdx.x % nfc;
-  const int row0 = tt * 128;
-  const int nrows = min(128, d.N - row0);
+  const int npair = (d.E + 1) / 2;       // items per head
   bool dead = false;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < MAX_A; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
-    for (int s = 0; s < 4; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 256); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 2);
+      mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 256);
+    }
+    mbar_init(sel_free, 256); mbar_init(sel_ready, 256);
     fence_barrier_init();
     tma_prefetch_desc(&mapAhat); tma_prefetch_desc(&mapWo);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
-  // destination-side counts of this tile, and its selections (contiguous in global memory)
-  for (int i = threadIdx.x; i < HE; i += blockDim.x) s_cnt[i] = g.blockcnt[(size_t)tt * d.G + HE + i];
-  {
-    const int per_tok = d.H * d.k;
-    const int total = nrows * per_tok;
-    const int* gi = g.idx + (size_t)row0 * per_tok;
-    const float* gg = g.gate + (size_t)row0 * per_tok;
-    for (int i = threadIdx.x; i < 128 * per_tok; i += blockDim.x) {
-      s_idx[i] = i < total ? gi[i] : 0;
-      s_gt[i] = i < total ? gg[i] : 0.f;
-    }
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -100,110 +94,135 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
 
   if (warp == 0) {
     if (lane == 0) {
-      int s = 0;
+      int s = 0, gh = 0;
       uint32_t e_par = 1;                                   // parity of a_empty[s] for the current ring pass
-      for (int h = 0; h < d.H; ++h) {
-        const int bs = h & 1;
-        if (!mbar_wait(&b_empty[bs], ((h >> 1) & 1) ^ 1, g.status, dead)) break;
-        mbar_expect_tx(&b_full[bs], SM::B_BYTES);
-#pragma unroll
-        for (int c = 0; c < DB; ++c)
-          tma_load_2d(sbase + b_off + bs * SM::B_BYTES + c * BLK, &mapAhat, &b_full[bs], h * D + c * 64, row0);
-        for (int e = 0; e < d.E && !dead; ++e) {
-          if (s_cnt[h * d.E + e] == 0) continue;
-          if (!mbar_wait(&a_empty[s], e_par, g.status, dead)) break;
-          mbar_expect_tx(&a_full[s], SM::A_BYTES);
+      for (int w = blockIdx.x; w < g.nwork && !dead; w += gridDim.x) {
+        const int row0 = (w / nfc) * 128, fc = w % nfc;
+        for (int h = 0; h < d.H && !dead; ++h, ++gh) {
+          const int bs = gh & 1;
+          if (!mbar_wait(&b_empty[bs], ((gh >> 1) & 1) ^ 1, g.status, dead)) break;
+          mbar_expect_tx(&b_full[bs], SM::B_BYTES);
 #pragma unroll
           for (int c = 0; c < DB; ++c)
-            tma_load_2d(sbase + a_off + s * SM::A_BYTES + c * BLK, &mapWo, &a_full[s], c * 64,
-                        (h * d.E + e) * d.M + fc * 128);
-          if (++s == AS) { s = 0; e_par ^= 1; }
+            tma_load_2d(sbase + b_off + bs * SM::B_BYTES + c * BLK, &mapAhat, &b_full[bs], h * D + c * 64, row0);
+          for (int p = 0; p < npair; ++p) {
+            const int e0 = 2 * p;
+            const bool two = e0 + 1 < d.E;
+            if (!mbar_wait(&a_empty[s], e_par, g.status, dead)) break;
+            mbar_expect_tx(&a_full[s], two ? 2 * SM::A_BYTES : SM::A_BYTES);
+            const uint32_t dst = sbase + a_off + s * 2 * SM::A_BYTES;
+            const int wrow = (h * d.E + e0) * d.M + fc * 128;
+#pragma unroll
+            for (int c = 0; c < DB; ++c) tma_load_2d(dst + c * BLK, &mapWo, &a_full[s], c * 64, wrow);
+            if (two) {
+#pragma unroll
+              for (int c = 0; c < DB; ++c) tma_load_2d(dst + SM::A_BYTES + c * BLK, &mapWo, &a_full[s], c * 64, wrow + d.M);
+            }
+            if (++s == AS) { s = 0; e_par ^= 1; }
+          }
         }
-        if (dead) break;
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 10) {
     if (lane == 0) {
+      const int iss = warp == 1 ? 0 : 1;                    // this issuer takes the items with gi % 2 == iss
       constexpr uint32_t idesc = make_idesc_f16(128, 128, 0, 0, 0);
-      const uint32_t a_lo0 = desc_lo_k(sbase + a_off), b_lo0 = desc_lo_k(sbase + b_off);
-      int it = 0, s = 0;
-      uint32_t a_par = 0;                                   // parity of a_full[s] for the current ring pass
-      for (int h = 0; h < d.H && !dead; ++h) {
-        const int bs = h & 1;
-        if (!mbar_wait(&b_full[bs], (h >> 1) & 1, g.status, dead)) break;
-        const uint32_t b_lo = b_lo0 + bs * (SM::B_BYTES >> 4);
-        for (int e = 0; e < d.E; ++e) {
-          if (s_cnt[h * d.E + e] == 0) continue;
-          const int buf = it & 3;
-          if (!mbar_wait(&a_full[s], a_par, g.status, dead)) break;
-          if (!mbar_wait(&d_empty[buf], ((it >> 2) & 1) ^ 1, g.status, dead)) break;
-          tc_fence_after();
-          const uint32_t a_lo = a_lo0 + s * (SM::A_BYTES >> 4);
-          const uint32_t td = tmem + buf * 128;
+      const uint32_t w_lo0 = desc_lo_k(sbase + a_off), t_lo0 = desc_lo_k(sbase + b_off);
+      int gh = 0, gi = 0;
+      for (int w = blockIdx.x; w < g.nwork && !dead; w += gridDim.x) {
+        for (int h = 0; h < d.H && !dead; ++h, ++gh) {
+          const int bs = gh & 1;
+          if (!mbar_wait(&b_full[bs], (gh >> 1) & 1, g.status, dead)) break;
+          const uint32_t t_lo = t_lo0 + bs * (SM::B_BYTES >> 4);
+          for (int p = 0; p < npair; ++p, ++gi) {
+            if ((gi & 1) != iss) continue;
+            const int nexp = (2 * p + 1 < d.E) ? 2 : 1;
+            const int buf = gi & 1;
+            const int s = AS == 2 ? buf : 0;                 // ring stage of item gi (AS is 1 or 2)
+            const uint32_t a_par = (AS == 2 ? (gi >> 1) : gi) & 1;
+            if (!mbar_wait(&a_full[s], a_par, g.status, dead)) break;
+            if (!mbar_wait(&d_empty[buf], ((gi >> 1) & 1) ^ 1, g.status, dead)) break;
+            tc_fence_after();
+            const uint32_t w_lo = w_lo0 + s * (2 * SM::A_BYTES >> 4);
+            const uint32_t td = tmem + buf * 256;
+            for (int x = 0; x < nexp; ++x) {
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
-            umma_f16(td, desc_pack(a_lo + koff), desc_pack(b_lo + koff), idesc, k != 0);
+              for (int k = 0; k < D / 16; ++k) {
+                const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+                umma_f16(td + x * 128, desc_pack(t_lo + koff), desc_pack(w_lo + x * (SM::A_BYTES >> 4) + koff), idesc, k != 0);
+              }
+            }
+            umma_commit(&a_empty[s]);
+            umma_commit(&d_full[buf]);
           }
-          umma_commit(&a_empty[s]);
-          umma_commit(&d_full[buf]);
-          ++it;
-          if (++s == AS) { s = 0; a_par ^= 1; }
+          umma_commit(&b_empty[bs]);
         }
-        umma_commit(&b_empty[bs]);
       }
     }
   } else {
-    // ---- epilogue: thread = output feature x token half; acc[t] = y[row0 + half*64 + t, feature] ----
+    // ---- epilogue: thread = token x feature half; acc[f] = y[row0 + token, fc*128 + half*64 + f] ----
     const int q = warp & 3;
     const int half = (warp - 2) >> 2;
-    const int f = q * 32 + lane;
-    const int et = threadIdx.x - 64;                      // 0..255; the first 128 build s_g (thread = token)
+    const int tok = q * 32 + lane;
+    const int et = threadIdx.x - 64;                       // 0..255
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    float acc[64];
-#pragma unroll
-    for (int t = 0; t < 64; ++t) acc[t] = 0.f;
-    int it = 0;
+    const int per_tok = d.H * d.k;
+    int gi = 0;
+    uint32_t wpar = 0;                                     // parity of this work unit for sel_free / sel_ready
     bool ok = true;
-    for (int h = 0; h < d.H && ok; ++h) {
-      // gates of this head: s_g[e][t] = gate if token t selected e, else 0
-      asm volatile("bar.sync 1, 256;" ::: "memory");      // everyone finished the previous head
-      for (int i = et; i < d.E * 128; i += 256) s_g[i] = 0.f;
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (et < nrows)
-        for (int j = 0; j < d.k; ++j) {
-          const int o = (et * d.H + h) * d.k + j;
-          s_g[s_idx[o] * 128 + et] = s_gt[o];
+    for (int w = blockIdx.x; w < g.nwork && ok; w += gridDim.x, wpar ^= 1) {
+      const int row0 = (w / nfc) * 128, fc = w % nfc;
+      const int nrows = min(128, d.N - row0);
+      // this tile's destination-side selections (contiguous in global memory) -> shared memory
+      // (mbarriers with bounded waits rather than bar.sync, so that a thread that gave up cannot
+      //  leave the others stuck)
+      mbar_arrive(sel_free);                               // this thread is done with the previous copy
+      if (!mbar_wait(sel_free, wpar, g.status, dead)) { ok = false; break; }
+      {
+        const int total = nrows * per_tok;
+        const int* gi_ = g.idx + (size_t)row0 * per_tok;
+        const float* gg = g.gate + (size_t)row0 * per_tok;
+        for (int i = et; i < 128 * per_tok; i += 256) {
+          s_idx[i] = i < total ? gi_[i] : -1;
+          s_gt[i] = i < total ? gg[i] : 0.f;
         }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      for (int e = 0; e < d.E; ++e) {
-        if (s_cnt[h * d.E + e] == 0) continue;
-        const int buf = it & 3;
-        if (!mbar_wait(&d_full[buf], (it >> 2) & 1, g.status, dead)) { ok = false; break; }
-        tc_fence_after();
-        const float4* ge = reinterpret_cast<const float4*>(s_g + e * 128 + half * 64);
-        uint32_t v[64];
-        tmem_ld32(tmem + lane_off + buf * 128 + half * 64, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-        tmem_ld32(tmem + lane_off + buf * 128 + half * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-        tmem_ld_wait();
-        tc_fence_before();
-        mbar_arrive(&d_empty[buf]);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float4 gv = ge[i];
-          acc[4 * i + 0] = fmaf(gv.x, __uint_as_float(v[4 * i + 0]), acc[4 * i + 0]);
-          acc[4 * i + 1] = fmaf(gv.y, __uint_as_float(v[4 * i + 1]), acc[4 * i + 1]);
-          acc[4 * i + 2] = fmaf(gv.z, __uint_as_float(v[4 * i + 2]), acc[4 * i + 2]);
-          acc[4 * i + 3] = fmaf(gv.w, __uint_as_float(v[4 * i + 3]), acc[4 * i + 3]);
-        }
-        ++it;
       }
-    }
-    if (ok) {
-      float* dst = g.out + (size_t)(row0 + half * 64) * d.M + fc * 128 + f;
+      mbar_arrive(sel_ready);
+      if (!mbar_wait(sel_ready, wpar, g.status, dead)) { ok = false; break; }
+      float acc[64];
 #pragma unroll
-      for (int t = 0; t < 64; ++t)
-        if (half * 64 + t < nrows) dst[(size_t)t * d.M] = acc[t];
+      for (int f = 0; f < 64; ++f) acc[f] = 0.f;
+      for (int h = 0; h < d.H && ok; ++h) {
+        const int sel = (tok * d.H + h) * d.k;               // this token's selections for head h
+        for (int p = 0; p < npair; ++p, ++gi) {
+          const int nexp = (2 * p + 1 < d.E) ? 2 : 1;
+          const int buf = gi & 1;
+          if (!mbar_wait(&d_full[buf], (gi >> 1) & 1, g.status, dead)) { ok = false; break; }
+          tc_fence_after();
+          for (int x = 0; x < nexp; ++x) {
+            const int e = 2 * p + x;
+            float gv = 0.f;                                  // gate of expert e for this token (0: not selected)
+            for (int j = 0; j < d.k; ++j)
+              if (s_idx[sel + j] == e) gv = s_gt[sel + j];
+            uint32_t v[64];
+            const uint32_t ta = tmem + lane_off + buf * 256 + x * 128 + half * 64;
+            tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+            tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+            tmem_ld_wait();
+            if (x == nexp - 1) {
+              tc_fence_before();
+              mbar_arrive(&d_empty[buf]);
+            }
+#pragma unroll
+            for (int f = 0; f < 64; ++f) acc[f] = fmaf(gv, __uint_as_float(v[f]), acc[f]);
+          }
+        }
+      }
+      if (ok && tok < nrows) {
+        float4* dst = reinterpret_cast<float4*>(g.out + (size_t)(row0 + tok) * d.M + fc * 128 + half * 64);
+#pragma unroll
+        for (int f = 0; f < 16; ++f) dst[f] = make_float4(acc[4 * f], acc[4 * f + 1], acc[4 * f + 2], acc[4 * f + 3]);
+      }
     }
   }
   tc_fence_before();
