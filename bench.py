@@ -159,7 +159,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2312_07987_b200 import binding, inputs
+    from paper_2312_07987_b200 import binding, inputs, sharding
 
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
     torch.cuda.set_device(local_rank)
@@ -170,10 +170,7 @@ def main():
 
     # each rank owns its own batch of independent sequences (same weights, rank-specific x)
     inp = inputs.make_inputs(cfg)
-    if rank > 0:
-        rng = np.random.Generator(np.random.PCG64(1000 + rank))
-        perm = rng.permutation(cfg.batch * cfg.seq)
-        inp.x = inp.x.reshape(-1, cfg.d_model)[perm].reshape(inp.x.shape)   # rows keep their gate margins
+    inp.x = sharding.rank_batch(inp.x, rank)                                 # rows keep their gate margins
     layer = binding.layer_from_inputs(inp)
     x = binding.to_device(inp.x, cfg.dtype)
     out = torch.empty(inp.x.shape, dtype=torch.float32, device="cuda")
@@ -243,16 +240,13 @@ def main():
     assert layer.sh_last_status() == 0, "device status word set during the timed region"
 
     # ---- max over ranks ----
-    tv = torch.tensor([t_total_ms, e2e_ms, warm_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tv, op=dist.ReduceOp.MAX)
-    t_total_ms, e2e_ms, warm_ms = tv.tolist()
+    t_total_ms, e2e_ms, warm_ms = sharding.max_over_ranks([t_total_ms, e2e_ms, warm_ms], device="cuda")
 
     if rank == 0:
         N = cfg.n_tokens
         fl = inputs.useful_flop(cfg)
         ms_step = t_total_ms / args.steps
-        value = world * N / (ms_step * 1e-3)
+        value = sharding.aggregate_throughput(N, world, ms_step * 1e-3)
         useful_tflops = world * fl["total"] / (ms_step * 1e-3) / 1e12
         stage_flop = dict(gate_topk_sort=0.0, qk_proj=fl["qk"], v_experts=fl["v"], attention=fl["attn_half"], o_experts=fl["o"])
         dom = int(np.argmax(stage[:5]))
