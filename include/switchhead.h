@@ -122,6 +122,33 @@ int sh_forward_timed(sh_layer* layer, const void* x, void* out, void* stream, fl
 int sh_gate_topk(sh_layer* layer, const void* x, int32_t* idx, float* gate, int32_t* offsets,
                  int32_t* lists, void* stream);
 
+/* (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
+ * Some callers run where cudaMalloc is not an option - inside a memory pool they do not own,
+ * in a process whose allocations are fixed at start-up, or simply without a workspace to
+ * hand over.  This entry point runs the gate + top-k + bucket-sort stage (the same kernels
+ * as sh_gate_topk on the CUDA cores) without a layer handle and without any allocation:
+ * its scratch memory - the per-block selection histograms, the gate values in list order
+ * and the row-tile table the sort kernel emits - lives in fixed arrays inside the library
+ * (about 2.3 MB on every GPU that loads it, held until the process exits).  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *   dtype    SH_F32 or SH_BF16: element type of x and w_gate
+ *   x        [n_tokens, d_model]
+ *   w_gate   [2*n_heads*n_experts, d_model]: one ROW per gate column, row (side*H + h)*E + e
+ *            (side 0 = source); i.e. W_S^h and W_D^h transposed and stacked
+ *   bias     [2*n_heads*n_experts] fp32 added to the logits, or NULL
+ *   idx, gate, offsets, lists: as for sh_gate_topk (all required here)
+ * Limits: n_tokens <= 16384, 2*n_heads*n_experts <= 256, n_tokens*n_heads*k <= 262144,
+ * n_experts <= 32, and n_heads*k small enough for the sort kernel's 48 KB of shared memory;
+ * anything larger is refused with SH_ERR_UNSUPPORTED and a message naming the limit.
+ * The first call on a device looks up the arrays' device addresses (a host-side set-up
+ * step), so make that first call outside any stream capture.  All calls on a device share
+ * the arrays, which keep the previous call's contents: nothing in them needs clearing
+ * between calls (each call overwrites what it reads), but two calls whose kernels overlap
+ * on the GPU - different streams, or different host threads - race on them; serialise them. */
+int sh_noalloc_gate_topk(int dtype, int n_tokens, int d_model, int n_heads, int n_experts, int k,
+                         const void* x, const void* w_gate, const float* bias, int32_t* idx,
+                         float* gate, int32_t* offsets, int32_t* lists, void* stream);
+
 /* Device pointer and size of an intermediate buffer inside the workspace (contents are
  * those of the last sh_forward / sh_gate_topk once the stream has drained).  Element type:
  * fp32 for SH_F32, fp16 for SH_BF16 (Q, K, V, AHAT); int32 / fp32 for the gate buffers.

@@ -50,6 +50,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_forward_timed.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float)]
     lib.sh_gate_topk.restype = i32
     lib.sh_gate_topk.argtypes = [vp] * 7
+    lib.sh_noalloc_gate_topk.restype = i32
+    lib.sh_noalloc_gate_topk.argtypes = [i32] * 6 + [vp] * 8
     lib.sh_debug_buffer.restype = i32
     lib.sh_debug_buffer.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(sz)]
     lib.sh_last_status.restype = i32
@@ -174,6 +176,22 @@ class Layer:
             self.close()
         except Exception:
             pass
+
+
+def sh_noalloc_gate_topk(dtype: int, x: torch.Tensor, w_gate: torch.Tensor, bias: Optional[torch.Tensor],
+                         n_heads: int, n_experts: int, k: int):
+    """Gate + top-k + bucket sort without a layer handle or workspace (see switchhead.h).
+    x [N, M]; w_gate [2*H*E, M] (one row per gate column); returns idx, gate, offsets, lists.
+    The output tensors are allocated here, by torch, before the call; the call itself allocates nothing."""
+    N, M = x.shape
+    dev = x.device
+    idx = torch.empty((2, N, n_heads, k), dtype=torch.int32, device=dev)
+    gate = torch.empty((2, N, n_heads, k), dtype=torch.float32, device=dev)
+    offsets = torch.empty((2, n_heads, n_experts + 1), dtype=torch.int32, device=dev)
+    lists = torch.empty((2, n_heads, N * k), dtype=torch.int32, device=dev)
+    _check(lib.sh_noalloc_gate_topk(dtype, N, M, n_heads, n_experts, k, _ptr(x), _ptr(w_gate), _ptr(bias),
+                                    _ptr(idx), _ptr(gate), _ptr(offsets), _ptr(lists), _stream()))
+    return idx, gate, offsets, lists
 
 
 def to_device(a: Optional[np.ndarray], dtype: int, device="cuda") -> Optional[torch.Tensor]:
