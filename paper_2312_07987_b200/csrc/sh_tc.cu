@@ -76,6 +76,10 @@ struct TcState {
   int qk_bn, o_bn, qk_variant;
   int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
+  // fork/join: the Q/K projection does not depend on the gate and sort kernels, so it runs on a
+  // side stream between two events recorded on the caller's stream
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 constexpr int QK_STAGES = 4;
@@ -88,7 +92,11 @@ static int set_smem(K kernel, int bytes) {
 
 void sh_tc_release(sh_layer* L) {
   if (L && L->tc) {
-    delete (TcState*)L->tc;
+    TcState* S = (TcState*)L->tc;
+    if (S->ev_fork) cudaEventDestroy(S->ev_fork);
+    if (S->ev_join) cudaEventDestroy(S->ev_join);
+    if (S->side) cudaStreamDestroy(S->side);
+    delete S;
     L->tc = nullptr;
   }
 }
@@ -105,8 +113,13 @@ int sh_tc_prepare(sh_layer* L) {
   const char* ov = getenv("SH_O_SCATTER");
   S->o_scatter = ov ? atoi(ov) : 0;
   const char* qv = getenv("SH_QK_VARIANT");
-  S->qk_variant = qv ? atoi(qv) : 0;
+  S->qk_variant = qv ? atoi(qv) : (((L->dense ? 3 : 2) * d.H * d.D) % 256 == 0 ? 2 : 0);
   S->qk_bn = (S->qk_variant == 2) ? 256 : 128;
+  if (!L->dense && !getenv("SH_NO_OVERLAP")) {
+    SH_CUDA_CHECK(cudaStreamCreateWithFlags(&S->side, cudaStreamNonBlocking));
+    SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_fork, cudaEventDisableTiming));
+    SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_join, cudaEventDisableTiming));
+  }
   S->o_bn = 128;
   const char* env = getenv("SH_SIMT_STAGES");
   S->simt_mask = env ? atoi(env) : 0;
@@ -213,6 +226,14 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   int* status = (int*)(ws + L->o.status);
 
   sh_mark(L, 0, st);
+  // stage-timed runs stay serial so that the stage boundaries mean something
+  const bool overlap = S->side && !L->ev && !(simt & SH_STAGE_QK);
+  cudaStream_t qst = st;
+  if (overlap) {
+    SH_CUDA_CHECK(cudaEventRecord(S->ev_fork, st));
+    SH_CUDA_CHECK(cudaStreamWaitEvent(S->side, S->ev_fork, 0));
+    qst = S->side;
+  }
   if (!L->dense) {
     if ((rc = tc_gate_sort(L, x, out, true, st))) return rc;
   }
@@ -224,6 +245,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   if (simt & SH_STAGE_QK) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_QK, x, out, st))) return rc;
   } else {
+    cudaStream_t st = qst;                                  // Q/K projection: side stream when overlapping
     TcGemmArgs g{};
     g.d = d; g.K = d.M; g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
     g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
@@ -239,6 +261,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     if (rc) return rc;
     L->launches += 1;
   }
+  if (overlap) SH_CUDA_CHECK(cudaEventRecord(S->ev_join, S->side));
   sh_mark(L, 2, st);
   // ---- value experts ---------------------------------------------------------------------------
   if (!L->dense) {
@@ -258,6 +281,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       L->launches += 1;
     }
   }
+  if (overlap) SH_CUDA_CHECK(cudaStreamWaitEvent(st, S->ev_join, 0));
   sh_mark(L, 3, st);
   // ---- attention ---------------------------------------------------------------------------------
   if (simt & SH_STAGE_ATTN) {
