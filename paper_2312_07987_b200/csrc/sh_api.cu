@@ -109,6 +109,7 @@ extern "C" int sh_configure(sh_layer* L, int dtype, int batch, int seq) {
   L->d.B = batch; L->d.T = seq; L->d.N = batch * seq;
   L->d.nblk = (L->d.N + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
   L->d.max_tiles = (int)((slots + SH_TILE_ROWS - 1) / SH_TILE_ROWS) + d0.H * d0.E;
+  L->d.tile_rows_src = SH_TILE_ROWS;
   L->ws = nullptr; L->ws_bytes = 0; L->weights_set = false;
   sh_tc_release(L);
   layout_workspace(L);

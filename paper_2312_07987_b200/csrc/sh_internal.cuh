@@ -20,6 +20,7 @@ struct ShDims {
   int G;                   // gate columns = 2*H*E
   int nblk;                // ceil(N / SH_TILE_ROWS)
   int max_tiles;           // upper bound on row tiles per side
+  int tile_rows_src;       // rows per tile of the source-side (value expert) tile table: 128 or 256
 };
 
 // Workspace sub-buffers (byte offsets from the workspace base).

@@ -91,7 +91,8 @@ sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const flo
 // selections in earlier blocks and the bucket total; from the totals the per-head exclusive
 // scan over experts.  It then places its own tokens, in ascending order, behind those of the
 // earlier blocks (a stable counting sort: within a bucket tokens stay ascending).  Block 0
-// also writes the offsets array and the row-tile table of the grouped GEMMs.
+// also writes the offsets array and the row-tile table of the grouped GEMMs (tiles of
+// d.tile_rows_src rows on the source side, 128 on the destination side).
 // Dynamic shared memory: 128*H*k*2*8 bytes (the block's idx and gate values, both sides)
 // + (6*G + 8) * 4 bytes.
 // ---------------------------------------------------------------------------------------
@@ -196,7 +197,8 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     int run = 0;
     for (int b = side * d.H * d.E; b < (side + 1) * d.H * d.E; ++b) {
       s_tbase[b] = run;
-      run += (s_tot[b] + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
+      const int tr = side == 0 ? d.tile_rows_src : SH_TILE_ROWS;
+      run += (s_tot[b] + tr - 1) / tr;
     }
     ntiles[side] = run;
   }
@@ -206,10 +208,11 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
     const int cnt = s_tot[b];
     ShTile* tp = tiles + (size_t)side * d.max_tiles + s_tbase[b];
-    for (int ti = i & 31; ti * SH_TILE_ROWS < cnt; ti += 32) {
+    const int tr = side == 0 ? d.tile_rows_src : SH_TILE_ROWS;
+    for (int ti = i & 31; ti * tr < cnt; ti += 32) {
       ShTile tl2;
-      tl2.h = h; tl2.e = e; tl2.row0 = s_off[b] + ti * SH_TILE_ROWS;
-      tl2.nrows = min(SH_TILE_ROWS, cnt - ti * SH_TILE_ROWS);
+      tl2.h = h; tl2.e = e; tl2.row0 = s_off[b] + ti * tr;
+      tl2.nrows = min(tr, cnt - ti * tr);
       tp[ti] = tl2;
     }
   }

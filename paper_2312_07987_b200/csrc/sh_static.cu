@@ -104,6 +104,7 @@ extern "C" int sh_noalloc_gate_topk(int dtype, int n_tokens, int d_model, int n_
   d.B = 1; d.T = n_tokens; d.N = n_tokens; d.G = (int)G;
   d.nblk = (n_tokens + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
   d.max_tiles = kMaxTiles;
+  d.tile_rows_src = SH_TILE_ROWS;
   cudaStream_t st = (cudaStream_t)stream;
   return dtype == SH_F32 ? run<float>(d, s, x, w_gate, bias, idx, gate, offsets, lists, st)
                          : run<__nv_bfloat16>(d, s, x, w_gate, bias, idx, gate, offsets, lists, st);

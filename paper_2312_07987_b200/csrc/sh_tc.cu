@@ -123,6 +123,16 @@ int sh_tc_prepare(sh_layer* L) {
   S->o_bn = 128;
   const char* env = getenv("SH_SIMT_STAGES");
   S->simt_mask = env ? atoi(env) : 0;
+  if (L->sm_count == 0) {
+    int dev = 0;
+    SH_CUDA_CHECK(cudaGetDevice(&dev));
+    SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
+  // value experts: 256-row tiles halve the weight traffic, but only pay off while there are
+  // enough of them to fill the SMs one and a half times
+  const long long slots = (long long)d.N * d.H * d.k;
+  const bool big = slots / 256 >= (3ll * L->sm_count) / 2;
+  L->d.tile_rows_src = (L->dense || (S->simt_mask & SH_STAGE_V) || getenv("SH_V_TILE128") || !big) ? 128 : 256;
   int rc;
   if ((rc = sh_tc_encode_2d(&S->map_wqk, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, S->qk_bn))) return rc;
   if (!L->dense) {
@@ -201,10 +211,10 @@ int sh_tc_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
   return tc_gate_sort(L, x, nullptr, false, st);
 }
 
-template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16>
+template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>
 static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, dim3 grid, cudaStream_t st) {
-  auto kern = sh_tc_gemm_kernel<BN, STAGES, MODE, A_BF16, B_BF16>;
-  constexpr int smem = GemmSmem<BN, STAGES>::TOTAL;
+  auto kern = sh_tc_gemm_kernel<BN, STAGES, MODE, A_BF16, B_BF16, MT>;
+  constexpr int smem = GemmSmem<BN, STAGES, MT>::TOTAL;
   static bool configured = false;
   if (!configured) {
     int rc = set_smem(kern, smem);
@@ -274,9 +284,15 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       g.lists = (const int*)(ws + L->o.lists); g.lgate = (const float*)(ws + L->o.lgate);
       g.tiles = (const ShTile*)(ws + L->o.tiles); g.ntiles = (const int*)(ws + L->o.ntiles);
       g.b_rows_per_group = d.D; g.out0 = ws + L->o.v; g.status = status;
-      dim3 grid(d.max_tiles, 1);
-      if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
-      else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
+      // 256-row tiles (two accumulators sharing the weight operand): at most half the 128-row bound plus one per group
+      dim3 grid(d.tile_rows_src == 256 ? d.max_tiles / 2 + d.H * d.E : d.max_tiles, 1);
+      if (d.tile_rows_src == 256) {
+        if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
+        else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
+      } else {
+        if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
+        else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
+      }
       if (rc) return rc;
       L->launches += 1;
     }

@@ -1,6 +1,7 @@
 // tcgen05 GEMM kernels of the bf16 configuration: the dense Q/K projection, the grouped
 // value-expert projection and the grouped output-expert projection with its gate-weighted
-// scatter-add epilogue.  One 128 x BN output tile per CTA, accumulator in TMEM, operands
+// scatter-add epilogue.  One (MT*128) x BN output tile per CTA (MT = 1 or 2 row tiles that
+// share the B operand, halving its L2 traffic), accumulators in TMEM, operands
 // staged in 128-byte-swizzled shared memory: B always by TMA, A by TMA (dense rows) or by
 // cp.async row gathers (rows addressed through a per-expert token list).
 //
@@ -34,19 +35,21 @@ struct TcGemmArgs {
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int MT = 1>
 struct GemmSmem {
-  static constexpr int A_BYTES = GEMM_BM * GEMM_BK * 2;
+  static constexpr int A_BYTES = MT * GEMM_BM * GEMM_BK * 2;
   static constexpr int B_BYTES = BN * GEMM_BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int BAR_OFF = STAGES * STAGE_BYTES;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;   // + barriers + alignment slack
 };
 
-template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16>
+template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>
 __global__ void __launch_bounds__(192)
 sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcGemmArgs g) {
-  using SM = GemmSmem<BN, STAGES>;
+  using SM = GemmSmem<BN, STAGES, MT>;
+  static_assert(MT * BN <= 512, "accumulators must fit the 512 TMEM columns");
+  constexpr int ROWS = MT * GEMM_BM;
   constexpr bool GATHER = (MODE == GEMM_V || MODE == GEMM_O);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -64,8 +67,8 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     const ShTile tl = g.tiles[blockIdx.x];
     th = tl.h; te = tl.e; row0 = tl.row0; nrows = tl.nrows;
   } else {
-    row0 = blockIdx.x * GEMM_BM;
-    nrows = min(GEMM_BM, g.nrows - row0);
+    row0 = blockIdx.x * ROWS;
+    nrows = min(ROWS, g.nrows - row0);
   }
   const int col0 = blockIdx.y * BN;
   const int KB = g.K / GEMM_BK;
@@ -82,7 +85,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     if (!GATHER) tma_prefetch_desc(&mapA);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, MT * BN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -98,7 +101,11 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         if (!mbar_wait(&empty_bar[s], ((kb / STAGES) & 1) ^ 1, g.status, dead)) break;
         const uint32_t sa = sbase + s * SM::STAGE_BYTES, sb = sa + SM::A_BYTES;
         mbar_expect_tx(&full_bar[s], GATHER ? SM::B_BYTES : SM::STAGE_BYTES);
-        if (!GATHER) tma_load_2d(sa, &mapA, &full_bar[s], kb * GEMM_BK, row0);
+        if (!GATHER) {
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            tma_load_2d(sa + mt * (GEMM_BM * GEMM_BK * 2), &mapA, &full_bar[s], kb * GEMM_BK, row0 + mt * GEMM_BM);
+        }
         tma_load_2d(sb, &mapB, &full_bar[s], kb * GEMM_BK, brow);
       }
     }
@@ -113,8 +120,12 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         tc_fence_after();
         const uint32_t a_lo = a_lo0 + s * (SM::STAGE_BYTES >> 4), b_lo = b_lo0 + s * (SM::STAGE_BYTES >> 4);
 #pragma unroll
-        for (int k = 0; k < GEMM_BK / 16; ++k)
-          umma_f16(tmem_d, desc_pack(a_lo + 2 * k), desc_pack(b_lo + 2 * k), idesc, (kb | k) != 0);
+        for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+          for (int k = 0; k < GEMM_BK / 16; ++k)
+            umma_f16(tmem_d + mt * BN, desc_pack(a_lo + mt * (GEMM_BM * GEMM_BK * 2 >> 4) + 2 * k), desc_pack(b_lo + 2 * k),
+                     idesc, (kb | k) != 0);
+        }
         umma_commit(&empty_bar[s]);
         if (++s == STAGES) { s = 0; par ^= 1; }
       }
@@ -125,12 +136,12 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
     if (GATHER) {
       // thread -> 16-byte chunk c of rows rb, rb+16, ... (8 threads cover one 128-byte row)
       const int c = et & 7, rb = et >> 3;
-      const char* src[8];
-      uint32_t ok[8];
+      const char* src[8 * MT];
+      uint32_t ok[8 * MT];
       const int abytes = A_BF16 ? 2 : 2;
       const long acol = (MODE == GEMM_O) ? (long)th * d.D : 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < 8 * MT; ++i) {
         const int r = rb + 16 * i;
         int tok = 0;
         ok[i] = 0;
@@ -144,7 +155,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         if (!mbar_wait(&empty_bar[s], ((kb / STAGES) & 1) ^ 1, g.status, dead)) break;
         const uint32_t sa = sbase + s * SM::STAGE_BYTES;
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 8 * MT; ++i)
           cp_async_16(sa + (rb + 16 * i) * 128 + dsw, src[i] + (long)kb * GEMM_BK * abytes, ok[i]);
         cp_async_commit();
         if (kb >= 2) {
@@ -159,9 +170,13 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
       if (!dead)
         for (; arrived < KB; ++arrived) mbar_arrive(&full_bar[arrived % STAGES]);
     }
-    // ---- epilogue: thread = accumulator row = TMEM lane --------------------------------------
+    // ---- epilogue: thread = accumulator row = TMEM lane (one pass per row tile) ---------------
     const int q = warp & 3;
-    const int r = q * 32 + lane;
+    const bool tm_ok = mbar_wait(tmem_full, 0, g.status, dead);
+    if (tm_ok) tc_fence_after();
+#pragma unroll 1
+    for (int mt = 0; mt < MT; ++mt) {
+    const int r = mt * GEMM_BM + q * 32 + lane;
     const bool live = r < nrows;
     int tok = 0;
     float gate = 0.f;
@@ -174,9 +189,8 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         tok = row0 + r;
       }
     }
-    if (mbar_wait(tmem_full, 0, g.status, dead)) {
-      tc_fence_after();
-      const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
+    if (tm_ok) {
+      const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + mt * BN;
       const int bb = tok / d.T, tt = tok % d.T;
 #pragma unroll 1
       for (int c00 = 0; c00 < BN; c00 += 64) {
@@ -233,12 +247,13 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         }
       }
     }
+    }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_d, BN);
+    tmem_dealloc(tmem_d, MT * BN);
   }
 }
 
