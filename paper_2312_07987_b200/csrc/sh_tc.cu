@@ -6,6 +6,7 @@
 #include "sh_simt.cuh"
 #include "sh_tc_gemm.cuh"
 #include "sh_tc_attn.cuh"
+#include "sh_tc_attn2.cuh"
 #include "sh_tc_gate.cuh"
 #include "sh_tc_oproj.cuh"
 
@@ -74,6 +75,7 @@ struct TcState {
   CUtensorMap map_wqk, map_wv, map_wo, map_ahat, map_wgate;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
   int qk_bn, o_bn, qk_variant;
+  int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
   int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
   // fork/join: the Q/K projection does not depend on the gate and sort kernels, so it runs on a
@@ -110,6 +112,7 @@ int sh_tc_prepare(sh_layer* L) {
   char* ws = L->ws;
   const int HD = d.H * d.D;
   const int nproj = L->dense ? 3 : 2;
+  S->attn_single_tile = getenv("SH_ATTN_SINGLE") ? 1 : 0;
   const char* ov = getenv("SH_O_SCATTER");
   S->o_scatter = ov ? atoi(ov) : 0;
   const char* qv = getenv("SH_QK_VARIANT");
@@ -305,15 +308,27 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   } else {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
-    const int nq = (d.T + 127) / 128;
-    const unsigned grid = (unsigned)(nq * d.B * d.H);
-    static bool cfg128 = false, cfg64 = false;
-    if (d.D == 128) {
-      if (!cfg128) { if ((rc = set_smem(sh_tc_attention_kernel<128>, AttnSmem<128>::TOTAL))) return rc; cfg128 = true; }
-      sh_tc_attention_kernel<128><<<grid, 192, AttnSmem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+    static bool cfg128 = false, cfg64 = false, cfg2_128 = false, cfg2_64 = false;
+    if (S->attn_single_tile) {
+      const int nq = (d.T + 127) / 128;
+      const unsigned grid = (unsigned)(nq * d.B * d.H);
+      if (d.D == 128) {
+        if (!cfg128) { if ((rc = set_smem(sh_tc_attention_kernel<128>, AttnSmem<128>::TOTAL))) return rc; cfg128 = true; }
+        sh_tc_attention_kernel<128><<<grid, 192, AttnSmem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+      } else {
+        if (!cfg64) { if ((rc = set_smem(sh_tc_attention_kernel<64>, AttnSmem<64>::TOTAL))) return rc; cfg64 = true; }
+        sh_tc_attention_kernel<64><<<grid, 192, AttnSmem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+      }
     } else {
-      if (!cfg64) { if ((rc = set_smem(sh_tc_attention_kernel<64>, AttnSmem<64>::TOTAL))) return rc; cfg64 = true; }
-      sh_tc_attention_kernel<64><<<grid, 192, AttnSmem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+      const int nq = (d.T + 255) / 256;
+      const unsigned grid = (unsigned)(nq * d.B * d.H);
+      if (d.D == 128) {
+        if (!cfg2_128) { if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc; cfg2_128 = true; }
+        sh_tc_attention2_kernel<128><<<grid, 320, Attn2Smem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+      } else {
+        if (!cfg2_64) { if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc; cfg2_64 = true; }
+        sh_tc_attention2_kernel<64><<<grid, 320, Attn2Smem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+      }
     }
     L->launches += 1;
   }

@@ -1,0 +1,278 @@
+// Causal softmax attention (Eq. 1 with the autoregressive mask) with TWO 128-query tiles per
+// CTA.  Both tiles read the same K/V stages, which halves the bytes pulled from L2 per FLOP -
+// the quantity that bounds the single-tile kernel - and while one tile's softmax runs on the
+// CUDA cores the tensor pipe works for the other tile.
+//
+// CTA = (batch, head, 256 queries); key/value tiles of 128 up to the diagonal of each query
+// tile (tile 0: steps 0..2*qt, tile 1: steps 0..2*qt+1).
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
+// warps 2..5 = softmax of query tile 0, warps 6..9 = softmax of query tile 1 (thread = query
+// row = TMEM lane).  TMEM columns: S0 at 0, S1 at 128, O0 at 256, O1 at 384.
+// P (fp16) goes through ONE shared-memory buffer used alternately by the two tiles; the
+// k-th use ("phase") may be written once the UMMAs of phase k-1 have completed (p_free).
+// Running maximum and rescale as in the single-tile kernel (raise only by more than 8 in
+// log2 units; O rescaled in TMEM when that happens).
+#pragma once
+#include "sh_tc_attn.cuh"
+
+namespace shtc {
+
+template <int D>
+struct Attn2Smem {
+  static constexpr int T_BYTES = 128 * D * 2;            // one 128-row tile of Q, K or V
+  static constexpr int P_BYTES = 128 * 128 * 2;
+  static constexpr int Q_OFF = 0;                          // 2 tiles
+  static constexpr int K_OFF = Q_OFF + 2 * T_BYTES;        // 2 stages
+  static constexpr int V_OFF = K_OFF + 2 * T_BYTES;        // 2 stages
+  static constexpr int P_OFF = V_OFF + 2 * T_BYTES;
+  static constexpr int BAR_OFF = P_OFF + P_BYTES;
+  static constexpr int TOTAL = BAR_OFF + 256 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(320, 1)
+sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                        const __grid_constant__ CUtensorMap mapV, TcAttnArgs g) {
+  using SM = Attn2Smem<D>;
+  constexpr int DB = D / 64;
+  constexpr uint32_t BLK = 128 * 128;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* sgen = smem_raw + (sbase - smem_u32(smem_raw));
+  uint64_t* bars = (uint64_t*)(sgen + SM::BAR_OFF);
+  uint64_t* q_full = bars;
+  uint64_t* k_full = bars + 1;    // [2]
+  uint64_t* k_empty = bars + 3;   // [2]
+  uint64_t* v_full = bars + 5;    // [2]
+  uint64_t* v_empty = bars + 7;   // [2]
+  uint64_t* s_full = bars + 9;    // [2] per query tile
+  uint64_t* s_empty = bars + 11;  // [2] per query tile
+  uint64_t* pv_done = bars + 13;  // [2] per query tile
+  uint64_t* p_full = bars + 15;
+  uint64_t* p_free = bars + 16;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 17);
+
+  const ShDims& d = g.d;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nq = (d.T + 255) / 256;
+  const int BH = d.B * d.H;
+  const int qt = nq - 1 - (int)(blockIdx.x / BH);        // heaviest query tiles first
+  const int bh = blockIdx.x % BH;
+  const int q0 = qt * 256;
+  const int n0 = 2 * qt + 1;                             // steps of query tile 0
+  const int n1 = (q0 + 128 < d.T) ? 2 * qt + 2 : 0;      // steps of query tile 1 (0: no such rows)
+  const int nsteps = n1 > n0 ? n1 : n0;
+  bool dead = false;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
+      mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
+      mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 128);
+      mbar_init(&pv_done[i], 1);
+    }
+    mbar_init(p_full, 128);
+    mbar_init(p_free, 1);
+    fence_barrier_init();
+    tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(q_full, (n1 > 0 ? 2 : 1) * SM::T_BYTES);
+      for (int t = 0; t < (n1 > 0 ? 2 : 1); ++t)
+#pragma unroll
+        for (int c = 0; c < DB; ++c)
+          tma_load_3d(sbase + SM::Q_OFF + t * SM::T_BYTES + c * BLK, &mapQ, q_full, c * 64, q0 + t * 128, bh);
+      for (int j = 0; j < nsteps; ++j) {
+        const int s = j & 1;
+        if (!mbar_wait(&k_empty[s], ((j >> 1) & 1) ^ 1, g.status, dead)) break;
+        mbar_expect_tx(&k_full[s], SM::T_BYTES);
+#pragma unroll
+        for (int c = 0; c < DB; ++c)
+          tma_load_3d(sbase + SM::K_OFF + s * SM::T_BYTES + c * BLK, &mapK, &k_full[s], c * 64, j * 128, bh);
+        if (!mbar_wait(&v_empty[s], ((j >> 1) & 1) ^ 1, g.status, dead)) break;
+        mbar_expect_tx(&v_full[s], SM::T_BYTES);
+#pragma unroll
+        for (int c = 0; c < DB; ++c)
+          tma_load_3d(sbase + SM::V_OFF + s * SM::T_BYTES + c * BLK, &mapV, &v_full[s], c * 64, j * 128, bh);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_f16(128, 128, 0, 0, 0);
+      constexpr uint32_t idesc_pv = make_idesc_f16(128, D, 0, 0, 1);
+      const uint32_t q_lo0 = desc_lo_k(sbase + SM::Q_OFF), k_lo0 = desc_lo_k(sbase + SM::K_OFF);
+      const uint32_t p_lo = desc_lo_k(sbase + SM::P_OFF), v_lo0 = desc_lo_mn(sbase + SM::V_OFF, BLK);
+      const int nt[2] = {n0, n1};
+      auto issue_s = [&](int t, int j) {                     // S_t = Q_t K_j^T
+        const uint32_t q_lo = q_lo0 + t * (SM::T_BYTES >> 4), k_lo = k_lo0 + (j & 1) * (SM::T_BYTES >> 4);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+          umma_f16(tmem + t * 128, desc_pack(q_lo + koff), desc_pack(k_lo + koff), idesc_s, k != 0);
+        }
+        umma_commit(&s_full[t]);
+      };
+      bool ok = mbar_wait(q_full, 0, g.status, dead) && mbar_wait(&k_full[0], 0, g.status, dead);
+      if (ok) {
+        tc_fence_after();
+        issue_s(0, 0);
+        if (n1 > 0) issue_s(1, 0);
+        umma_commit(&k_empty[0]);
+      }
+      uint32_t pp = 0;                                       // phase counter of the shared P buffer
+      for (int j = 0; ok && j < nsteps; ++j) {
+        const int s = j & 1;
+        if (!mbar_wait(&v_full[s], (j >> 1) & 1, g.status, dead)) break;
+        const uint32_t v_lo = v_lo0 + s * (SM::T_BYTES >> 4);
+        bool k_next_ready = false;
+        for (int t = 0; t < 2 && ok; ++t) {
+          if (j >= nt[t]) continue;
+          if (!mbar_wait(p_full, pp & 1, g.status, dead)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {                     // 128 keys in steps of 16
+            const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+            umma_f16(tmem + 256 + t * 128, desc_pack(p_lo + koff), desc_pack(v_lo + k * (2048 >> 4)), idesc_pv, (j | k) != 0);
+          }
+          umma_commit(p_free);
+          umma_commit(&pv_done[t]);
+          ++pp;
+          if (j + 1 < nt[t]) {
+            if (!k_next_ready) {
+              if (!mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, g.status, dead)) { ok = false; break; }
+              k_next_ready = true;
+            }
+            if (!mbar_wait(&s_empty[t], j & 1, g.status, dead)) { ok = false; break; }
+            tc_fence_after();
+            issue_s(t, j + 1);
+          }
+        }
+        if (!ok) break;
+        umma_commit(&v_empty[s]);
+        if (j + 1 < nsteps) umma_commit(&k_empty[(j + 1) & 1]);
+      }
+    }
+  } else {
+    // ---- softmax: warps 2..5 own query tile 0, warps 6..9 query tile 1; thread = query row ------
+    const int t = (warp - 2) >> 2;
+    const int n = t == 0 ? n0 : n1;
+    const int other = t == 0 ? n1 : n0;
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    const uint32_t tmem_s = tmem + t * 128, tmem_o = tmem + 256 + t * 128;
+    float m = -INFINITY, l = 0.f;
+    const uint32_t prow = sbase + SM::P_OFF + r * 128;
+    const uint32_t sw = (uint32_t)(r & 7);
+    bool ok = true;
+    for (int j = 0; j < n; ++j) {
+      if (!mbar_wait(&s_full[t], j & 1, g.status, dead)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t sv[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + lane_off + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(&s_empty[t]);
+      float mx = -INFINITY;
+      if (j == n - 1) {                                      // diagonal tile: key c visible iff c <= r
+#pragma unroll
+        for (int c = 0; c < 128; ++c) {
+          float v = (c <= r) ? __uint_as_float(sv[c]) : -INFINITY;
+          sv[c] = __float_as_uint(v);
+          mx = fmaxf(mx, v);
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
+      }
+      float alpha = 1.f;
+      bool raise = false;
+      if (mx > m + 8.f) {
+        alpha = fast_exp2(m - mx);                           // first tile: exp2(-inf) = 0
+        m = mx;
+        raise = j > 0;
+      }
+      float sum = 0.f;
+      uint32_t pk[64];
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        const float p0 = fast_exp2(__uint_as_float(sv[2 * c]) - m);
+        const float p1 = fast_exp2(__uint_as_float(sv[2 * c + 1]) - m);
+        sum += p0 + p1;
+        __half2 h = __floats2half2_rn(p0, p1);
+        pk[c] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      l = l * alpha + sum;
+      // phase of the shared P buffer this write is: tile 0 step j comes after min(j, n1) writes of
+      // tile 1; tile 1 step j after min(j + 1, n0) writes of tile 0
+      const int phase = j + (t == 0 ? (j < other ? j : other) : (j + 1 < other ? j + 1 : other));
+      if (phase > 0) {
+        if (!mbar_wait(p_free, (phase - 1) & 1, g.status, dead)) { ok = false; break; }
+        tc_fence_after();
+      }
+      if (j > 0 && __any_sync(0xffffffffu, raise)) {         // rescale this warp's 32 rows of O
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t ov[32];
+          tmem_ld32(tmem_o + lane_off + c * 32, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+          tmem_st32(tmem_o + lane_off + c * 32, ov);
+        }
+        tmem_st_wait();
+      }
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) {
+        const uint32_t addr = prow + (ch >> 3) * BLK + (((uint32_t)(ch & 7) ^ sw) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]),
+                     "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(p_full);
+    }
+    if (ok && n > 0 && mbar_wait(&pv_done[t], (n - 1) & 1, g.status, dead)) {
+      tc_fence_after();
+      const int tq = q0 + t * 128 + r;
+      const float inv = 1.f / l;
+      const int bb = bh / d.H, hh = bh % d.H;
+      __half* dst = g.ahat + (((size_t)bb * d.T + tq) * d.H + hh) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t ov[32];
+        tmem_ld32(tmem_o + lane_off + c * 32, ov);
+        tmem_ld_wait();
+        if (tq < d.T) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint32_t w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              __half2 h = __floats2half2_rn(__uint_as_float(ov[8 * i + 2 * u]) * inv, __uint_as_float(ov[8 * i + 2 * u + 1]) * inv);
+              w[u] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            *reinterpret_cast<uint4*>(dst + c * 32 + 8 * i) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace shtc
