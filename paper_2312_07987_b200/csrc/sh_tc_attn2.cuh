@@ -130,9 +130,21 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       uint32_t pp = 0;                                       // phase counter of the shared P buffer
       for (int j = 0; ok && j < nsteps; ++j) {
         const int s = j & 1;
+        // S of the NEXT step first: it only needs K(j+1) and the softmax warps to have read S(j) out
+        // of TMEM, so the next softmax can start while this step's P V products are still queued
+        if (j + 1 < nsteps) {
+          if (!mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, g.status, dead)) break;
+          for (int t = 0; t < 2 && ok; ++t) {
+            if (j + 1 >= nt[t]) continue;
+            if (!mbar_wait(&s_empty[t], j & 1, g.status, dead)) { ok = false; break; }
+            tc_fence_after();
+            issue_s(t, j + 1);
+          }
+          if (!ok) break;
+          umma_commit(&k_empty[(j + 1) & 1]);
+        }
         if (!mbar_wait(&v_full[s], (j >> 1) & 1, g.status, dead)) break;
         const uint32_t v_lo = v_lo0 + s * (SM::T_BYTES >> 4);
-        bool k_next_ready = false;
         for (int t = 0; t < 2 && ok; ++t) {
           if (j >= nt[t]) continue;
           if (!mbar_wait(p_full, pp & 1, g.status, dead)) { ok = false; break; }
@@ -145,19 +157,9 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           umma_commit(p_free);
           umma_commit(&pv_done[t]);
           ++pp;
-          if (j + 1 < nt[t]) {
-            if (!k_next_ready) {
-              if (!mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, g.status, dead)) { ok = false; break; }
-              k_next_ready = true;
-            }
-            if (!mbar_wait(&s_empty[t], j & 1, g.status, dead)) { ok = false; break; }
-            tc_fence_after();
-            issue_s(t, j + 1);
-          }
         }
         if (!ok) break;
         umma_commit(&v_empty[s]);
-        if (j + 1 < nsteps) umma_commit(&k_empty[(j + 1) & 1]);
       }
     }
   } else {
@@ -182,18 +184,20 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive(&s_empty[t]);
-      float mx = -INFINITY;
       if (j == n - 1) {                                      // diagonal tile: key c visible iff c <= r
 #pragma unroll
-        for (int c = 0; c < 128; ++c) {
-          float v = (c <= r) ? __uint_as_float(sv[c]) : -INFINITY;
-          sv[c] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
+        for (int c = 0; c < 128; ++c)
+          if (c > r) sv[c] = 0xff800000u;                    // -inf
       }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+#pragma unroll
+      for (int c = 0; c < 128; c += 4) {
+        mx4[0] = fmaxf(mx4[0], __uint_as_float(sv[c]));
+        mx4[1] = fmaxf(mx4[1], __uint_as_float(sv[c + 1]));
+        mx4[2] = fmaxf(mx4[2], __uint_as_float(sv[c + 2]));
+        mx4[3] = fmaxf(mx4[3], __uint_as_float(sv[c + 3]));
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       float alpha = 1.f;
       bool raise = false;
       if (mx > m + 8.f) {
@@ -201,17 +205,17 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         m = mx;
         raise = j > 0;
       }
-      float sum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) {
         const float p0 = fast_exp2(__uint_as_float(sv[2 * c]) - m);
         const float p1 = fast_exp2(__uint_as_float(sv[2 * c + 1]) - m);
-        sum += p0 + p1;
+        sum4[c & 3] += p0 + p1;
         __half2 h = __floats2half2_rn(p0, p1);
         pk[c] = *reinterpret_cast<uint32_t*>(&h);
       }
-      l = l * alpha + sum;
+      l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
       // phase of the shared P buffer this write is: tile 0 step j comes after min(j, n1) writes of
       // tile 1; tile 1 step j after min(j + 1, n0) writes of tile 0
       const int phase = j + (t == 0 ? (j < other ? j : other) : (j + 1 < other ? j + 1 : other));
