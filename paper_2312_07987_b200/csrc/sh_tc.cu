@@ -362,19 +362,19 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     }
     const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
     static int cfg_smem128 = 0, cfg_smem64 = 0;
-    int as = 2, smem = 0;
-    for (; as >= 1; --as) {
+    int as = 4, smem = 0;
+    for (; as >= 2; as >>= 1) {
       smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.k) : OprojSmem<64>::total(as, d.H, d.k);
       if (smem <= 227 * 1024) break;
     }
-    if (as < 1) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
-    a.a_stages = as;
+    if (as < 2) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
+    a.a_slots = as;
     if (d.D == 128) {
       if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
-      sh_tc_oproj_kernel<128><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo, a);
+      sh_tc_oproj_kernel<128><<<grid, 384, smem, st>>>(S->map_ahat, S->map_wo, a);
     } else {
       if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
-      sh_tc_oproj_kernel<64><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo, a);
+      sh_tc_oproj_kernel<64><<<grid, 384, smem, st>>>(S->map_ahat, S->map_wo, a);
     }
     L->launches += 1;
   } else {

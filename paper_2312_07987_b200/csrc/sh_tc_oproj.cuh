@@ -12,15 +12,18 @@
 // out is written exactly once (no atomics, no clearing, run-to-run deterministic).  The price
 // is that unselected tokens ride along in the UMMA (E/k times the useful FLOP of this stage).
 //
-// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer for the
-// even pipeline items, warp 10 = UMMA issuer for the odd items (two issuing threads, each
-// owning one TMEM buffer, so that one thread's barrier round trips hide behind the other's
-// UMMAs), warps 2..9 = epilogue (thread = one token = TMEM lane, and one half of the 128
-// features; two warps share a lane quarter).
-// Two experts of a head form one pipeline item (one weight stage of two tiles, one 256-column
-// TMEM buffer), so that every barrier round trip of the single UMMA-issuing thread is backed
-// by 1024 tensor-pipe cycles of work.  All rings run on across work units, so the producer
-// and the UMMA issuer work ahead into the next unit while the epilogue stores the last one.
+// Warp roles (384 threads): warps 0 and 11 = TMA producers (warp 0: token tiles and the first
+// 64-column block of every weight tile, warp 11: the second block - one thread issues a TMA
+// box only every ~150 ns), warp 1 = TMEM owner + UMMA issuer for the even pipeline items,
+// warp 10 = UMMA issuer for the odd items, warps 2..9 = epilogue (thread =
+// one token = TMEM lane, and one half of the 128 features; two warps share a lane quarter).
+// One expert = one pipeline item: a weight-tile slot (ring of 4) and a 128-column TMEM buffer
+// (ring of 4).  Both rings are deep on purpose: L2 answers a TMA load after ~0.9 us and the
+// epilogue hands a TMEM buffer back ~1000 cycles after the UMMAs that filled it were issued,
+// so with only two of either the tensor pipe idles most of the time.  The issuers alternate
+// experts, so one thread's barrier round trips hide behind the other's UMMAs.  All rings run
+// on across work units, so the producers and the issuers work ahead into the next unit while the epilogue
+// stores the last one.
 #pragma once
 #include "sh_tc_prims.cuh"
 
@@ -31,7 +34,7 @@ struct TcOprojArgs {
   const int* idx;        // destination side: [N, H, k]
   const float* gate;     // destination side: [N, H, k]
   float* out;            // [N, M]
-  int a_stages;          // stages of TWO weight tiles
+  int a_slots;           // weight-tile slots in the ring (power of two: 2 or 4)
   int nwork;             // nblk * (M / 128)
   int* status;
 };
@@ -40,24 +43,25 @@ template <int D>
 struct OprojSmem {
   static constexpr int A_BYTES = 128 * D * 2;            // one weight tile: 128 features x D
   static constexpr int B_BYTES = 128 * D * 2;            // Ahat tile: 128 tokens x D
-  static int total(int a_stages, int H, int k) {
-    return a_stages * 2 * A_BYTES + 2 * B_BYTES + 128 * H * k * 8 + 512 + 1024;
+  static int total(int a_slots, int H, int k) {
+    return a_slots * A_BYTES + 2 * B_BYTES + 128 * H * k * 8 + 512 + 1024;
   }
 };
 
 template <int D>
-__global__ void __launch_bounds__(352, 1)
+__global__ void __launch_bounds__(384, 1)
 sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g) {
   using SM = OprojSmem<D>;
   constexpr int DB = D / 64;
   constexpr uint32_t BLK = 128 * 128;
-  constexpr int MAX_A = 3;
+  constexpr int MAX_A = 4;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* sgen = smem_raw + (sbase - smem_u32(smem_raw));
   const ShDims& d = g.d;
-  const int AS = g.a_stages;
-  const uint32_t a_off = 0, b_off = AS * 2 * SM::A_BYTES, misc_off = b_off + 2 * SM::B_BYTES;
+  const int AS = g.a_slots;                // power of two
+  const int as_shift = AS == 4 ? 2 : 1;
+  const uint32_t a_off = 0, b_off = AS * SM::A_BYTES, misc_off = b_off + 2 * SM::B_BYTES;
   int* s_idx = (int*)(sgen + misc_off);                       // [128, H, k] selections of the current tokens
   float* s_gt = (float*)(s_idx + 128 * d.H * d.k);            // [128, H, k]
   uint64_t* bars = (uint64_t*)(((uintptr_t)(s_gt + 128 * d.H * d.k) + 15) & ~(uintptr_t)15);
@@ -65,23 +69,20 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   uint64_t* a_empty = bars + MAX_A;      // [MAX_A]
   uint64_t* b_full = bars + 2 * MAX_A;   // [2]
   uint64_t* b_empty = b_full + 2;        // [2]
-  uint64_t* d_full = b_empty + 2;        // [2]
-  uint64_t* d_empty = d_full + 2;        // [2]
-  uint64_t* sel_free = d_empty + 2;      // epilogue threads are done with the selections copy
+  uint64_t* d_full = b_empty + 2;        // [4]
+  uint64_t* d_empty = d_full + 4;        // [4]
+  uint64_t* sel_free = d_empty + 4;      // epilogue threads are done with the selections copy
   uint64_t* sel_ready = sel_free + 1;    // the selections copy of the current work unit is complete
   uint32_t* tmem_slot = (uint32_t*)(sel_ready + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nfc = d.M / 128;
-  const int npair = (d.E + 1) / 2;       // items per head
   bool dead = false;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < MAX_A; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 2);
-      mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 256);
-    }
+    for (int s = 0; s < MAX_A; ++s) { mbar_init(&a_full[s], DB); mbar_init(&a_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 2); }
+    for (int s = 0; s < 4; ++s) { mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 256); }
     mbar_init(sel_free, 256); mbar_init(sel_ready, 256);
     fence_barrier_init();
     tma_prefetch_desc(&mapAhat); tma_prefetch_desc(&mapWo);
@@ -92,67 +93,55 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 0) {
-    if (lane == 0) {
-      int s = 0, gh = 0;
-      uint32_t e_par = 1;                                   // parity of a_empty[s] for the current ring pass
+  if (warp == 0 || warp == 11) {
+    if (lane == 0 && (warp == 0 || DB == 2)) {
+      const int c = warp == 0 ? 0 : 1;                      // the 64-column block this producer loads
+      int gh = 0, ge = 0;                                   // running head / expert counters
       for (int w = blockIdx.x; w < g.nwork && !dead; w += gridDim.x) {
         const int row0 = (w / nfc) * 128, fc = w % nfc;
         for (int h = 0; h < d.H && !dead; ++h, ++gh) {
-          const int bs = gh & 1;
-          if (!mbar_wait(&b_empty[bs], ((gh >> 1) & 1) ^ 1, g.status, dead)) break;
-          mbar_expect_tx(&b_full[bs], SM::B_BYTES);
+          if (warp == 0) {
+            const int bs = gh & 1;
+            if (!mbar_wait(&b_empty[bs], ((gh >> 1) & 1) ^ 1, g.status, dead)) break;
+            mbar_expect_tx(&b_full[bs], SM::B_BYTES);
 #pragma unroll
-          for (int c = 0; c < DB; ++c)
-            tma_load_2d(sbase + b_off + bs * SM::B_BYTES + c * BLK, &mapAhat, &b_full[bs], h * D + c * 64, row0);
-          for (int p = 0; p < npair; ++p) {
-            const int e0 = 2 * p;
-            const bool two = e0 + 1 < d.E;
-            if (!mbar_wait(&a_empty[s], e_par, g.status, dead)) break;
-            mbar_expect_tx(&a_full[s], two ? 2 * SM::A_BYTES : SM::A_BYTES);
-            const uint32_t dst = sbase + a_off + s * 2 * SM::A_BYTES;
-            const int wrow = (h * d.E + e0) * d.M + fc * 128;
-#pragma unroll
-            for (int c = 0; c < DB; ++c) tma_load_2d(dst + c * BLK, &mapWo, &a_full[s], c * 64, wrow);
-            if (two) {
-#pragma unroll
-              for (int c = 0; c < DB; ++c) tma_load_2d(dst + SM::A_BYTES + c * BLK, &mapWo, &a_full[s], c * 64, wrow + d.M);
-            }
-            if (++s == AS) { s = 0; e_par ^= 1; }
+            for (int cc = 0; cc < DB; ++cc)
+              tma_load_2d(sbase + b_off + bs * SM::B_BYTES + cc * BLK, &mapAhat, &b_full[bs], h * D + cc * 64, row0);
+          }
+          for (int e = 0; e < d.E; ++e, ++ge) {
+            const int s = ge & (AS - 1);
+            if (!mbar_wait(&a_empty[s], ((ge >> as_shift) & 1) ^ 1, g.status, dead)) break;
+            mbar_expect_tx(&a_full[s], BLK);
+            tma_load_2d(sbase + a_off + s * SM::A_BYTES + c * BLK, &mapWo, &a_full[s], c * 64,
+                        (h * d.E + e) * d.M + fc * 128);
           }
         }
       }
     }
   } else if (warp == 1 || warp == 10) {
     if (lane == 0) {
-      const int iss = warp == 1 ? 0 : 1;                    // this issuer takes the items with gi % 2 == iss
+      const int iss = warp == 1 ? 0 : 1;                    // this issuer takes the experts with ge % 2 == iss
       constexpr uint32_t idesc = make_idesc_f16(128, 128, 0, 0, 0);
       const uint32_t w_lo0 = desc_lo_k(sbase + a_off), t_lo0 = desc_lo_k(sbase + b_off);
-      int gh = 0, gi = 0;
+      int gh = 0, ge = 0;
       for (int w = blockIdx.x; w < g.nwork && !dead; w += gridDim.x) {
         for (int h = 0; h < d.H && !dead; ++h, ++gh) {
           const int bs = gh & 1;
           if (!mbar_wait(&b_full[bs], (gh >> 1) & 1, g.status, dead)) break;
           const uint32_t t_lo = t_lo0 + bs * (SM::B_BYTES >> 4);
-          for (int p = 0; p < npair; ++p, ++gi) {
-            if ((gi & 1) != iss) continue;
-            const int nexp = (2 * p + 1 < d.E) ? 2 : 1;
-            const int buf = gi & 1;
-            const int s = AS == 2 ? buf : 0;                 // ring stage of item gi (AS is 1 or 2)
-            const uint32_t a_par = (AS == 2 ? (gi >> 1) : gi) & 1;
-            if (!mbar_wait(&a_full[s], a_par, g.status, dead)) break;
-            if (!mbar_wait(&d_empty[buf], ((gi >> 1) & 1) ^ 1, g.status, dead)) break;
+          for (int e = 0; e < d.E; ++e, ++ge) {
+            if ((ge & 1) != iss) continue;
+            const int s = ge & (AS - 1), buf = ge & 3;
+            if (!mbar_wait(&a_full[s], (ge >> as_shift) & 1, g.status, dead)) break;
+            if (!mbar_wait(&d_empty[buf], ((ge >> 2) & 1) ^ 1, g.status, dead)) break;
             tc_fence_after();
-            const uint32_t w_lo = w_lo0 + s * (2 * SM::A_BYTES >> 4);
-            const uint32_t td = tmem + buf * 256;
-            for (int x = 0; x < nexp; ++x) {
+            const uint32_t w_lo = w_lo0 + s * (SM::A_BYTES >> 4);
 #pragma unroll
-              for (int k = 0; k < D / 16; ++k) {
-                const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
-                umma_f16(td + x * 128, desc_pack(t_lo + koff), desc_pack(w_lo + x * (SM::A_BYTES >> 4) + koff), idesc, k != 0);
-              }
+            for (int k = 0; k < D / 16; ++k) {
+              const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
+              umma_f16(tmem + buf * 128, desc_pack(t_lo + koff), desc_pack(w_lo + koff), idesc, k != 0);
             }
-            umma_commit(&a_empty[s]);
+            umma_commit(&a_empty[s]);                       // this slot can load its next tile
             umma_commit(&d_full[buf]);
           }
           umma_commit(&b_empty[bs]);
@@ -167,7 +156,7 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
     const int et = threadIdx.x - 64;                       // 0..255
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const int per_tok = d.H * d.k;
-    int gi = 0;
+    int ge = 0;
     uint32_t wpar = 0;                                     // parity of this work unit for sel_free / sel_ready
     bool ok = true;
     for (int w = blockIdx.x; w < g.nwork && ok; w += gridDim.x, wpar ^= 1) {
@@ -194,28 +183,22 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
       for (int f = 0; f < 64; ++f) acc[f] = 0.f;
       for (int h = 0; h < d.H && ok; ++h) {
         const int sel = (tok * d.H + h) * d.k;               // this token's selections for head h
-        for (int p = 0; p < npair; ++p, ++gi) {
-          const int nexp = (2 * p + 1 < d.E) ? 2 : 1;
-          const int buf = gi & 1;
-          if (!mbar_wait(&d_full[buf], (gi >> 1) & 1, g.status, dead)) { ok = false; break; }
+        for (int e = 0; e < d.E; ++e, ++ge) {
+          const int buf = ge & 3;
+          float gv = 0.f;                                    // gate of expert e for this token (0: not selected)
+          for (int j = 0; j < d.k; ++j)
+            if (s_idx[sel + j] == e) gv = s_gt[sel + j];
+          if (!mbar_wait(&d_full[buf], (ge >> 2) & 1, g.status, dead)) { ok = false; break; }
           tc_fence_after();
-          for (int x = 0; x < nexp; ++x) {
-            const int e = 2 * p + x;
-            float gv = 0.f;                                  // gate of expert e for this token (0: not selected)
-            for (int j = 0; j < d.k; ++j)
-              if (s_idx[sel + j] == e) gv = s_gt[sel + j];
-            uint32_t v[64];
-            const uint32_t ta = tmem + lane_off + buf * 256 + x * 128 + half * 64;
-            tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-            tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-            tmem_ld_wait();
-            if (x == nexp - 1) {
-              tc_fence_before();
-              mbar_arrive(&d_empty[buf]);
-            }
+          uint32_t v[64];
+          const uint32_t ta = tmem + lane_off + buf * 128 + half * 64;
+          tmem_ld32(ta, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+          tmem_ld32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+          tmem_ld_wait();
+          tc_fence_before();
+          mbar_arrive(&d_empty[buf]);
 #pragma unroll
-            for (int f = 0; f < 64; ++f) acc[f] = fmaf(gv, __uint_as_float(v[f]), acc[f]);
-          }
+          for (int f = 0; f < 64; ++f) acc[f] = fmaf(gv, __uint_as_float(v[f]), acc[f]);
         }
       }
       if (ok && tok < nrows) {
