@@ -72,7 +72,7 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
-  CUtensorMap map_wqk, map_wv, map_wo, map_ahat, map_wgate;
+  CUtensorMap map_wqk, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
   int qk_bn, o_bn, qk_variant;
   int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
@@ -141,6 +141,7 @@ int sh_tc_prepare(sh_layer* L) {
   if (!L->dense) {
     if ((rc = sh_tc_encode_2d(&S->map_wv, 0, ws + L->o.wv, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, S->o_bn))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_wo256, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 256))) return rc;
   } else {
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, S->o_bn))) return rc;
   }
@@ -354,7 +355,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     const size_t side1 = (size_t)d.N * d.H * d.k;
     a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
     a.out = (float*)out; a.status = status;
-    a.nwork = d.nblk * (d.M / 128);
+    a.nwork = d.nblk * ((d.M + 255) / 256);
     if (L->sm_count == 0) {
       int dev = 0;
       SH_CUDA_CHECK(cudaGetDevice(&dev));
@@ -362,8 +363,8 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     }
     const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
     static int cfg_smem128 = 0, cfg_smem64 = 0;
-    int as = 4, smem = 0;
-    for (; as >= 2; as >>= 1) {
+    int as = 3, smem = 0;
+    for (; as >= 2; --as) {
       smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.k) : OprojSmem<64>::total(as, d.H, d.k);
       if (smem <= 227 * 1024) break;
     }
@@ -371,10 +372,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     a.a_slots = as;
     if (d.D == 128) {
       if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
-      sh_tc_oproj_kernel<128><<<grid, 384, smem, st>>>(S->map_ahat, S->map_wo, a);
+      sh_tc_oproj_kernel<128><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo256, a);
     } else {
       if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
-      sh_tc_oproj_kernel<64><<<grid, 384, smem, st>>>(S->map_ahat, S->map_wo, a);
+      sh_tc_oproj_kernel<64><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo256, a);
     }
     L->launches += 1;
   } else {
