@@ -12,14 +12,16 @@
 // out is written exactly once (no atomics, no clearing, run-to-run deterministic).  The price
 // is that unselected tokens ride along in the UMMA (E/k times the useful FLOP of this stage).
 //
-// Why 256 features: on this part a 128 x N x 16 UMMA takes ~134 cycles for N = 64, 128 and
-// 256 alike (measured, operands resident in shared memory), so only N = 256 runs the tensor
-// pipe at its full rate; with N = 128 this kernel was tensor-bound at half speed whatever the
-// pipeline depth.
+// Why 256 features: the UMMA-issuing thread pays a fixed price per expert (barrier waits,
+// fence, commits: ~400 cycles during which the tensor pipe drains, because tcgen05.mma issue
+// is throttled to the pipe's own rate and queues almost nothing ahead), and every work unit
+// re-reads the token tiles.  N = 256 doubles the tensor work behind each fixed price and
+// halves the token-tile traffic; the accumulators (128 tokens x 256 features fp32) just fit
+// the registers of 256 epilogue threads.
 //
-// Warp roles (352 threads): warp 0 = TMA producer, warps 1 and 10 = UMMA issuers for the even /
-// odd experts (each owns one of the two TMEM buffers, so one thread's barrier round trips hide
-// behind the other's UMMAs; warp 1 also owns the TMEM allocation), warps 2..9 = epilogue (thread = one token = TMEM lane, and one half of the 256 features;
+// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer (warp 10
+// can issue the odd experts when built with OPROJ_ISSUERS = 2; measured: no gain),
+// warps 2..9 = epilogue (thread = one token = TMEM lane, and one half of the 256 features;
 // two warps share a lane quarter).  One expert = one 256-column TMEM buffer (ring of 2); its
 // weights arrive as D/64 stages of 256 features x 64 columns (32 KB, one TMA box each) through
 // a ring of 3 (or 2) stages that are released one by one: L2 answers a TMA load after ~0.9 us,
