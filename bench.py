@@ -26,6 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 DEFAULT_CONFIG = "c4_262m_bf16"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's main kernel, from the ncu
+# capture summarised in profiles/c4_262m_bf16_forward_kernels.md (MB, workload c4_262m_bf16)
+DRAM_TRAFFIC_MB = {"c4_262m_bf16": {"gate_topk_sort": 16.87 + 1.09, "qk_proj": 18.89, "v_experts": 29.92,
+                                    "attention": 25.21, "o_experts": 13.18}}
 STAGES = ["gate_topk_sort", "qk_proj", "v_experts", "attention", "o_experts"]
 
 
@@ -261,7 +265,9 @@ def main():
         else:
             ach = stage_flop[dom_name] / (stage[dom] * 1e-3) / 1e12
             roof = dict(bound="tensor", achieved=ach, peak=peaks["tflops"], unit="TFLOP/s", frac=ach / peaks["tflops"], traffic=None)
-        roof.update(kernel=dom_name, ms=float(stage[dom]), peak_source=peaks["source"])
+        traffic = DRAM_TRAFFIC_MB.get(cfg.name, {}).get(dom_name)
+        roof.update(kernel=dom_name, ms=float(stage[dom]), peak_source=peaks["source"],
+                    traffic=None if traffic is None else traffic * 1e6, traffic_unit="bytes per launch (ncu)")
 
         line = {
             "metric": "switchhead_layer_fwd_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
