@@ -5,6 +5,7 @@
 #include "sh_internal.cuh"
 #include "sh_simt.cuh"
 #include "sh_tc_gemm.cuh"
+#include "sh_tc_pgemm.cuh"
 #include "sh_tc_attn.cuh"
 #include "sh_tc_attn2.cuh"
 #include "sh_tc_gate.cuh"
@@ -75,6 +76,7 @@ struct TcState {
   CUtensorMap map_wqk, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
   int qk_bn, o_bn, qk_variant;
+  int persistent;       // 1 = persistent Q/K and value-expert GEMMs (default); 0 = one CTA per tile (experiment switch)
   int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
   int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
@@ -113,6 +115,7 @@ int sh_tc_prepare(sh_layer* L) {
   const int HD = d.H * d.D;
   const int nproj = L->dense ? 3 : 2;
   S->attn_single_tile = getenv("SH_ATTN_SINGLE") ? 1 : 0;
+  S->persistent = getenv("SH_NO_PERSISTENT") ? 0 : 1;
   const char* ov = getenv("SH_O_SCATTER");
   S->o_scatter = ov ? atoi(ov) : 0;
   const char* qv = getenv("SH_QK_VARIANT");
@@ -215,6 +218,20 @@ int sh_tc_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
   return tc_gate_sort(L, x, nullptr, false, st);
 }
 
+template <int BN, int STAGES, int MODE, int MT>
+static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, unsigned grid, cudaStream_t st) {
+  auto kern = sh_tc_pgemm_kernel<BN, STAGES, MODE, MT>;
+  constexpr int smem = PGemmSmem<BN, STAGES, MT>::TOTAL;
+  static bool configured = false;
+  if (!configured) {
+    int rc = set_smem(kern, smem);
+    if (rc != SH_OK) return rc;
+    configured = true;
+  }
+  kern<<<grid, 320, smem, st>>>(mapA, mapB, g);
+  return SH_OK;
+}
+
 template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>
 static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, dim3 grid, cudaStream_t st) {
   auto kern = sh_tc_gemm_kernel<BN, STAGES, MODE, A_BF16, B_BF16, MT>;
@@ -268,7 +285,12 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     dim3 grid(d.nblk, (g.ncols + S->qk_bn - 1) / S->qk_bn);
     switch (S->qk_variant) {
       case 1: rc = launch_gemm<128, 3, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
-      case 2: rc = launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
+      case 2: {
+        const unsigned tiles = (unsigned)(d.nblk * ((g.ncols + 255) / 256));
+        rc = S->persistent ? launch_pgemm<256, 4, PG_QKV, 1>(map_x, S->map_wqk, g, tiles < (unsigned)L->sm_count ? tiles : (unsigned)L->sm_count, st)
+                           : launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st);
+        break;
+      }
       case 3: rc = launch_gemm<128, 6, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
       default: rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
     }
@@ -291,7 +313,8 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       // 256-row tiles (two accumulators sharing the weight operand): at most half the 128-row bound plus one per group
       dim3 grid(d.tile_rows_src == 256 ? d.max_tiles / 2 + d.H * d.E : d.max_tiles, 1);
       if (d.tile_rows_src == 256) {
-        if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
+        if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 2>(map_x, S->map_wv, g, grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count, st)
+                                           : launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
         else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
       } else {
         if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
