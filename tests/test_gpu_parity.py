@@ -80,6 +80,15 @@ def test_bf16_edge_shapes(T, B, E, k, H, D):
     full_check(inputs.make_inputs(cfg))
 
 
+@pytest.mark.parametrize("M,T,B,E,k,H,D", [(384, 300, 3, 6, 2, 2, 128),    # d_model not a multiple of 256
+                                              (640, 700, 2, 3, 1, 1, 64),     # odd E, one head, ragged 256-row tiles
+                                              (1024, 1100, 20, 4, 2, 2, 128), # enough selections for 256-row value tiles
+                                              (512, 257, 1, 32, 4, 4, 64)])   # E = 32, a query tile with one row
+def test_bf16_wider_shapes(M, T, B, E, k, H, D):
+    cfg = inputs.LayerConfig("edge_bf16_wide", inputs.DTYPE_BF16, B, T, M, H, D, E, k, seed=300 + T)
+    full_check(inputs.make_inputs(cfg))
+
+
 def test_causality_on_gpu():
     cfg = inputs.CONFIGS["small_bf16"]
     inp = inputs.make_inputs(cfg, batch=2)
