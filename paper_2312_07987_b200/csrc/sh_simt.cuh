@@ -119,6 +119,24 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
   const int tok0 = blk * SH_TILE_ROWS;
   const int nrows = min(SH_TILE_ROWS, d.N - tok0);
   for (int i = tid; i < 2 * nb; i += blockDim.x) s_pre[i] = 0;   // s_pre and s_tot
+  // bucket b = tid % nb; the thread sums the blocks part, part + parts, ... in registers.  These
+  // loads do not depend on the selections copy below, so both are in flight together.
+  int my_b = -1, my_tot = 0, my_pre = 0;
+  {
+    const int parts = max(1, (int)blockDim.x / nb);
+    if (nb <= (int)blockDim.x) {
+      if (tid / nb < parts) {
+        my_b = tid % nb;
+        const int part = tid / nb;
+#pragma unroll 4
+        for (int bk = part; bk < d.nblk; bk += parts) {
+          const int c = blockcnt[(size_t)bk * nb + my_b];
+          my_tot += c;
+          my_pre += bk < blk ? c : 0;
+        }
+      }
+    }
+  }
   for (int side = 0; side < 2; ++side) {                          // this block's selections
     const size_t base = ((size_t)side * d.N + tok0) * per_tok;
     for (int i = tid; i < nrows * per_tok; i += blockDim.x) {
@@ -127,20 +145,19 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     }
   }
   __syncthreads();
-  {
-    // bucket b = tid % nb; the thread sums the blocks part, part + parts, ... in registers
-    const int parts = max(1, (int)blockDim.x / nb);
-    for (int b = tid % nb + (tid / nb / parts) * nb; b < nb; b += blockDim.x) {  // executes once unless nb > blockDim
-      const int part = (tid / nb) % parts;
+  if (my_b >= 0) {
+    if (my_tot) atomicAdd(&s_tot[my_b], my_tot);
+    if (my_pre) atomicAdd(&s_pre[my_b], my_pre);
+  } else if (nb > (int)blockDim.x) {                              // more buckets than threads: plain loop
+    for (int b = tid; b < nb; b += blockDim.x) {
       int tot = 0, pre = 0;
-#pragma unroll 4
-      for (int bk = part; bk < d.nblk; bk += parts) {
+      for (int bk = 0; bk < d.nblk; ++bk) {
         const int c = blockcnt[(size_t)bk * nb + b];
         tot += c;
         pre += bk < blk ? c : 0;
       }
-      if (tot) atomicAdd(&s_tot[b], tot);
-      if (pre) atomicAdd(&s_pre[b], pre);
+      s_tot[b] = tot;
+      s_pre[b] = pre;
     }
   }
   __syncthreads();

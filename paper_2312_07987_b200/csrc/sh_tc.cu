@@ -160,11 +160,11 @@ int sh_tc_prepare(sh_layer* L) {
   return SH_OK;
 }
 
-constexpr int GATE_STAGES = 4;
-
-static int gate_smem_bytes(int Gp, int G) {
+// The gate kernel's x stream comes cold from HBM (~1.2 us per box round trip), so what bounds its
+// main loop is the bytes in flight per CTA: 8 stages when they fit, else 4.
+static int gate_smem_bytes(int Gp, int G, int stages) {
   const int stage = 128 * 64 * 2 + ((Gp * 128 + 1023) & ~1023);
-  const int pipe = GATE_STAGES * stage, stag = 128 * (Gp + 1) * 4;
+  const int pipe = stages * stage, stag = 128 * (Gp + 1) * 4;
   const int bar_off = ((pipe > stag ? pipe : stag) + 1023) & ~1023;
   return bar_off + 256 + 3 * G * 4 + 1024;
 }
@@ -193,13 +193,15 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.zero_v = zero_for_forward ? (__half*)(ws + L->o.v) : nullptr;
   g.zero_out = (zero_for_forward && (S->o_scatter || (S->simt_mask & SH_STAGE_O))) ? (float*)out : nullptr;
   g.status = (int*)(ws + L->o.status);
-  const int smem = gate_smem_bytes(S->gate_gp, d.G);
-  static int configured = 0;
-  if (configured < smem) {
-    if ((rc = set_smem(sh_tc_gate_kernel<GATE_STAGES>, smem))) return rc;
-    configured = smem;
+  const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
+  const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
+  static int configured[2] = {0, 0};
+  if (configured[deep] < smem) {
+    if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
+    configured[deep] = smem;
   }
-  sh_tc_gate_kernel<GATE_STAGES><<<d.nblk, 192, smem, st>>>(map_x, S->map_wgate, g);
+  if (deep) sh_tc_gate_kernel<8><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
+  else sh_tc_gate_kernel<4><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
   const size_t ssm = sh_sort_smem_bytes(d);
   static size_t sort_cfg = 48 * 1024;
   if (ssm > sort_cfg) {

@@ -6,8 +6,9 @@
 // runs, the otherwise idle epilogue warps clear the V and out rows of the CTA's tokens (both
 // are accumulated into later).
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
-// warps 2..5 = zero-fill, then selection epilogue.
+// Warp roles (224 threads): warps 0 and 6 = TMA producers (x boxes / gate-weight boxes: one
+// thread issues a box only every ~150 ns), warp 1 = TMEM owner + UMMA issuer, warps 2..5 =
+// zero-fill, then selection epilogue.
 #pragma once
 #include "sh_tc_prims.cuh"
 
@@ -25,7 +26,7 @@ struct TcGateArgs {
 };
 
 template <int STAGES>
-__global__ void __launch_bounds__(192)
+__global__ void __launch_bounds__(224)
 sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, TcGateArgs g) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -51,7 +52,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   while ((int)tmem_cols < Gp) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
     mbar_init(tmem_full, 1);
     fence_barrier_init();
     tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapW);
@@ -63,15 +64,19 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 6) {
     if (lane == 0) {
       for (int kb = 0; kb < KB; ++kb) {
         const int s = kb % STAGES;
         if (!mbar_wait(&empty_bar[s], ((kb / STAGES) & 1) ^ 1, g.status, dead)) break;
         const uint32_t sa = sbase + s * stage_bytes, sb = sa + a_bytes;
-        mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-        tma_load_2d(sa, &mapX, &full_bar[s], kb * 64, row0);
-        tma_load_2d(sb, &mapW, &full_bar[s], kb * 64, 0);
+        if (warp == 0) {
+          mbar_expect_tx(&full_bar[s], a_bytes);
+          tma_load_2d(sa, &mapX, &full_bar[s], kb * 64, row0);
+        } else {
+          mbar_expect_tx(&full_bar[s], b_bytes);
+          tma_load_2d(sb, &mapW, &full_bar[s], kb * 64, 0);
+        }
       }
     }
   } else if (warp == 1) {
