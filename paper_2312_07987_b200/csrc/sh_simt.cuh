@@ -119,6 +119,10 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
   const int tok0 = blk * SH_TILE_ROWS;
   const int nrows = min(SH_TILE_ROWS, d.N - tok0);
   for (int i = tid; i < 2 * nb; i += blockDim.x) s_pre[i] = 0;   // s_pre and s_tot
+  // programmatic dependent launch (no-ops in an ordinary launch): let the next kernel in the
+  // stream become resident, then wait for the gate kernel's selections to be complete and visible
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // bucket b = tid % nb; the thread sums the blocks part, part + parts, ... in registers.  These
   // loads do not depend on the selections copy below, so both are in flight together.
   int my_b = -1, my_tot = 0, my_pre = 0;
@@ -236,8 +240,9 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
 }
 
 static inline int sh_sort_threads(const ShDims& d) {
+  // at most 512 threads (16 K registers), so that a block fits beside a 320-thread GEMM CTA on an SM
   int gs = 2 * d.H;
-  if (gs > 8) gs = 8;
+  if (gs > 4) gs = 4;
   return 128 * gs;
 }
 

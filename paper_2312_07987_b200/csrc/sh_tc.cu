@@ -1,6 +1,7 @@
 // Tensor-core (tcgen05) path of the bf16 configuration: tensor maps and launch sequence.
 #include <cstdlib>
 #include <new>
+#include <utility>
 
 #include "sh_internal.cuh"
 #include "sh_simt.cuh"
@@ -82,15 +83,36 @@ struct TcState {
   int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
   // fork/join: the Q/K projection does not depend on the gate and sort kernels, so it runs on a
   // side stream between two events recorded on the caller's stream
+  bool pdl = true;
+  int pdl_mask = 31;
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 constexpr int QK_STAGES = 4;
 
+// Kernel launch, optionally with the programmatic-stream-serialization attribute: the kernel may
+// then become resident while the kernel before it in the stream is still running, and decides
+// itself (griddepcontrol.wait) when it needs that kernel's results.
+template <typename... P, typename... A>
+static int launch_k(bool pdl, void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+  SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...));
+  return SH_OK;
+}
+
 template <typename K>
 static int set_smem(K kernel, int bytes) {
   SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  // Always the largest shared-memory carve-out: kernels of one forward pass share SMs (a sort block
+  // beside a GEMM CTA; the next kernel's CTAs arriving while this one drains), and an SM set up
+  // with a smaller carve-out has to run empty before it can be set up again.
+  SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return SH_OK;
 }
 
@@ -121,6 +143,12 @@ int sh_tc_prepare(sh_layer* L) {
   const char* qv = getenv("SH_QK_VARIANT");
   S->qk_variant = qv ? atoi(qv) : (((L->dense ? 3 : 2) * d.H * d.D) % 256 == 0 ? 2 : 0);
   S->qk_bn = (S->qk_variant == 2) ? 256 : 128;
+  // Default: the kernels of the caller's stream are chained by programmatic dependent launch (each
+  // becomes resident while the one before it drains, and waits on the device for its results);
+  // the dense Q/K projection, which needs nothing from the gate and sort kernels, is launched the
+  // ordinary way on a side stream so that it runs beside them.  SH_NO_PDL=1: ordinary launches only.
+  S->pdl = !getenv("SH_NO_PDL");
+  if (const char* m = getenv("SH_PDL_MASK")) S->pdl_mask = atoi(m);   // debugging: bit 0 sort, 1 Q/K, 2 V, 3 attention, 4 O
   if (!L->dense && !getenv("SH_NO_OVERLAP")) {
     SH_CUDA_CHECK(cudaStreamCreateWithFlags(&S->side, cudaStreamNonBlocking));
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_fork, cudaEventDisableTiming));
@@ -204,13 +232,23 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   else sh_tc_gate_kernel<4><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
   const size_t ssm = sh_sort_smem_bytes(d);
   static size_t sort_cfg = 48 * 1024;
+  static bool sort_carveout = false;
+  if (!sort_carveout) {
+    // Sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow: ask for
+    // the largest shared-memory carve-out, or an SM that a sort block configured would have to
+    // drain before such a CTA could join it.
+    SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    sort_carveout = true;
+  }
   if (ssm > sort_cfg) {
     SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
     sort_cfg = ssm;
   }
-  sh_sort_kernel<<<d.nblk, sh_sort_threads(d), ssm, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
-      (const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
-      (float*)(ws + L->o.lgate), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);
+  if ((rc = launch_k(S->pdl && !L->ev && (S->pdl_mask & 1), sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(d)), ssm, st,
+                     (const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate), (const int*)(ws + L->o.blockcnt),
+                     (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists), (float*)(ws + L->o.lgate),
+                     (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d)))
+    return rc;
   L->launches += 2;
   return SH_OK;
 }
@@ -221,7 +259,7 @@ int sh_tc_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
 }
 
 template <int BN, int STAGES, int MODE, int MT>
-static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, unsigned grid, cudaStream_t st) {
+static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, unsigned grid, cudaStream_t st, bool pdl) {
   auto kern = sh_tc_pgemm_kernel<BN, STAGES, MODE, MT>;
   constexpr int smem = PGemmSmem<BN, STAGES, MT>::TOTAL;
   static bool configured = false;
@@ -230,8 +268,7 @@ static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const 
     if (rc != SH_OK) return rc;
     configured = true;
   }
-  kern<<<grid, 320, smem, st>>>(mapA, mapB, g);
-  return SH_OK;
+  return launch_k(pdl, kern, dim3(grid), dim3(320), smem, st, mapA, mapB, g);
 }
 
 template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>
@@ -257,6 +294,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   int rc;
   const int simt = S->simt_mask;
   int* status = (int*)(ws + L->o.status);
+  const bool pdl = S->pdl && !L->ev;                       // stage-timed runs use ordinary launches
 
   sh_mark(L, 0, st);
   // stage-timed runs stay serial so that the stage boundaries mean something
@@ -284,12 +322,13 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
     g.qscale = 1.4426950408889634f / sqrtf((float)d.D);
     g.status = status;
+    g.sched = status + 16;
     dim3 grid(d.nblk, (g.ncols + S->qk_bn - 1) / S->qk_bn);
     switch (S->qk_variant) {
       case 1: rc = launch_gemm<128, 3, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
       case 2: {
         const unsigned tiles = (unsigned)(d.nblk * ((g.ncols + 255) / 256));
-        rc = S->persistent ? launch_pgemm<256, 4, PG_QKV, 1>(map_x, S->map_wqk, g, tiles < (unsigned)L->sm_count ? tiles : (unsigned)L->sm_count, st)
+        rc = S->persistent ? launch_pgemm<256, 4, PG_QKV, 1>(map_x, S->map_wqk, g, tiles < (unsigned)L->sm_count ? tiles : (unsigned)L->sm_count, st, pdl && !overlap && (S->pdl_mask & 2))
                            : launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st);
         break;
       }
@@ -315,7 +354,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       // 256-row tiles (two accumulators sharing the weight operand): at most half the 128-row bound plus one per group
       dim3 grid(d.tile_rows_src == 256 ? d.max_tiles / 2 + d.H * d.E : d.max_tiles, 1);
       if (d.tile_rows_src == 256) {
-        if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 2>(map_x, S->map_wv, g, grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count, st)
+        if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 2>(map_x, S->map_wv, g, grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count, st, pdl && (S->pdl_mask & 4))
                                            : launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
         else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
       } else {
@@ -350,10 +389,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       const unsigned grid = (unsigned)(nq * d.B * d.H);
       if (d.D == 128) {
         if (!cfg2_128) { if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc; cfg2_128 = true; }
-        sh_tc_attention2_kernel<128><<<grid, 320, Attn2Smem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+        if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
       } else {
         if (!cfg2_64) { if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc; cfg2_64 = true; }
-        sh_tc_attention2_kernel<64><<<grid, 320, Attn2Smem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
+        if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<64>, dim3(grid), dim3(320), Attn2Smem<64>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
       }
     }
     L->launches += 1;
@@ -397,10 +436,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     a.a_slots = as;
     if (d.D == 128) {
       if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
-      sh_tc_oproj_kernel<128><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo256, a);
+      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<128>, dim3(grid), dim3(352), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
     } else {
       if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
-      sh_tc_oproj_kernel<64><<<grid, 352, smem, st>>>(S->map_ahat, S->map_wo256, a);
+      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<64>, dim3(grid), dim3(352), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
     }
     L->launches += 1;
   } else {

@@ -82,6 +82,8 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_trigger();                                         // programmatic dependent launch: the next kernel may become resident,
+  pdl_wait();                                            // and this one starts consuming once the kernel before it has completed
 
   if (warp == 0) {
     if (lane == 0) {
@@ -219,6 +221,11 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       // phase of the shared P buffer this write is: tile 0 step j comes after min(j, n1) writes of
       // tile 1; tile 1 step j after min(j + 1, n0) writes of tile 0
       const int phase = j + (t == 0 ? (j < other ? j : other) : (j + 1 < other ? j + 1 : other));
+      // This group's own previous P V product first: a parity wait cannot tell phase p from phase
+      // p - 2, and without this the group could reach the p_free wait below while p_free is still
+      // two phases back (the issuer queues the next S before this step's P V), pass it on the stale
+      // phase and overwrite P under a running product.
+      if (j > 0 && !mbar_wait(&pv_done[t], (j - 1) & 1, g.status, dead)) { ok = false; break; }
       if (phase > 0) {
         if (!mbar_wait(p_free, (phase - 1) & 1, g.status, dead)) { ok = false; break; }
         tc_fence_after();

@@ -63,6 +63,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
+  pdl_trigger();                                        // the sort kernel may become resident (it waits for this grid)
 
   if (warp == 0 || warp == 6) {
     if (lane == 0) {

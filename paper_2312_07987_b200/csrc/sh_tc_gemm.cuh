@@ -30,6 +30,7 @@ struct TcGemmArgs {
   void* out0; void* out1; void* out2;
   float qscale;
   int* status;
+  int* sched;            // persistent dense mode: {next tile, CTAs that made their final claim}, both 0 between launches
 };
 
 constexpr int GEMM_BM = 128;

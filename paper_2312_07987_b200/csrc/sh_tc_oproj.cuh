@@ -102,6 +102,8 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_trigger();                                         // programmatic dependent launch: the next kernel may become resident,
+  pdl_wait();                                            // and this one starts consuming once the kernel before it has completed
 
   if (warp == 0) {
     if (lane == 0) {

@@ -1,7 +1,10 @@
 // Persistent tcgen05 GEMMs for the two projections that dominate the front of the layer: the
 // dense Q/K projection (PG_QKV) and the grouped value-expert projection (PG_V).
 //
-// One CTA per SM walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The operand ring (TMA for
+// One CTA per SM walks tiles: blockIdx.x, blockIdx.x + gridDim.x, ... for the value experts; for
+// the dense projection, which starts while the gate kernel still holds part of the GPU (so its
+// CTAs start at different times), tiles are claimed one at a time from a global counter by the
+// producer thread and handed to the other roles through a small shared-memory ring.  The operand ring (TMA for
 // B and for dense A; cp.async row gathers for the value experts' A) and the two TMEM
 // accumulator buffers run on across tiles, so the ~3 us a CTA needs to set itself up and
 // the first ~0.9 us TMA round trip are paid once per SM instead of once per tile, and the
@@ -43,17 +46,21 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
   uint64_t* acc_full = empty_bar + STAGES;     // [2]
   uint64_t* acc_empty = acc_full + 2;          // [2]
   uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+  constexpr int TQ = 4;                                    // claimed-tile ring (dense mode)
+  uint64_t* tq_full = (uint64_t*)(sgen + SM::BAR_OFF + 128);
+  uint64_t* tq_empty = tq_full + TQ;
+  int* tq_tile = (int*)(tq_empty + TQ);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const ShDims& d = g.d;
   const int KB = g.K / 64;
   const int ncol = (g.ncols + BN - 1) / BN;                // column tiles (dense mode)
-  const int ntiles = GATHER ? *g.ntiles : ((g.nrows + ROWS - 1) / ROWS) * ncol;
   bool dead = false;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 129 : 2); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    for (int j = 0; j < TQ; ++j) { mbar_init(&tq_full[j], 1); mbar_init(&tq_empty[j], 130); }   // A producer + issuer + 128 epilogue threads
     fence_barrier_init();
     tma_prefetch_desc(&mapB);
     if (!GATHER) tma_prefetch_desc(&mapA);
@@ -63,6 +70,28 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // Programmatic dependent launch: the next kernel in the stream may become resident from here on.
+  // The value experts need the sorted lists (kernel before this one) now.  The dense projection
+  // reads nothing an earlier kernel of the same forward pass wrote, so it only waits at its end
+  // (which makes "this grid completed" imply "everything before it completed") -- but measured on
+  // B200, the TMA loads of a grid launched this way do not return before the grid ahead of it has
+  // completed (plain loads do), so the layer launches this projection the ordinary way on a
+  // second stream instead when it wants it to run beside the gate and sort kernels.
+  pdl_trigger();
+  if (GATHER) pdl_wait();
+  const int ntiles = GATHER ? *g.ntiles : ((g.nrows + ROWS - 1) / ROWS) * ncol;
+  // the qi-th tile of this CTA for every role but the claiming producer, or -1 when there is none
+  auto next_tile = [&](int qi) -> int {
+    if (GATHER) {
+      const int t = blockIdx.x + qi * gridDim.x;
+      return t < ntiles ? t : -1;
+    }
+    const int j = qi & (TQ - 1);
+    if (!mbar_wait(&tq_full[j], (qi / TQ) & 1, g.status, dead)) return -1;
+    const int t = tq_tile[j];
+    mbar_arrive(&tq_empty[j]);
+    return t;
+  };
 
   if (warp == 0 || (!GATHER && warp == 6)) {
     // one thread issues a TMA box only every ~150 ns, so in the dense mode the A and the B boxes
@@ -71,7 +100,24 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
       const bool do_b = warp == 0, do_a = !GATHER && warp == 6;
       int s = 0;
       uint32_t par = 1;
-      for (int t = blockIdx.x; t < ntiles && !dead; t += gridDim.x) {
+      for (int qi = 0; !dead; ++qi) {
+        int t;
+        if (!GATHER && do_b) {
+          // claim the next tile only now, when the loads of the previous one are all issued
+          const int j = qi & (TQ - 1);
+          if (!mbar_wait(&tq_empty[j], ((qi / TQ) & 1) ^ 1, g.status, dead)) break;
+          t = atomicAdd(g.sched, 1);
+          if (t >= ntiles) t = -1;
+          tq_tile[j] = t;
+          mbar_arrive(&tq_full[j]);
+          if (t < 0) {
+            // the CTA whose final claim comes last puts both counters back for the next launch
+            if (atomicAdd(g.sched + 1, 1) == (int)gridDim.x - 1) { g.sched[0] = 0; g.sched[1] = 0; }
+          }
+        } else {
+          t = next_tile(qi);
+        }
+        if (t < 0) break;
         int row0, brow;
         if (GATHER) {
           const ShTile tl = g.tiles[t];
@@ -104,7 +150,8 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
       const uint32_t a_lo0 = desc_lo_k(sbase), b_lo0 = desc_lo_k(sbase + SM::A_BYTES);
       int s = 0, it = 0;
       uint32_t par = 0;
-      for (int t = blockIdx.x; t < ntiles && !dead; t += gridDim.x, ++it) {
+      for (; !dead; ++it) {
+        if (next_tile(it) < 0) break;
         const int b = it & 1;
         if (!mbar_wait(&acc_empty[b], ((it >> 1) & 1) ^ 1, g.status, dead)) break;
         const uint32_t td = tmem + b * ACC_COLS;
@@ -133,7 +180,9 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
       const uint32_t dsw = (uint32_t)((c ^ (rb & 7)) << 4);
       int s = 0, issued = 0, n_arr = 0, s_arr = 0;
       uint32_t par = 1;
-      for (int t = blockIdx.x; t < ntiles && !dead; t += gridDim.x) {
+      for (int qi = 0; !dead; ++qi) {
+        const int t = next_tile(qi);
+        if (t < 0) break;
         const ShTile tl = g.tiles[t];
         const char* src[8 * MT];
         uint32_t ok[8 * MT];
@@ -176,7 +225,9 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     const int q = warp & 3;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     int it = 0;
-    for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+    for (;; ++it) {
+      const int t = next_tile(it);
+      if (t < 0) break;
       const int b = it & 1;
       int th = 0, row0, nrows, col0 = 0;
       if (GATHER) {
@@ -257,6 +308,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
       }
     }
   }
+  if (!GATHER) pdl_wait();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

@@ -55,7 +55,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
       if (global_timer_ns() - t0 > SH_WAIT_LIMIT_NS || *(volatile int*)status != 0) {
-        atomicCAS(status, 0, SH_ERR_TIMEOUT);
+        if (atomicCAS(status, 0, SH_ERR_TIMEOUT) == 0) {   // first give-up of the launch: say where (diagnostics)
+          status[1] = (int)blockIdx.x; status[2] = (int)threadIdx.x; status[3] = (int)smem_u32(bar);
+          status[4] = (int)parity; status[5] = (int)gridDim.x; status[6] = (int)blockDim.x;
+        }
         dead = true;
         return false;
       }
@@ -113,6 +116,15 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+// ---- programmatic dependent launch -------------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may become resident while
+// the kernel before it in the stream still runs: pdl_trigger() in the earlier kernel (once every
+// CTA has executed it or exited) lets the later one be scheduled, and pdl_wait() in the later one
+// returns only when the earlier grid has completed and its writes are visible.  Both are no-ops in
+// a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
