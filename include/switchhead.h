@@ -102,7 +102,8 @@ int sh_set_weights(sh_layer* layer, const void* Wq, const void* Wk, const void* 
 
 /* The whole forward pass (gates + top-k + bucket sort, Q/K projections, value experts,
  * causal attention, output experts with the gate-weighted sum) of x [B, T, d_model] into
- * out [B, T, d_model] fp32.  out is fully overwritten.  Enqueues kernels only. */
+ * out [B, T, d_model] fp32.  Both are device pointers aligned to 16 bytes (else
+ * SH_ERR_INVALID_ARG).  out is fully overwritten.  Enqueues kernels only. */
 int sh_forward(sh_layer* layer, const void* x, void* out, void* stream);
 
 /* Measurement aid: sh_forward with CUDA events recorded on `stream` at the stage boundaries;

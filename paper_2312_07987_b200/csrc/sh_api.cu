@@ -311,6 +311,7 @@ extern "C" int sh_forward(sh_layer* L, const void* x, void* out, void* stream) {
   int rc = check_ready(L);
   if (rc != SH_OK) return rc;
   if (!x || !out) { sh_set_error("x and out must not be NULL"); return SH_ERR_INVALID_ARG; }
+  if ((uintptr_t)x % 16 != 0 || (uintptr_t)out % 16 != 0) { sh_set_error("x and out must be 16-byte aligned"); return SH_ERR_INVALID_ARG; }
   cudaStream_t st = (cudaStream_t)stream;
   L->launches = 0;
   if (L->dtype == SH_F32) return forward_simt<float, float>(L, SH_STAGE_ALL, x, out, st);

@@ -436,10 +436,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     a.a_slots = as;
     if (d.D == 128) {
       if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
-      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<128>, dim3(grid), dim3(352), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
+      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<128>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
     } else {
       if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
-      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<64>, dim3(grid), dim3(352), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
+      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<64>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
     }
     L->launches += 1;
   } else {

@@ -19,9 +19,8 @@
 // halves the token-tile traffic; the accumulators (128 tokens x 256 features fp32) just fit
 // the registers of 256 epilogue threads.
 //
-// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer (warp 10
-// can issue the odd experts when built with OPROJ_ISSUERS = 2; measured: no gain),
-// warps 2..9 = epilogue (thread = one token = TMEM lane, and one half of the 256 features;
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer (a second
+// issuing thread for the odd experts was tried: no gain), warps 2..9 = epilogue (thread = one token = TMEM lane, and one half of the 256 features;
 // two warps share a lane quarter).  One expert = one 256-column TMEM buffer (ring of 2); its
 // weights arrive as D/64 stages of 256 features x 64 columns (32 KB, one TMA box each) through
 // a ring of 3 (or 2) stages that are released one by one: L2 answers a TMA load after ~0.9 us,
@@ -32,10 +31,6 @@
 #include "sh_tc_prims.cuh"
 
 namespace shtc {
-
-#ifndef OPROJ_ISSUERS
-#define OPROJ_ISSUERS 1          // UMMA-issuing threads (2: even / odd experts)
-#endif
 
 struct TcOprojArgs {
   ShDims d;
@@ -58,11 +53,10 @@ struct OprojSmem {
 };
 
 template <int D>
-__global__ void __launch_bounds__(352, 1)
+__global__ void __launch_bounds__(320, 1)
 sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g) {
   using SM = OprojSmem<D>;
   constexpr int DB = D / 64;
-  constexpr int N_ISS = OPROJ_ISSUERS;
   constexpr uint32_t TBLK = 128 * 128;                   // one 64-column block of the token tile
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -90,8 +84,8 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   if (threadIdx.x == 0) {
     for (int s = 0; s < 4; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], N_ISS);
-      mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 256);
+      mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1);
+      mbar_init(&d_full[s], 1); mbar_init(&d_empty[s], 8);
     }
     mbar_init(sel_free, 256); mbar_init(sel_ready, 256);
     fence_barrier_init();
@@ -131,9 +125,8 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
         }
       }
     }
-  } else if (warp == 1 || warp == 10) {
-    if (lane == 0 && (warp == 1 || N_ISS == 2)) {
-      const int iss = warp == 1 ? 0 : 1;                    // this issuer takes the experts with ge % N_ISS == iss
+  } else if (warp == 1) {
+    if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_f16(128, 256, 0, 0, 0);
       const uint32_t w_lo0 = desc_lo_k(sbase + a_off), t_lo0 = desc_lo_k(sbase + b_off);
       int gh = 0, ge = 0, s = 0;
@@ -145,24 +138,19 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
           const uint32_t t_lo = t_lo0 + bs * (SM::B_BYTES >> 4);
           for (int e = 0; e < d.E && !dead; ++e, ++ge) {
             const int buf = ge & 1;
-            const bool mine = N_ISS == 1 || buf == iss;
-            if (mine && !mbar_wait(&d_empty[buf], ((ge >> 1) & 1) ^ 1, g.status, dead)) break;
+            if (!mbar_wait(&d_empty[buf], ((ge >> 1) & 1) ^ 1, g.status, dead)) break;
             for (int c = 0; c < DB; ++c) {
-              // every issuer observes every phase of the ring (a parity wait cannot skip one);
-              // the expert's owner issues the UMMAs and hands the stage back
               if (!mbar_wait(&a_full[s], apar, g.status, dead)) break;
-              if (mine) {
-                tc_fence_after();
-                const uint32_t w_lo = w_lo0 + s * (SM::A_BYTES >> 4), tc_lo = t_lo + c * (TBLK >> 4);
+              tc_fence_after();
+              const uint32_t w_lo = w_lo0 + s * (SM::A_BYTES >> 4), tc_lo = t_lo + c * (TBLK >> 4);
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                  umma_f16(tmem + buf * 256, desc_pack(tc_lo + 2 * k), desc_pack(w_lo + 2 * k), idesc, (c | k) != 0);
-                umma_commit(&a_empty[s]);                   // this stage can load its next box
-              }
+              for (int k = 0; k < 4; ++k)
+                umma_f16(tmem + buf * 256, desc_pack(tc_lo + 2 * k), desc_pack(w_lo + 2 * k), idesc, (c | k) != 0);
+              umma_commit(&a_empty[s]);                     // this stage can load its next box
               if (++s == AS) { s = 0; apar ^= 1; }
             }
             if (dead) break;
-            if (mine) umma_commit(&d_full[buf]);
+            umma_commit(&d_full[buf]);
           }
           umma_commit(&b_empty[bs]);
         }
@@ -218,7 +206,8 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
             tmem_ld_wait();
             if (c == 3) {                                    // everything is in registers: hand the buffer back
               tc_fence_before();
-              mbar_arrive(&d_empty[buf]);
+              __syncwarp();                                  // one arrival per warp: 256 arrivals on one barrier
+              if (lane == 0) mbar_arrive(&d_empty[buf]);     // word would serialise in the LSU
             }
 #pragma unroll
             for (int f = 0; f < 32; ++f) acc[c * 32 + f] = fmaf(gv, __uint_as_float(v[f]), acc[c * 32 + f]);
@@ -240,8 +229,14 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
             *reinterpret_cast<float4*>(stg + lane * 32 + ((ch ^ (lane & 7)) << 2)) =
                 make_float4(acc[c * 32 + 4 * ch], acc[c * 32 + 4 * ch + 1], acc[c * 32 + 4 * ch + 2], acc[c * 32 + 4 * ch + 3]);
           __syncwarp();
-          for (int r = 0; r < rows_here; ++r)
-            obase[(size_t)r * d.M + c * 32 + lane] = stg[r * 32 + ((((lane >> 2) ^ (r & 7)) << 2) | (lane & 3))];
+          // 8 lanes cover one row's 128 bytes, a warp instruction four rows
+#pragma unroll
+          for (int r4 = 0; r4 < 32; r4 += 4) {
+            const int r = r4 + (lane >> 3), ch = lane & 7;
+            if (r < rows_here)
+              *reinterpret_cast<float4*>(obase + (size_t)r * d.M + c * 32 + 4 * ch) =
+                  *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2));
+          }
         }
       }
     }
