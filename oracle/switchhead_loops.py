@@ -12,6 +12,7 @@ with V^h[s] = sum_{e in E_S^h(s)} sigmoid(z_S^h[s,e]) * x[s] W_V^{h,e}  and
 """
 from __future__ import annotations
 
+import cmath
 import math
 
 
@@ -47,7 +48,18 @@ def _vecmat(v, W):
     return out
 
 
-def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=None, causal=True):
+def _rope_complex(vec, pos, base):
+    """Rotary embedding written with complex numbers: the pair (v[2i], v[2i+1]) is one complex
+    number, multiplied by exp(i * pos * base**(-2i/D)) (RoFormer's formulation)."""
+    D = len(vec)
+    out = [0.0] * D
+    for i in range(D // 2):
+        z = complex(vec[2 * i], vec[2 * i + 1]) * cmath.exp(1j * pos * base ** (-2.0 * i / D))
+        out[2 * i], out[2 * i + 1] = z.real, z.imag
+    return out
+
+
+def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=None, causal=True, rope_base=None):
     """Nested lists or arrays in, nested list y [B][T][M] out."""
     x = [[list(map(float, tok)) for tok in seq] for seq in x]
     B, T, M = len(x), len(x[0]), len(x[0][0])
@@ -63,8 +75,11 @@ def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=N
             Q, K, V, selD = [], [], [], []
             for t in range(T):
                 xt = x[b][t]
-                Q.append(_vecmat(xt, Wq[h]))
-                K.append(_vecmat(xt, Wk[h]))
+                q_t, k_t = _vecmat(xt, Wq[h]), _vecmat(xt, Wk[h])
+                if rope_base is not None:
+                    q_t, k_t = _rope_complex(q_t, t, rope_base), _rope_complex(k_t, t, rope_base)
+                Q.append(q_t)
+                K.append(k_t)
                 zs = _vecmat(xt, Ws[h])
                 zd = _vecmat(xt, Wd[h])
                 if bias_s is not None:

@@ -16,6 +16,10 @@ What it computes, following the paper's Sec. 2.2 ("From Dense to SwitchHead"):
   output                  y = sum_h sum_{e in E_D^h} s_D^h[e] A^h V^h W_O^{h,e}
                                                               (the MoE output equation)
 
+Optional (off by default): rotary position embeddings on Q and K (the paper's appendix on
+RoPE positional encodings: square causal attention, no cache), pairs (2i, 2i+1), angle
+p * base**(-2i/d_head).
+
 Readings where the paper is silent (each is listed in the design notes):
   * top-k is taken on the pre-sigmoid logits (sigmoid is strictly increasing, so the set
     is the same in exact arithmetic); ties go to the lower expert index; -0.0 == +0.0.
@@ -100,14 +104,40 @@ def bucket_lists(idx: np.ndarray, n_experts: int):
     return offsets, lists
 
 
+def rope_rotate(a: np.ndarray, positions: np.ndarray, base: float) -> np.ndarray:
+    """Rotary position embedding (the RoPE variant of the paper's appendix "RoPE Positional
+    Encodings", which takes it from RoFormer): feature pairs (2i, 2i+1) of the vector at
+    position p are rotated by the angle p * base**(-2i/D).
+
+    a [..., T, D] (D even), positions [T].  Written out pair by pair:
+      a'[2i]   = a[2i] cos(p theta_i) - a[2i+1] sin(p theta_i)
+      a'[2i+1] = a[2i] sin(p theta_i) + a[2i+1] cos(p theta_i)."""
+    a = np.asarray(a, dtype=np.float64)
+    D = a.shape[-1]
+    if D % 2:
+        raise ValueError("rotary embedding needs an even d_head")
+    i = np.arange(D // 2, dtype=np.float64)
+    theta = np.power(float(base), -2.0 * i / D)                       # [D/2]
+    ang = np.asarray(positions, dtype=np.float64)[:, None] * theta[None, :]   # [T, D/2]
+    c, s_ = np.cos(ang), np.sin(ang)
+    out = np.empty_like(a)
+    out[..., 0::2] = a[..., 0::2] * c - a[..., 1::2] * s_
+    out[..., 1::2] = a[..., 0::2] * s_ + a[..., 1::2] * c
+    return out
+
+
 def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=None,
                        causal: bool = True, gate_override: Optional[float] = None,
-                       return_stages: bool = True):
+                       return_stages: bool = True, rope_base: Optional[float] = None,
+                       rope_offset: int = 0):
     """Forward pass of one SwitchHead layer in fp64.
 
     x [B, T, M]; Wq, Wk [H, M, D]; Wv [H, E, M, D]; Wo [H, E, D, M]; Ws, Wd [H, M, E].
     gate_override: if given, every selected expert's gate is replaced by this constant
     (used only to pin the E=1 case to plain multi-head attention).
+    rope_base: if given, queries and keys are rotated by rotary position embeddings with
+    this base before the attention scores (token t of a sequence sits at position
+    rope_offset + t; no cache, square attention); None = no positional encoding.
     Returns a dict with y [B, T, M] and, if return_stages, the intermediate stages."""
     f = lambda a: None if a is None else np.asarray(a, dtype=np.float64)
     x, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d = map(f, (x, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d))
@@ -134,6 +164,14 @@ def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=No
                 rows = np.nonzero(idxS[:, h, j] == e)[0]
                 if rows.size:
                     V[rows, h, :] += gateS[rows, h, j][:, None] * (x2d[rows] @ Wv[h, e])
+
+    if rope_base is not None:
+        pos = rope_offset + np.arange(T)
+        # [N, H, D] -> [B, H, T, D] so that the position axis sits next to the feature axis
+        to_bhtd = lambda a: a.reshape(B, T, H, D).transpose(0, 2, 1, 3)
+        back = lambda a: a.transpose(0, 2, 1, 3).reshape(N, H, D)
+        Q = back(rope_rotate(to_bhtd(Q), pos, rope_base))
+        K = back(rope_rotate(to_bhtd(K), pos, rope_base))
 
     Ahat = np.empty((N, H, D))
     scale = 1.0 / np.sqrt(D)

@@ -305,3 +305,55 @@ def test_mac_formulas_reproduce_printed_table():
     assert round(100 * r) == 44 and round(100 * m) == 27
     # the printed SwitchHead equation exceeds the tabulated value (documented erratum)
     assert mac_count.switchhead_macs_printed(4, 512, 112, 1024, 2) > 2.45e9
+
+
+# ---- rotary position embeddings (appendix "RoPE Positional Encodings") --------------------
+def test_rope_closed_form_two_dimensions():
+    """d_head = 2 has a single pair and theta_0 = 1: position p rotates (1, 0) to
+    (cos p, sin p) and (0, 1) to (-sin p, cos p), whatever the base."""
+    from oracle.switchhead_oracle import rope_rotate
+    pos = np.array([0, 1, 2, 7])
+    e0 = rope_rotate(np.tile([1.0, 0.0], (4, 1)), pos, 10000.0)
+    e1 = rope_rotate(np.tile([0.0, 1.0], (4, 1)), pos, 123.0)
+    assert np.allclose(e0, np.stack([np.cos(pos), np.sin(pos)], -1), atol=1e-15)
+    assert np.allclose(e1, np.stack([-np.sin(pos), np.cos(pos)], -1), atol=1e-15)
+
+
+def test_rope_angles_norms_and_relative_position():
+    from oracle.switchhead_oracle import rope_rotate
+    rng = np.random.default_rng(5)
+    D, T, base = 8, 11, 10000.0
+    a, b = rng.standard_normal((T, D)), rng.standard_normal((T, D))
+    pos = np.arange(T)
+    ra, rb = rope_rotate(a, pos, base), rope_rotate(b, pos, base)
+    # position 0 is the identity; every pair keeps its norm
+    assert np.array_equal(ra[0], a[0])
+    assert np.allclose(ra[:, 0::2] ** 2 + ra[:, 1::2] ** 2, a[:, 0::2] ** 2 + a[:, 1::2] ** 2, rtol=1e-13)
+    # pair i of the vector at position p is turned by p * base**(-2i/D): check the angle itself
+    for i in range(D // 2):
+        got = np.arctan2(ra[3, 2 * i + 1], ra[3, 2 * i]) - np.arctan2(a[3, 2 * i + 1], a[3, 2 * i])
+        want = 3 * base ** (-2.0 * i / D)
+        assert abs((got - want + np.pi) % (2 * np.pi) - np.pi) < 1e-12
+    # scores depend on the two positions only through their difference
+    s1 = rope_rotate(a, pos, base) @ rope_rotate(b, pos, base).T
+    s2 = rope_rotate(a, pos + 37, base) @ rope_rotate(b, pos + 37, base).T
+    assert np.allclose(s1, s2, rtol=1e-10, atol=1e-12)
+    # and differ from the unrotated scores off the diagonal, agree on it
+    s0 = a @ b.T
+    assert np.allclose(np.diag(s1), np.diag(s0), rtol=1e-12)
+    assert not np.allclose(s1, s0)
+
+
+def test_rope_layer_is_shift_invariant_and_matches_the_complex_form():
+    rng = np.random.default_rng(77)
+    L = rand_layer(rng, 2, 9, 8, 2, 4, 3)
+    y0 = switchhead_forward(**L, k=2, rope_base=10000.0)
+    y1 = switchhead_forward(**L, k=2, rope_base=10000.0, rope_offset=1000)
+    assert np.allclose(y0["y"], y1["y"], rtol=1e-9, atol=1e-11)          # only relative positions matter
+    assert not np.allclose(y0["y"], switchhead_forward(**L, k=2)["y"])     # and it is not a no-op
+    assert np.array_equal(y0["V"], switchhead_forward(**L, k=2)["V"])      # values are not rotated
+    yl = np.array(switchhead_forward_loops(**L, k=2, rope_base=10000.0))   # complex-number writing
+    assert np.allclose(y0["y"], yl, rtol=1e-11, atol=1e-12)
+    # a single token sits at position 0: rotary embedding changes nothing
+    L1 = rand_layer(rng, 3, 1, 8, 2, 4, 3)
+    assert np.array_equal(switchhead_forward(**L1, k=2, rope_base=10000.0)["y"], switchhead_forward(**L1, k=2)["y"])
