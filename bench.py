@@ -87,7 +87,7 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(cfg, inp, seconds_budget=12.0):
+def oracle_sample(cfg, inp, seconds_budget=12.0, rope_base=None):
     """Times the oracle, as it stands, on whole sequences of the workload (batch elements are
     independent), cycling through the batch until about `seconds_budget` seconds are spent."""
     from oracle.switchhead_oracle import switchhead_forward
@@ -100,7 +100,7 @@ def oracle_sample(cfg, inp, seconds_budget=12.0):
         nb = min(nb, B - lo)
         t1 = time.perf_counter()
         switchhead_forward(inp.x[lo:lo + nb], inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, cfg.k,
-                           inp.bias_s, inp.bias_d, return_stages=False)
+                           inp.bias_s, inp.bias_d, return_stages=False, rope_base=rope_base)
         dt = time.perf_counter() - t1
         done += nb
         t_used = time.perf_counter() - t0
@@ -122,7 +122,8 @@ def run_reference(args, rank, world):
     inp = inputs.make_inputs(cfg, batch=sample_b)
     from oracle.switchhead_oracle import switchhead_forward
     run = lambda: switchhead_forward(inp.x, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, cfg.k,
-                                     inp.bias_s, inp.bias_d, return_stages=False)
+                                     inp.bias_s, inp.bias_d, return_stages=False,
+                                     rope_base=args.rope if args.rope > 0 else None)
     for _ in range(min(args.warmup, 1)):
         run()
     t0 = time.perf_counter()
@@ -153,6 +154,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--rope", type=float, default=0.0,
+                    help="rotary position embeddings on Q, K with this base (0 = off, the headline configuration)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -178,6 +181,8 @@ def main():
     inp = inputs.make_inputs(cfg)
     inp.x = sharding.rank_batch(inp.x, rank)                                 # rows keep their gate margins
     layer = binding.layer_from_inputs(inp)
+    if args.rope > 0:
+        layer.sh_set_rope(args.rope)
     x = binding.to_device(inp.x, cfg.dtype)
     out = torch.empty(inp.x.shape, dtype=torch.float32, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # > 126 MB L2
@@ -276,7 +281,8 @@ def main():
             "data": "synthetic",
             "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "seq_len": cfg.seq, "d_model": cfg.d_model,
                        "n_heads": cfg.n_heads, "d_head": cfg.d_head, "n_experts": cfg.n_experts, "k": cfg.k,
-                       "causal": True, "l2": "flushed before every timed step (256 MiB write)",
+                       "causal": True, "rope_base": args.rope if args.rope > 0 else None,
+                       "l2": "flushed before every timed step (256 MiB write)",
                        "parallelism": f"batch-sharded replicas x{world}, no collective"},
             "useful_tflops": useful_tflops,
             "frac_of_bf16_peak_measured": useful_tflops / (world * peaks["tflops"]),
@@ -315,7 +321,7 @@ def main():
                                        "useful_tflops": dense_flop / (dms * 1e-3) / 1e12}
             dl.close()
         if not args.no_cpu_baseline:
-            v, nseq, secs = oracle_sample(cfg, inp)
+            v, nseq, secs = oracle_sample(cfg, inp, rope_base=args.rope if args.rope > 0 else None)
             line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)),
                                     "kind": "oracle",
                                     "sample": f"{nseq} sequences of {cfg.seq} tokens drawn from the workload's {cfg.batch}, {secs:.1f} s, fp64 numpy"}

@@ -100,6 +100,17 @@ int sh_set_weights(sh_layer* layer, const void* Wq, const void* Wk, const void* 
                    const void* Wo, const void* Ws, const void* Wd, const float* bias_s,
                    const float* bias_d, void* stream);
 
+/* Rotary position embeddings on the queries and keys (the paper's appendix "RoPE Positional
+ * Encodings": square causal attention without a cache, RoPE as in RoFormer).  Token t of a
+ * sequence sits at position t; the feature pair (2i, 2i+1) of its query and key vectors of
+ * every head is rotated by the angle t * base^(-2i/d_head) before the attention scores are
+ * taken; values are not rotated.  base > 0 switches it on (10000 is RoFormer's value) and
+ * writes the (cos, sin) table for the configured sequence length into the workspace,
+ * asynchronously on `stream`; base == 0 switches it off (the default, and the state after
+ * every sh_configure and sh_set_workspace).  Needs a configured layer with its workspace (else
+ * SH_ERR_NOT_CONFIGURED) and an even d_head. */
+int sh_set_rope(sh_layer* layer, double base, void* stream);
+
 /* The whole forward pass (gates + top-k + bucket sort, Q/K projections, value experts,
  * causal attention, output experts with the gate-weighted sum) of x [B, T, d_model] into
  * out [B, T, d_model] fp32.  Both are device pointers aligned to 16 bytes (else

@@ -64,6 +64,7 @@ static void layout_workspace(sh_layer* L) {
   o.lgate = take(slots * 4);
   o.tiles = take((size_t)2 * d.max_tiles * sizeof(ShTile));
   o.ntiles = take(256);
+  o.rope = take((size_t)d.T * (d.D / 2) * 8);     // (cos, sin) per feature pair and position
   o.total = off;
 }
 
@@ -110,7 +111,8 @@ extern "C" int sh_configure(sh_layer* L, int dtype, int batch, int seq) {
   L->d.nblk = (L->d.N + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
   L->d.max_tiles = (int)((slots + SH_TILE_ROWS - 1) / SH_TILE_ROWS) + d0.H * d0.E;
   L->d.tile_rows_src = SH_TILE_ROWS;
-  L->ws = nullptr; L->ws_bytes = 0; L->weights_set = false;
+  L->ws = nullptr; L->ws_bytes = 0; L->rope = false;
+  L->weights_set = false;
   sh_tc_release(L);
   layout_workspace(L);
   return SH_OK;
@@ -128,7 +130,7 @@ extern "C" int sh_set_workspace(sh_layer* L, void* workspace, size_t bytes) {
   if (!workspace) { sh_set_error("workspace is NULL"); return SH_ERR_WORKSPACE; }
   if ((uintptr_t)workspace % 256 != 0) { sh_set_error("workspace must be 256-byte aligned"); return SH_ERR_WORKSPACE; }
   if (bytes < L->o.total) { sh_set_error("workspace too small: %zu bytes given, %zu needed", bytes, L->o.total); return SH_ERR_WORKSPACE; }
-  L->ws = (char*)workspace; L->ws_bytes = bytes; L->weights_set = false;
+  L->ws = (char*)workspace; L->ws_bytes = bytes; L->weights_set = false; L->rope = false;
   sh_tc_release(L);
   return SH_OK;
 }
@@ -252,6 +254,7 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   g.A = x; g.lda = d.M; g.Bt = ws + L->o.wqk; g.ldb = d.M; g.K = d.M;
   g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
   g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v; g.qscale = qscale;
+  g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
   dim3 grid_qk(d.nblk, (g.ncols + 63) / 64);
   sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_qk, 256, 0, st>>>(g);
   L->launches += 1;
@@ -304,6 +307,34 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
 
 int sh_simt_run_bf16(sh_layer* L, int stages, const void* x, void* out, cudaStream_t st) {
   return forward_simt<__nv_bfloat16, __half>(L, stages, x, out, st);
+}
+
+// (cos, sin)(t * base^(-2i/D)) for every feature pair i < D/2 and position t < T, computed in
+// double precision, stored as float2 [D/2][T] (positions contiguous: the epilogue threads of a
+// warp hold consecutive tokens and read one pair at a time).
+static __global__ void sh_rope_table_kernel(float2* table, int T, int D, double base) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int half = D / 2;
+  if (idx >= T * half) return;
+  const int t = idx / half, i = idx % half;
+  const double ang = (double)t * pow(base, -2.0 * (double)i / (double)D);
+  double s, c;
+  sincos(ang, &s, &c);
+  table[(size_t)i * T + t] = make_float2((float)c, (float)s);
+}
+
+extern "C" int sh_set_rope(sh_layer* L, double base, void* stream) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0 || !L->ws) { sh_set_error("sh_set_rope needs a configured layer with its workspace"); return SH_ERR_NOT_CONFIGURED; }
+  if (!(base >= 0.0) || base != base) { sh_set_error("rotary base must be positive (0 switches it off), got %g", base); return SH_ERR_INVALID_ARG; }
+  if (base == 0.0) { L->rope = false; return SH_OK; }
+  if (L->d.D % 2) { sh_set_error("rotary embedding needs an even d_head"); return SH_ERR_UNSUPPORTED; }
+  const int n = L->d.T * (L->d.D / 2);
+  sh_rope_table_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>((float2*)(L->ws + L->o.rope), L->d.T, L->d.D, base);
+  SH_CUDA_CHECK(cudaGetLastError());
+  L->rope = true;
+  return SH_OK;
 }
 
 extern "C" int sh_forward(sh_layer* L, const void* x, void* out, void* stream) {

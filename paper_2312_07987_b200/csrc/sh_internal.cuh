@@ -26,7 +26,7 @@ struct ShDims {
 // Workspace sub-buffers (byte offsets from the workspace base).
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, total;
+         offsets, lists, lgate, tiles, ntiles, rope, total;
 };
 
 struct sh_layer {
@@ -37,6 +37,7 @@ struct sh_layer {
   size_t ws_bytes = 0;
   ShWorkspace o{};
   bool weights_set = false;
+  bool rope = false;       // rotary position embeddings on Q, K (table in the workspace)
   int launches = 0;
   int sm_count = 0;
   void* tc = nullptr;      // tensor-core path state (tensor maps), owned by the layer

@@ -272,6 +272,7 @@ struct ShGemmArgs {
   int a_head_stride;                // grouped O: column offset of head h inside an A row
   void* out0; void* out1; void* out2;
   float qscale;
+  const float2* rope;               // QKV epilogue: (cos, sin) table [D/2, T] of the rotary embedding, or nullptr
   ShDims d;
 };
 
@@ -362,12 +363,18 @@ sh_simt_gemm_kernel(ShGemmArgs g) {
     for (int j = 0; j < 4; ++j) {
       const int n = col0 + tc * 4 + j;
       if (n >= g.ncols) continue;
-      const float v = acc[i][j];
+      float v = acc[i][j];
       if (EPI == SH_EPI_QKV) {
         // column n -> (which, head, dd); row gr -> (b, t); target layout [B, H, T, D]
         const int HD = d.H * d.D;
         const int which = n / HD, hh = (n % HD) / d.D, dd = n % d.D;
         const int b = gr / d.T, t = gr % d.T;
+        if (g.rope && which < 2) {
+          // rotary embedding: the pair (dd even, dd + 1) sits in acc[i][j even], acc[i][j + 1]
+          const float2 cs = g.rope[(size_t)(dd >> 1) * d.T + t];
+          const float a0 = acc[i][j & ~1], a1 = acc[i][j | 1];
+          v = (j & 1) ? a0 * cs.y + a1 * cs.x : a0 * cs.x - a1 * cs.y;
+        }
         TC* dst = (TC*)(which == 0 ? g.out0 : which == 1 ? g.out1 : g.out2);
         dst[(((size_t)b * d.H + hh) * d.T + t) * d.D + dd] = sh_from_float<TC>(which == 0 ? v * g.qscale : v);
       } else if (EPI == SH_EPI_V) {

@@ -323,6 +323,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     g.qscale = 1.4426950408889634f / sqrtf((float)d.D);
     g.status = status;
     g.sched = status + 16;
+    g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
     dim3 grid(d.nblk, (g.ncols + S->qk_bn - 1) / S->qk_bn);
     switch (S->qk_variant) {
       case 1: rc = launch_gemm<128, 3, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;

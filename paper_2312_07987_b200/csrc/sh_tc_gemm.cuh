@@ -29,9 +29,22 @@ struct TcGemmArgs {
   int b_rows_per_group;  // rows of the B tensor map per (h*E + e)
   void* out0; void* out1; void* out2;
   float qscale;
+  const float2* rope;    // dense Q/K mode: (cos, sin) table [D/2, T] of the rotary embedding, or nullptr
   int* status;
   int* sched;            // persistent dense mode: {next tile, CTAs that made their final claim}, both 0 between launches
 };
+
+// Rotary embedding of the 16 adjacent feature pairs held in v[0..31] (fp32 bit patterns): pair i of
+// the chunk is pair pair0 + i of its head; cs = the (cos, sin) table [D/2][T] at the token's position.
+__device__ __forceinline__ void rope_pairs16(uint32_t* v, const float2* cs, int pair0, int T) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float2 c = cs[(size_t)(pair0 + i) * T];
+    const float a0 = __uint_as_float(v[2 * i]), a1 = __uint_as_float(v[2 * i + 1]);
+    v[2 * i] = __float_as_uint(a0 * c.x - a1 * c.y);
+    v[2 * i + 1] = __float_as_uint(a0 * c.y + a1 * c.x);
+  }
+}
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
@@ -212,6 +225,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
           __half* dst = (__half*)(which == 0 ? g.out0 : which == 1 ? g.out1 : g.out2) +
                         (((size_t)bb * d.H + hh) * d.T + tt) * d.D + dd;
           const float sc = which == 0 ? g.qscale : 1.f;
+          if (g.rope && which < 2) rope_pairs16(v, g.rope + tt, dd >> 1, d.T);
           uint32_t p[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {

@@ -274,7 +274,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
 #pragma unroll
           for (int hh2 = 0; hh2 < 2; ++hh2) {
             const int c0 = c00 + hh2 * 32;
-            const uint32_t* v = &vv[hh2 * 32];
+            uint32_t* v = &vv[hh2 * 32];
             const int n0 = col0 + c0;
             if (!live || n0 >= g.ncols) continue;
             uint32_t p[16];
@@ -284,6 +284,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
               __half* dst = (__half*)(which == 0 ? g.out0 : which == 1 ? g.out1 : g.out2) +
                             (((size_t)bb * d.H + hd) * d.T + tt) * d.D + dd;
               const float sc = which == 0 ? g.qscale : 1.f;
+              if (g.rope && which < 2) rope_pairs16(v, g.rope + tt, dd >> 1, d.T);
 #pragma unroll
               for (int i = 0; i < 16; ++i) {
                 __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * sc, __uint_as_float(v[2 * i + 1]) * sc);

@@ -11,10 +11,10 @@ from paper_2312_07987_b200 import binding, inputs
 TOL_Y = {inputs.DTYPE_F32: 1e-4, inputs.DTYPE_BF16: 2e-2}
 
 
-def oracle_for(inp, batches=None):
+def oracle_for(inp, batches=None, rope_base=None):
     x = inp.x if batches is None else inp.x[batches]
     return switchhead_forward(x, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, inp.cfg.k,
-                              inp.bias_s, inp.bias_d)
+                              inp.bias_s, inp.bias_d, rope_base=rope_base)
 
 
 def rel_rms_err(got, ref):

@@ -135,3 +135,42 @@ def test_dense_comparator_matches_dense_mha_oracle():
         assert L.sh_last_status() == 0
         assert pu.rel_rms_err(y, ref) < tol
         L.close()
+
+
+# ---- rotary position embeddings on Q and K (sh_set_rope) ------------------------------------
+def rope_check(inp, base=10000.0, batches=None):
+    cfg = inp.cfg
+    layer, x, y_plain = pu.run_layer(inp)
+    layer.sh_set_rope(base)
+    y = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0
+    ref = pu.oracle_for(inp, batches, rope_base=base)
+    pu.check_stages(layer, ref, cfg, batches)                # Q and K are compared after the rotation
+    yb = y.cpu().numpy() if batches is None else y.cpu().numpy()[batches]
+    err = pu.rel_rms_err(yb, ref["y"])
+    assert err < pu.TOL_Y[cfg.dtype], f"output max-abs error / rms = {err:.3e}"
+    if inp.x.shape[1] > 1:
+        assert not torch.equal(y, y_plain), "the rotation changed nothing"
+    layer.sh_set_rope(0.0)                                   # off again: the plain layer
+    y_off = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    # (not bit for bit: the k-way V sums are atomic / vector reductions in arrival order)
+    assert pu.rel_rms_err(y_off.cpu().numpy(), y_plain.cpu().numpy()) < (1e-5 if cfg.dtype == inputs.DTYPE_F32 else 1e-2)
+    layer.close()
+
+
+def test_rope_tiny_f32_and_edge_shapes():
+    rope_check(inputs.make_inputs(inputs.CONFIGS["tiny_f32"]))
+    rope_check(inputs.make_inputs(inputs.LayerConfig("rope_f32", inputs.DTYPE_F32, 2, 129, 192, 3, 64, 3, 2, seed=31)), base=500.0)
+    rope_check(inputs.make_inputs(inputs.LayerConfig("rope_f32_t1", inputs.DTYPE_F32, 3, 1, 64, 1, 32, 2, 1, seed=32)))
+
+
+def test_rope_bf16_configs():
+    rope_check(inputs.make_inputs(inputs.CONFIGS["small_bf16"]))                       # non-persistent 128-column Q/K tiles
+    rope_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=4))            # persistent Q/K GEMM
+    rope_check(inputs.make_inputs(inputs.LayerConfig("rope_bf16", inputs.DTYPE_BF16, 1, 515, 256, 3, 128, 4, 2, seed=33)))
+
+
+def test_rope_long_context_sampled_sequence():
+    rope_check(inputs.make_inputs(inputs.CONFIGS["long_ctx_bf16"]), batches=[2])       # positions up to 4095
