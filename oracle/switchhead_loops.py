@@ -59,7 +59,7 @@ def _rope_complex(vec, pos, base):
     return out
 
 
-def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=None, causal=True, rope_base=None):
+def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=None, causal=True, rope_base=None, shared_selection=False):
     """Nested lists or arrays in, nested list y [B][T][M] out."""
     x = [[list(map(float, tok)) for tok in seq] for seq in x]
     B, T, M = len(x), len(x[0]), len(x[0][0])
@@ -81,11 +81,12 @@ def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=N
                 Q.append(q_t)
                 K.append(k_t)
                 zs = _vecmat(xt, Ws[h])
-                zd = _vecmat(xt, Wd[h])
+                zd = _vecmat(xt, Ws[h] if shared_selection else Wd[h])
                 if bias_s is not None:
                     zs = [a + c for a, c in zip(zs, bias_s[h])]
-                if bias_d is not None:
-                    zd = [a + c for a, c in zip(zd, bias_d[h])]
+                bd = bias_s if shared_selection else bias_d
+                if bd is not None:
+                    zd = [a + c for a, c in zip(zd, bd[h])]
                 v = [0.0] * D
                 for e in _select(zs, k):
                     g = _sigmoid(zs[e])

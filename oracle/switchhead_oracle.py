@@ -129,12 +129,15 @@ def rope_rotate(a: np.ndarray, positions: np.ndarray, base: float) -> np.ndarray
 def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=None,
                        causal: bool = True, gate_override: Optional[float] = None,
                        return_stages: bool = True, rope_base: Optional[float] = None,
-                       rope_offset: int = 0):
+                       rope_offset: int = 0, shared_selection: bool = False):
     """Forward pass of one SwitchHead layer in fp64.
 
     x [B, T, M]; Wq, Wk [H, M, D]; Wv [H, E, M, D]; Wo [H, E, D, M]; Ws, Wd [H, M, E].
     gate_override: if given, every selected expert's gate is replaced by this constant
     (used only to pin the E=1 case to plain multi-head attention).
+    shared_selection: the "Shared Selection" variant of the paper's appendix: one gate serves
+    both sides, i.e. the destination side uses the source side's selection and scores
+    (Wd and bias_d are ignored).
     rope_base: if given, queries and keys are rotated by rotary position embeddings with
     this base before the attention scores (token t of a sequence sits at position
     rope_offset + t; no cache, square attention); None = no positional encoding.
@@ -147,7 +150,10 @@ def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=No
     x2d = x.reshape(N, M)
 
     zS, sS, idxS, gateS = gate_and_select(x2d, Ws, bias_s, k)
-    zD, sD, idxD, gateD = gate_and_select(x2d, Wd, bias_d, k)
+    if shared_selection:
+        zD, sD, idxD, gateD = zS, sS, idxS, gateS
+    else:
+        zD, sD, idxD, gateD = gate_and_select(x2d, Wd, bias_d, k)
     if gate_override is not None:
         gateS = np.full_like(gateS, gate_override)
         gateD = np.full_like(gateD, gate_override)

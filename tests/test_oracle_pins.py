@@ -357,3 +357,24 @@ def test_rope_layer_is_shift_invariant_and_matches_the_complex_form():
     # a single token sits at position 0: rotary embedding changes nothing
     L1 = rand_layer(rng, 3, 1, 8, 2, 4, 3)
     assert np.array_equal(switchhead_forward(**L1, k=2, rope_base=10000.0)["y"], switchhead_forward(**L1, k=2)["y"])
+
+
+# ---- shared selection (appendix "Shared Selection") ---------------------------------------
+def test_shared_selection_is_the_layer_with_one_gate_on_both_sides():
+    rng = np.random.default_rng(91)
+    L = rand_layer(rng, 2, 10, 8, 2, 4, 4)
+    bs, bd = rng.standard_normal((2, 4)), rng.standard_normal((2, 4))
+    sh = switchhead_forward(**L, k=2, bias_s=bs, bias_d=bd, shared_selection=True)
+    # the same numbers as the ordinary layer whose destination gate is a copy of the source gate
+    L2 = dict(L, Wd=L["Ws"])
+    ref = switchhead_forward(**L2, k=2, bias_s=bs, bias_d=bs)
+    assert np.array_equal(sh["y"], ref["y"])
+    assert np.array_equal(sh["idxD"], sh["idxS"]) and np.array_equal(sh["gateD"], sh["gateS"])
+    assert np.array_equal(sh["listsD"], sh["listsS"])
+    # W_D and b_D play no part; the ordinary layer with a different W_D gives something else
+    other = dict(L, Wd=rng.standard_normal(L["Wd"].shape))
+    assert np.array_equal(switchhead_forward(**other, k=2, bias_s=bs, bias_d=None, shared_selection=True)["y"], sh["y"])
+    assert not np.allclose(switchhead_forward(**L, k=2, bias_s=bs, bias_d=bd)["y"], sh["y"])
+    # literal loop writing
+    yl = np.array(switchhead_forward_loops(**L, k=2, bias_s=bs, bias_d=bd, shared_selection=True))
+    assert np.allclose(sh["y"], yl, rtol=1e-11, atol=1e-12)
