@@ -87,7 +87,7 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(cfg, inp, seconds_budget=12.0, rope_base=None):
+def oracle_sample(cfg, inp, seconds_budget=12.0, rope_base=None, shared_selection=False):
     """Times the oracle, as it stands, on whole sequences of the workload (batch elements are
     independent), cycling through the batch until about `seconds_budget` seconds are spent."""
     from oracle.switchhead_oracle import switchhead_forward
@@ -100,7 +100,8 @@ def oracle_sample(cfg, inp, seconds_budget=12.0, rope_base=None):
         nb = min(nb, B - lo)
         t1 = time.perf_counter()
         switchhead_forward(inp.x[lo:lo + nb], inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, cfg.k,
-                           inp.bias_s, inp.bias_d, return_stages=False, rope_base=rope_base)
+                           inp.bias_s, inp.bias_d, return_stages=False, rope_base=rope_base,
+                           shared_selection=shared_selection)
         dt = time.perf_counter() - t1
         done += nb
         t_used = time.perf_counter() - t0
@@ -123,7 +124,8 @@ def run_reference(args, rank, world):
     from oracle.switchhead_oracle import switchhead_forward
     run = lambda: switchhead_forward(inp.x, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, cfg.k,
                                      inp.bias_s, inp.bias_d, return_stages=False,
-                                     rope_base=args.rope if args.rope > 0 else None)
+                                     rope_base=args.rope if args.rope > 0 else None,
+                                     shared_selection=args.shared_selection)
     for _ in range(min(args.warmup, 1)):
         run()
     t0 = time.perf_counter()
@@ -154,6 +156,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--shared-selection", action="store_true",
+                    help="one gate for the source and the destination side (the paper's Shared Selection variant)")
     ap.add_argument("--rope", type=float, default=0.0,
                     help="rotary position embeddings on Q, K with this base (0 = off, the headline configuration)")
     args = ap.parse_args()
@@ -180,7 +184,7 @@ def main():
     # each rank owns its own batch of independent sequences (same weights, rank-specific x)
     inp = inputs.make_inputs(cfg)
     inp.x = sharding.rank_batch(inp.x, rank)                                 # rows keep their gate margins
-    layer = binding.layer_from_inputs(inp)
+    layer = binding.layer_from_inputs(inp, shared_selection=args.shared_selection)
     if args.rope > 0:
         layer.sh_set_rope(args.rope)
     x = binding.to_device(inp.x, cfg.dtype)
@@ -282,6 +286,7 @@ def main():
             "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "seq_len": cfg.seq, "d_model": cfg.d_model,
                        "n_heads": cfg.n_heads, "d_head": cfg.d_head, "n_experts": cfg.n_experts, "k": cfg.k,
                        "causal": True, "rope_base": args.rope if args.rope > 0 else None,
+                       "shared_selection": bool(args.shared_selection),
                        "l2": "flushed before every timed step (256 MiB write)",
                        "parallelism": f"batch-sharded replicas x{world}, no collective"},
             "useful_tflops": useful_tflops,
@@ -321,7 +326,8 @@ def main():
                                        "useful_tflops": dense_flop / (dms * 1e-3) / 1e12}
             dl.close()
         if not args.no_cpu_baseline:
-            v, nseq, secs = oracle_sample(cfg, inp, rope_base=args.rope if args.rope > 0 else None)
+            v, nseq, secs = oracle_sample(cfg, inp, rope_base=args.rope if args.rope > 0 else None,
+                                          shared_selection=args.shared_selection)
             line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)),
                                     "kind": "oracle",
                                     "sample": f"{nseq} sequences of {cfg.seq} tokens drawn from the workload's {cfg.batch}, {secs:.1f} s, fp64 numpy"}

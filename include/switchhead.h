@@ -65,6 +65,14 @@ enum {
  * d_model a positive multiple of 64.  Returns NULL on error (see sh_last_error). */
 sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k);
 
+/* The "Shared Selection" variant of the paper's appendix: one gate serves the source and the
+ * destination side, so the output experts of a token are the ones its value projection
+ * selected, with the same scores; one top-k and one bucket sort per head instead of two.
+ * Same arguments and limits as sh_create.  sh_set_weights takes the gate as Ws / bias_s and
+ * wants NULL for Wd and bias_d; the two sides of sh_gate_topk's outputs (and of the
+ * idx / gate / offsets / lists debug buffers' first half) are then equal. */
+sh_layer* sh_create_shared(int d_model, int n_heads, int d_head, int n_experts, int k);
+
 /* Dense multi-head attention comparator (Eq. 1-2) built from the same kernels: every head
  * has one dense W_V and W_O and there are no gates.  Used only to time a parameter-matched
  * dense layer beside SwitchHead.  Weights are passed to sh_set_weights with n_experts = 1

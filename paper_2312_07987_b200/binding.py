@@ -21,7 +21,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
                -4: "SH_ERR_WORKSPACE", -5: "SH_ERR_CUDA", -6: "SH_ERR_TIMEOUT", -7: "SH_ERR_BOUNDS"}
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
-EXPORTS = ["sh_create", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
+EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
            "sh_set_weights", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
            "sh_launch_count", "sh_last_error", "sh_destroy"]
 
@@ -34,6 +34,8 @@ def _load() -> ctypes.CDLL:
     vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
     lib.sh_create.restype = vp
     lib.sh_create.argtypes = [i32] * 5
+    lib.sh_create_shared.restype = vp
+    lib.sh_create_shared.argtypes = [i32] * 5
     lib.sh_create_dense.restype = vp
     lib.sh_create_dense.argtypes = [i32] * 3
     lib.sh_configure.restype = i32
@@ -98,11 +100,16 @@ class Layer:
     """Owns one sh_layer handle plus the torch tensors that back its workspace."""
 
     def __init__(self, d_model: int, n_heads: int, d_head: int, n_experts: int = 1, k: int = 1,
-                 dense: bool = False):
+                 dense: bool = False, shared_selection: bool = False):
         self.dense = dense
+        self.shared_selection = shared_selection
         self.dims = (d_model, n_heads, d_head, n_experts, k)
-        h = lib.sh_create_dense(d_model, n_heads, d_head) if dense else \
-            lib.sh_create(d_model, n_heads, d_head, n_experts, k)
+        if dense:
+            h = lib.sh_create_dense(d_model, n_heads, d_head)
+        elif shared_selection:
+            h = lib.sh_create_shared(d_model, n_heads, d_head, n_experts, k)
+        else:
+            h = lib.sh_create(d_model, n_heads, d_head, n_experts, k)
         if not h:
             raise SwitchHeadError(-1)
         self.handle = ctypes.c_void_p(h)
@@ -209,14 +216,16 @@ def to_device(a: Optional[np.ndarray], dtype: int, device="cuda") -> Optional[to
     return t.to(device).contiguous()
 
 
-def layer_from_inputs(inp, batch=None, seq=None, device="cuda") -> "Layer":
-    """Create, configure and load a Layer from a LayerInputs record (see inputs.py)."""
+def layer_from_inputs(inp, batch=None, seq=None, device="cuda", shared_selection=False) -> "Layer":
+    """Create, configure and load a Layer from a LayerInputs record (see inputs.py).
+    shared_selection: the source gate (Ws, bias_s) serves both sides; Wd and bias_d are not used."""
     cfg = inp.cfg
     B, T = inp.x.shape[0], inp.x.shape[1]
-    L = Layer(cfg.d_model, cfg.n_heads, cfg.d_head, cfg.n_experts, cfg.k)
+    L = Layer(cfg.d_model, cfg.n_heads, cfg.d_head, cfg.n_experts, cfg.k, shared_selection=shared_selection)
     L.sh_configure(cfg.dtype, B, T, device=device)
     dv = lambda a: to_device(a, cfg.dtype, device)
     bias = lambda a: None if a is None else torch.from_numpy(a).to(device)
-    L.sh_set_weights(dv(inp.Wq), dv(inp.Wk), dv(inp.Wv), dv(inp.Wo), dv(inp.Ws), dv(inp.Wd),
-                     bias(inp.bias_s), bias(inp.bias_d))
+    L.sh_set_weights(dv(inp.Wq), dv(inp.Wk), dv(inp.Wv), dv(inp.Wo), dv(inp.Ws),
+                     None if shared_selection else dv(inp.Wd),
+                     bias(inp.bias_s), None if shared_selection else bias(inp.bias_d))
     return L

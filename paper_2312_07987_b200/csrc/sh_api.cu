@@ -68,7 +68,7 @@ static void layout_workspace(sh_layer* L) {
   o.total = off;
 }
 
-static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_experts, int k, bool dense) {
+static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_experts, int k, bool dense, int sides = 2) {
   g_err[0] = 0;
   if (d_model <= 0 || d_model % 64 != 0) { sh_set_error("d_model must be a positive multiple of 64 (got %d)", d_model); return nullptr; }
   if (n_heads < 1) { sh_set_error("n_heads must be >= 1 (got %d)", n_heads); return nullptr; }
@@ -78,13 +78,18 @@ static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_exper
   sh_layer* L = new (std::nothrow) sh_layer();
   if (!L) { sh_set_error("out of host memory"); return nullptr; }
   L->d.M = d_model; L->d.H = n_heads; L->d.D = d_head; L->d.E = n_experts; L->d.k = k;
-  L->d.G = 2 * n_heads * n_experts;
+  L->d.sides = sides;
+  L->d.G = sides * n_heads * n_experts;
   L->dense = dense;
   return L;
 }
 
 extern "C" sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k) {
   return create_common(d_model, n_heads, d_head, n_experts, k, false);
+}
+
+extern "C" sh_layer* sh_create_shared(int d_model, int n_heads, int d_head, int n_experts, int k) {
+  return create_common(d_model, n_heads, d_head, n_experts, k, false, 1);
 }
 
 extern "C" sh_layer* sh_create_dense(int d_model, int n_heads, int d_head) {
@@ -165,13 +170,15 @@ static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void
     // Ws, Wd [H, M, E] -> Wgate[(side*H + h)*E + e][m]
     TI* wg = (TI*)(ws + L->o.wgate);
     repack<TI, TI>(Ws, wg, d.H, d.M, d.E, (long)d.E * d.M, d.M, 1, st);
-    repack<TI, TI>(Wd, wg + (long)d.H * d.E * d.M, d.H, d.M, d.E, (long)d.E * d.M, d.M, 1, st);
+    if (d.sides == 2) repack<TI, TI>(Wd, wg + (long)d.H * d.E * d.M, d.H, d.M, d.E, (long)d.E * d.M, d.M, 1, st);
     float* gb = (float*)(ws + L->o.gbias);
     const size_t hb = (size_t)d.H * d.E * 4;
     if (bias_s) SH_CUDA_CHECK(cudaMemcpyAsync(gb, bias_s, hb, cudaMemcpyDeviceToDevice, st));
     else SH_CUDA_CHECK(cudaMemsetAsync(gb, 0, hb, st));
-    if (bias_d) SH_CUDA_CHECK(cudaMemcpyAsync(gb + d.H * d.E, bias_d, hb, cudaMemcpyDeviceToDevice, st));
-    else SH_CUDA_CHECK(cudaMemsetAsync(gb + d.H * d.E, 0, hb, st));
+    if (d.sides == 2) {
+      if (bias_d) SH_CUDA_CHECK(cudaMemcpyAsync(gb + d.H * d.E, bias_d, hb, cudaMemcpyDeviceToDevice, st));
+      else SH_CUDA_CHECK(cudaMemsetAsync(gb + d.H * d.E, 0, hb, st));
+    }
     // Wv [H, E, M, D] -> [H, E, D, M];  Wo [H, E, D, M] -> [H, E, M, D]
     repack<TI, TI>(Wv, ws + L->o.wv, d.H * d.E, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
     repack<TI, TM>(Wo, ws + L->o.wo, d.H * d.E, d.D, d.M, (long)d.D * d.M, d.D, 1, st);
@@ -188,7 +195,8 @@ extern "C" int sh_set_weights(sh_layer* L, const void* Wq, const void* Wk, const
   if (L->dtype < 0) { sh_set_error("sh_configure has not been called"); return SH_ERR_NOT_CONFIGURED; }
   if (!L->ws) { sh_set_error("sh_set_workspace has not been called"); return SH_ERR_WORKSPACE; }
   if (!Wq || !Wk || !Wv || !Wo) { sh_set_error("Wq, Wk, Wv and Wo must not be NULL"); return SH_ERR_INVALID_ARG; }
-  if (!L->dense && (!Ws || !Wd)) { sh_set_error("Ws and Wd must not be NULL for a SwitchHead layer"); return SH_ERR_INVALID_ARG; }
+  if (!L->dense && (!Ws || (!Wd && L->d.sides == 2))) { sh_set_error("Ws and Wd must not be NULL for a SwitchHead layer"); return SH_ERR_INVALID_ARG; }
+  if (!L->dense && L->d.sides == 1 && (Wd || bias_d)) { sh_set_error("a shared-selection layer has one gate: pass NULL for Wd and bias_d"); return SH_ERR_INVALID_ARG; }
   if (L->dense && (Ws || Wd || bias_s || bias_d)) { sh_set_error("a dense layer has no gates: pass NULL for Ws, Wd and the biases"); return SH_ERR_INVALID_ARG; }
   cudaStream_t st = (cudaStream_t)stream;
   int rc = (L->dtype == SH_F32)
@@ -285,9 +293,11 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
     ShGemmArgs o{};
     o.d = d; o.A = ws + L->o.ahat; o.lda = HD; o.a_head_stride = d.D; o.Bt = ws + L->o.wo; o.ldb = d.D;
     o.K = d.D; o.ncols = d.M;
-    const size_t side1 = (size_t)d.H * d.N * d.k;
+    // destination-side lists and tiles (with a shared selection: the one side there is)
+    const size_t side1 = d.sides == 2 ? (size_t)d.H * d.N * d.k : 0;
     o.lists = (const int*)(ws + L->o.lists) + side1; o.lgate = (const float*)(ws + L->o.lgate) + side1;
-    o.tiles = (const ShTile*)(ws + L->o.tiles) + d.max_tiles; o.ntiles = (const int*)(ws + L->o.ntiles) + 1;
+    o.tiles = (const ShTile*)(ws + L->o.tiles) + (d.sides == 2 ? d.max_tiles : 0);
+    o.ntiles = (const int*)(ws + L->o.ntiles) + (d.sides == 2 ? 1 : 0);
     o.b_group_stride = (long)d.M * d.D; o.out0 = out;
     dim3 grid_o(d.max_tiles, (d.M + 63) / 64);
     sh_simt_gemm_kernel<TM, TM, float, SH_EPI_O><<<grid_o, 256, 0, st>>>(o);
@@ -382,11 +392,15 @@ extern "C" int sh_gate_topk(sh_layer* L, const void* x, int32_t* idx, float* gat
   rc = (L->dtype == SH_F32) ? launch_gate_sort<float>(L, x, st) : sh_tc_gate_sort(L, x, st);
   if (rc != SH_OK) return rc;
   const ShDims& d = L->d;
-  const size_t slots = (size_t)2 * d.N * d.H * d.k;
-  if (idx) SH_CUDA_CHECK(cudaMemcpyAsync(idx, L->ws + L->o.idx, slots * 4, cudaMemcpyDeviceToDevice, st));
-  if (gate) SH_CUDA_CHECK(cudaMemcpyAsync(gate, L->ws + L->o.gate, slots * 4, cudaMemcpyDeviceToDevice, st));
-  if (offsets) SH_CUDA_CHECK(cudaMemcpyAsync(offsets, L->ws + L->o.offsets, (size_t)2 * d.H * (d.E + 1) * 4, cudaMemcpyDeviceToDevice, st));
-  if (lists) SH_CUDA_CHECK(cudaMemcpyAsync(lists, L->ws + L->o.lists, slots * 4, cudaMemcpyDeviceToDevice, st));
+  // side s of the outputs <- side s of the workspace (with a shared selection both <- the one side)
+  const size_t half = (size_t)d.N * d.H * d.k * 4, ohalf = (size_t)d.H * (d.E + 1) * 4;
+  for (int side = 0; side < 2; ++side) {
+    const size_t src = d.sides == 2 ? side : 0;
+    if (idx) SH_CUDA_CHECK(cudaMemcpyAsync((char*)idx + side * half, L->ws + L->o.idx + src * half, half, cudaMemcpyDeviceToDevice, st));
+    if (gate) SH_CUDA_CHECK(cudaMemcpyAsync((char*)gate + side * half, L->ws + L->o.gate + src * half, half, cudaMemcpyDeviceToDevice, st));
+    if (offsets) SH_CUDA_CHECK(cudaMemcpyAsync((char*)offsets + side * ohalf, L->ws + L->o.offsets + src * ohalf, ohalf, cudaMemcpyDeviceToDevice, st));
+    if (lists) SH_CUDA_CHECK(cudaMemcpyAsync((char*)lists + side * half, L->ws + L->o.lists + src * half, half, cudaMemcpyDeviceToDevice, st));
+  }
   return SH_OK;
 }
 

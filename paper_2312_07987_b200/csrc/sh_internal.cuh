@@ -17,7 +17,8 @@ struct ShDims {
   int M, H, D, E, k;
   int B, T;
   int N;                   // B*T tokens
-  int G;                   // gate columns = 2*H*E
+  int sides;               // 2: source and destination gates; 1: shared selection (one gate serves both)
+  int G;                   // gate columns = sides*H*E
   int nblk;                // ceil(N / SH_TILE_ROWS)
   int max_tiles;           // upper bound on row tiles per side
   int tile_rows_src;       // rows per tile of the source-side (value expert) tile table: 128 or 256

@@ -31,8 +31,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const float* __restrict__ gbias,
                     int* __restrict__ idx, float* __restrict__ gate, int* __restrict__ blockcnt, ShDims d) {
-  extern __shared__ int s_hist[];            // [2*H*E]
-  const int nb = 2 * d.H * d.E;
+  extern __shared__ int s_hist[];            // [G]
+  const int nb = d.G;
   for (int i = threadIdx.x; i < nb; i += blockDim.x) s_hist[i] = 0;
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -41,7 +41,7 @@ sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const flo
     const int t = tok0 + tt;
     if (t >= d.N) break;
     const T* xr = x + (size_t)t * d.M;
-    for (int grp = 0; grp < 2 * d.H; ++grp) {
+    for (int grp = 0; grp < d.sides * d.H; ++grp) {
       float z = 0.f;                         // lane e keeps logit e
       for (int e0 = 0; e0 < d.E; e0 += 4) {
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -141,7 +141,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
       }
     }
   }
-  for (int side = 0; side < 2; ++side) {                          // this block's selections
+  for (int side = 0; side < d.sides; ++side) {                    // this block's selections
     const size_t base = ((size_t)side * d.N + tok0) * per_tok;
     for (int i = tid; i < nrows * per_tok; i += blockDim.x) {
       s_idx[side * 128 * per_tok + i] = idx[base + i];
@@ -165,14 +165,14 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     }
   }
   __syncthreads();
-  for (int g = tid; g < 2 * d.H; g += blockDim.x) {
+  for (int g = tid; g < d.sides * d.H; g += blockDim.x) {
     int run = 0;
     for (int e = 0; e < d.E; ++e) {
       s_off[g * d.E + e] = run;
       run += s_tot[g * d.E + e];
     }
   }
-  for (int grp = gs; grp < 2 * d.H; grp += GS) {                  // per-warp counts of this block's tokens
+  for (int grp = gs; grp < d.sides * d.H; grp += GS) {            // per-warp counts of this block's tokens
     const int side = grp / d.H, h = grp % d.H;
     unsigned mask = 0;
     if (tl < nrows)
@@ -185,7 +185,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
   __syncthreads();
   {
     const int t = tok0 + tl;
-    for (int grp = gs; grp < 2 * d.H; grp += GS) {
+    for (int grp = gs; grp < d.sides * d.H; grp += GS) {
       const int side = grp / d.H, h = grp % d.H;
       const int sel = side * 128 * per_tok + (tl * d.H + h) * d.k;
       unsigned mask = 0;
@@ -209,11 +209,11 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     }
   }
   if (blk != 0) return;
-  for (int g = tid; g < 2 * d.H; g += blockDim.x) {
+  for (int g = tid; g < d.sides * d.H; g += blockDim.x) {
     for (int e = 0; e < d.E; ++e) offsets[g * (d.E + 1) + e] = s_off[g * d.E + e];
     offsets[g * (d.E + 1) + d.E] = s_off[g * d.E + d.E - 1] + s_tot[g * d.E + d.E - 1];
   }
-  if (tid < 2) {
+  if (tid < d.sides) {
     const int side = tid;
     int run = 0;
     for (int b = side * d.H * d.E; b < (side + 1) * d.H * d.E; ++b) {
@@ -241,7 +241,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
 
 static inline int sh_sort_threads(const ShDims& d) {
   // at most 512 threads (16 K registers), so that a block fits beside a 320-thread GEMM CTA on an SM
-  int gs = 2 * d.H;
+  int gs = d.sides * d.H;
   if (gs > 4) gs = 4;
   return 128 * gs;
 }

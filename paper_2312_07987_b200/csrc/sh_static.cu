@@ -101,7 +101,7 @@ extern "C" int sh_noalloc_gate_topk(int dtype, int n_tokens, int d_model, int n_
   if (rc != SH_OK) return rc;
   ShDims d{};
   d.M = d_model; d.H = n_heads; d.D = 0; d.E = n_experts; d.k = k;
-  d.B = 1; d.T = n_tokens; d.N = n_tokens; d.G = (int)G;
+  d.B = 1; d.T = n_tokens; d.N = n_tokens; d.sides = 2; d.G = (int)G;
   d.nblk = (n_tokens + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
   d.max_tiles = kMaxTiles;
   d.tile_rows_src = SH_TILE_ROWS;

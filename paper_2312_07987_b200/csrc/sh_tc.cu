@@ -166,7 +166,10 @@ int sh_tc_prepare(sh_layer* L) {
   // enough of them to fill the SMs one and a half times
   const long long slots = (long long)d.N * d.H * d.k;
   const bool big = slots / 256 >= (3ll * L->sm_count) / 2;
-  L->d.tile_rows_src = (L->dense || (S->simt_mask & SH_STAGE_V) || getenv("SH_V_TILE128") || !big) ? 128 : 256;
+  // (with a shared selection the destination-side consumers of the tile table -- the CUDA-core and
+  //  scatter-add output projections, debugging paths here -- read the source side's 128-row tiles)
+  const bool dst_reads_src_tiles = L->d.sides == 1 && ((S->simt_mask & SH_STAGE_O) || getenv("SH_O_SCATTER"));
+  L->d.tile_rows_src = (L->dense || (S->simt_mask & SH_STAGE_V) || getenv("SH_V_TILE128") || !big || dst_reads_src_tiles) ? 128 : 256;
   int rc;
   if ((rc = sh_tc_encode_2d(&S->map_wqk, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, S->qk_bn))) return rc;
   if (!L->dense) {
@@ -407,9 +410,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     TcGemmArgs g{};
     g.d = d; g.K = d.D; g.ncols = d.M;
     g.A = ws + L->o.ahat; g.lda = HD;
-    const size_t side1 = (size_t)d.H * d.N * d.k;
+    const size_t side1 = d.sides == 2 ? (size_t)d.H * d.N * d.k : 0;
     g.lists = (const int*)(ws + L->o.lists) + side1; g.lgate = (const float*)(ws + L->o.lgate) + side1;
-    g.tiles = (const ShTile*)(ws + L->o.tiles) + d.max_tiles; g.ntiles = (const int*)(ws + L->o.ntiles) + 1;
+    g.tiles = (const ShTile*)(ws + L->o.tiles) + (d.sides == 2 ? d.max_tiles : 0);
+    g.ntiles = (const int*)(ws + L->o.ntiles) + (d.sides == 2 ? 1 : 0);
     g.b_rows_per_group = d.M; g.out0 = out; g.status = status;
     dim3 grid(d.max_tiles, (d.M + 127) / 128);
     if ((rc = launch_gemm<128, 3, GEMM_O, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
@@ -417,7 +421,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   } else if (!L->dense) {
     TcOprojArgs a{};
     a.d = d;
-    const size_t side1 = (size_t)d.N * d.H * d.k;
+    const size_t side1 = d.sides == 2 ? (size_t)d.N * d.H * d.k : 0;   // shared selection: the one side there is
     a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
     a.out = (float*)out; a.status = status;
     a.nwork = d.nblk * ((d.M + 255) / 256);

@@ -145,7 +145,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       }
       const int t = row0 + r;
       if (r < nrows) {
-        for (int grp = 0; grp < 2 * d.H; ++grp) {
+        for (int grp = 0; grp < d.sides * d.H; ++grp) {
           const float* z = srow + grp * d.E;
           const int side = grp / d.H, h = grp % d.H;
           const size_t o = (((size_t)side * d.N + t) * d.H + h) * d.k;

@@ -11,10 +11,10 @@ from paper_2312_07987_b200 import binding, inputs
 TOL_Y = {inputs.DTYPE_F32: 1e-4, inputs.DTYPE_BF16: 2e-2}
 
 
-def oracle_for(inp, batches=None, rope_base=None):
+def oracle_for(inp, batches=None, rope_base=None, shared_selection=False):
     x = inp.x if batches is None else inp.x[batches]
     return switchhead_forward(x, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, inp.cfg.k,
-                              inp.bias_s, inp.bias_d, rope_base=rope_base)
+                              inp.bias_s, inp.bias_d, rope_base=rope_base, shared_selection=shared_selection)
 
 
 def rel_rms_err(got, ref):
@@ -45,9 +45,9 @@ def check_lists(off_gpu, lists_gpu, ref):
         assert np.array_equal(lists_gpu[side], ref[lk]), f"side {side}: token lists differ"
 
 
-def run_layer(inp, device="cuda"):
+def run_layer(inp, device="cuda", shared_selection=False):
     cfg = inp.cfg
-    layer = binding.layer_from_inputs(inp, device=device)
+    layer = binding.layer_from_inputs(inp, device=device, shared_selection=shared_selection)
     x = binding.to_device(inp.x, cfg.dtype, device)
     y = layer.sh_forward(x)
     torch.cuda.synchronize()

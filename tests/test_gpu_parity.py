@@ -10,11 +10,11 @@ from tests import parity_util as pu
 pytestmark = pytest.mark.gpu
 
 
-def full_check(inp, check_stage_buffers=True, batches=None):
+def full_check(inp, check_stage_buffers=True, batches=None, shared_selection=False):
     cfg = inp.cfg
     B, T = inp.x.shape[:2]
-    layer, x, y = pu.run_layer(inp)
-    ref = pu.oracle_for(inp, batches)
+    layer, x, y = pu.run_layer(inp, shared_selection=shared_selection)
+    ref = pu.oracle_for(inp, batches, shared_selection=shared_selection)
     yb = y.cpu().numpy() if batches is None else y.cpu().numpy()[batches]
     idx, gate, off, lists = (t.cpu().numpy() for t in layer.sh_gate_topk(x))
     torch.cuda.synchronize()
@@ -174,3 +174,28 @@ def test_rope_bf16_configs():
 
 def test_rope_long_context_sampled_sequence():
     rope_check(inputs.make_inputs(inputs.CONFIGS["long_ctx_bf16"]), batches=[2])       # positions up to 4095
+
+
+# ---- shared selection (sh_create_shared): one gate for the source and the destination side ---
+def test_shared_selection_f32():
+    full_check(inputs.make_inputs(inputs.CONFIGS["tiny_f32"]), shared_selection=True)
+    cfg = inputs.LayerConfig("shared_f32", inputs.DTYPE_F32, 2, 130, 128, 3, 32, 5, 2, seed=41, zipf_bias=1.2)
+    full_check(inputs.make_inputs(cfg), shared_selection=True)
+
+
+def test_shared_selection_bf16():
+    full_check(inputs.make_inputs(inputs.CONFIGS["small_bf16"]), shared_selection=True)
+    full_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=4), shared_selection=True)
+    cfg = inputs.LayerConfig("shared_bf16", inputs.DTYPE_BF16, 1, 515, 256, 3, 128, 16, 4, seed=42)
+    full_check(inputs.make_inputs(cfg), shared_selection=True)
+
+
+def test_shared_selection_rejects_a_destination_gate():
+    inp = inputs.make_inputs(inputs.CONFIGS["tiny_f32"])
+    from paper_2312_07987_b200 import binding
+    L = binding.Layer(inp.cfg.d_model, inp.cfg.n_heads, inp.cfg.d_head, inp.cfg.n_experts, inp.cfg.k, shared_selection=True)
+    L.sh_configure(inp.cfg.dtype, *inp.x.shape[:2])
+    dv = lambda a: binding.to_device(a, inp.cfg.dtype)
+    with pytest.raises(binding.SwitchHeadError):
+        L.sh_set_weights(dv(inp.Wq), dv(inp.Wk), dv(inp.Wv), dv(inp.Wo), dv(inp.Ws), dv(inp.Wd))
+    L.close()
