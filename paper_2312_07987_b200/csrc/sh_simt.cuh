@@ -224,7 +224,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     ntiles[side] = run;
   }
   __syncthreads();
-  for (int i = tid; i < nb * 32; i += blockDim.x) {               // 32 threads share a bucket's tiles
+  for (int i = tid; i < d.sides * d.H * d.E * 32; i += blockDim.x) {   // 32 threads share a bucket's tiles
     const int b = i >> 5;
     const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
     const int cnt = s_tot[b];

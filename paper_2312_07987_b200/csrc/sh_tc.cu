@@ -247,10 +247,16 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
     SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
     sort_cfg = ssm;
   }
-  if ((rc = launch_k(S->pdl && !L->ev && (S->pdl_mask & 1), sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(d)), ssm, st,
+  // In a forward pass only the value experts read sorted lists (the output projection works from
+  // idx / gate, token tile by token tile), so only the source side is sorted there -- unless the
+  // scatter-add or CUDA-core output projection (debugging paths) is selected.  The histogram stride
+  // stays G; the kernel's loops run over sides * H groups.
+  ShDims ds = d;
+  if (zero_for_forward && !S->o_scatter && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
+  if ((rc = launch_k(S->pdl && !L->ev && (S->pdl_mask & 1), sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(ds)), ssm, st,
                      (const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate), (const int*)(ws + L->o.blockcnt),
                      (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists), (float*)(ws + L->o.lgate),
-                     (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d)))
+                     (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), ds)))
     return rc;
   L->launches += 2;
   return SH_OK;
