@@ -108,6 +108,12 @@ int sh_set_weights(sh_layer* layer, const void* Wq, const void* Wk, const void* 
                    const void* Wo, const void* Ws, const void* Wd, const float* bias_s,
                    const float* bias_d, void* stream);
 
+/* Attention mask.  causal != 0 (the default): the language-model setting, key s is visible to
+ * query t iff s <= t.  causal == 0: every key of the sequence is visible (the paper's ListOps
+ * classifier uses SwitchHead without autoregressive masking).  Host-only; takes effect with
+ * the next sh_forward. */
+int sh_set_causal(sh_layer* layer, int causal);
+
 /* Rotary position embeddings on the queries and keys (the paper's appendix "RoPE Positional
  * Encodings": square causal attention without a cache, RoPE as in RoFormer).  Token t of a
  * sequence sits at position t; the feature pair (2i, 2i+1) of its query and key vectors of

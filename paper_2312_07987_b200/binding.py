@@ -22,7 +22,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
 EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
-           "sh_set_weights", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
+           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
            "sh_launch_count", "sh_last_error", "sh_destroy"]
 
 
@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_gate_topk.argtypes = [vp] * 7
     lib.sh_noalloc_gate_topk.restype = i32
     lib.sh_noalloc_gate_topk.argtypes = [i32] * 6 + [vp] * 8
+    lib.sh_set_causal.restype = i32
+    lib.sh_set_causal.argtypes = [vp, i32]
     lib.sh_set_rope.restype = i32
     lib.sh_set_rope.argtypes = [vp, ctypes.c_double, vp]
     lib.sh_debug_buffer.restype = i32
@@ -132,6 +134,9 @@ class Layer:
             assert t is None or (t.is_cuda and t.is_contiguous())
         _check(lib.sh_set_weights(self.handle, *[_ptr(t) for t in ts], _stream()))
         torch.cuda.current_stream().synchronize()   # the source tensors may now be released
+
+    def sh_set_causal(self, causal: bool) -> None:
+        _check(lib.sh_set_causal(self.handle, 1 if causal else 0))
 
     def sh_set_rope(self, base: float) -> None:
         _check(lib.sh_set_rope(self.handle, float(base), _stream()))

@@ -79,6 +79,7 @@ static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_exper
   if (!L) { sh_set_error("out of host memory"); return nullptr; }
   L->d.M = d_model; L->d.H = n_heads; L->d.D = d_head; L->d.E = n_experts; L->d.k = k;
   L->d.sides = sides;
+  L->d.causal = 1;
   L->d.G = sides * n_heads * n_experts;
   L->dense = dense;
   return L;
@@ -331,6 +332,13 @@ static __global__ void sh_rope_table_kernel(float2* table, int T, int D, double 
   double s, c;
   sincos(ang, &s, &c);
   table[(size_t)i * T + t] = make_float2((float)c, (float)s);
+}
+
+extern "C" int sh_set_causal(sh_layer* L, int causal) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  L->d.causal = causal ? 1 : 0;
+  return SH_OK;
 }
 
 extern "C" int sh_set_rope(sh_layer* L, double base, void* stream) {

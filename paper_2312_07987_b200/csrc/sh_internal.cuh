@@ -22,6 +22,7 @@ struct ShDims {
   int nblk;                // ceil(N / SH_TILE_ROWS)
   int max_tiles;           // upper bound on row tiles per side
   int tile_rows_src;       // rows per tile of the source-side (value expert) tile table: 128 or 256
+  int causal;              // 1: key s visible to query t iff s <= t (default); 0: every key of the sequence
 };
 
 // Workspace sub-buffers (byte offsets from the workspace base).

@@ -390,7 +390,7 @@ sh_simt_gemm_kernel(ShGemmArgs g) {
 }
 
 // ---------------------------------------------------------------------------------------
-// CUDA-core causal attention (Eq. 1 with the autoregressive mask): one warp per query row,
+// CUDA-core attention (Eq. 1, with the autoregressive mask unless d.causal == 0): one warp per query row,
 // keys in chunks of 32 (lane = key), online softmax in base 2 (Q carries log2(e)/sqrt(D)).
 // Q, K, V [B, H, T, D]; Ahat [B*T, H, D].
 // ---------------------------------------------------------------------------------------
@@ -412,10 +412,11 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
   __syncwarp();
   float o[4] = {0.f, 0.f, 0.f, 0.f};                    // lane owns d = lane + 32*i
   float m = -INFINITY, l = 0.f;
-  for (int s0 = 0; s0 <= t; s0 += 32) {
+  const int last = d.causal ? t : d.T - 1;              // last visible key
+  for (int s0 = 0; s0 <= last; s0 += 32) {
     const int s = s0 + lane;
     float sc = -INFINITY;
-    if (s <= t) {
+    if (s <= last) {
       const TM* kr = Kb + (long)s * d.D;
       float a = 0.f;
       for (int i = 0; i < d.D; ++i) a = fmaf(s_q[warp][i], sh_to_float<TM>(kr[i]), a);
@@ -426,7 +427,7 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
     for (int x = 16; x > 0; x >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, x));
     const float mn = fmaxf(m, cm);
     const float alpha = exp2f(m - mn);                  // m = -inf first time -> 0
-    const float p = (s <= t) ? exp2f(sc - mn) : 0.f;
+    const float p = (s <= last) ? exp2f(sc - mn) : 0.f;
     float ps = p;
 #pragma unroll
     for (int x = 16; x > 0; x >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, x);
@@ -434,7 +435,7 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
     m = mn;
 #pragma unroll
     for (int i = 0; i < 4; ++i) o[i] *= alpha;
-    const int cnt = min(32, t - s0 + 1);
+    const int cnt = min(32, last - s0 + 1);
     for (int j = 0; j < cnt; ++j) {
       const float pj = __shfl_sync(0xffffffffu, p, j);
       const TM* vr = Vb + (long)(s0 + j) * d.D;

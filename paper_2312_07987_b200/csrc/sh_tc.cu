@@ -384,7 +384,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
     static bool cfg128 = false, cfg64 = false, cfg2_128 = false, cfg2_64 = false;
-    if (S->attn_single_tile) {
+    if (S->attn_single_tile && d.causal) {
       const int nq = (d.T + 127) / 128;
       const unsigned grid = (unsigned)(nq * d.B * d.H);
       if (d.D == 128) {

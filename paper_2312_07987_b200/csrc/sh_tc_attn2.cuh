@@ -59,8 +59,10 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   const int qt = nq - 1 - (int)(blockIdx.x / BH);        // heaviest query tiles first
   const int bh = blockIdx.x % BH;
   const int q0 = qt * 256;
-  const int n0 = 2 * qt + 1;                             // steps of query tile 0
-  const int n1 = (q0 + 128 < d.T) ? 2 * qt + 2 : 0;      // steps of query tile 1 (0: no such rows)
+  // key tiles each query tile attends to: up to its diagonal tile, or (d.causal == 0) all of them
+  const int nkt = (d.T + 127) / 128;
+  const int n0 = d.causal ? 2 * qt + 1 : nkt;            // steps of query tile 0
+  const int n1 = (q0 + 128 < d.T) ? (d.causal ? 2 * qt + 2 : nkt) : 0;   // steps of query tile 1 (0: no such rows)
   const int nsteps = n1 > n0 ? n1 : n0;
   bool dead = false;
 
@@ -186,10 +188,13 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive(&s_empty[t]);
-      if (j == n - 1) {                                      // diagonal tile: key c visible iff c <= r
+      if (j == n - 1) {
+        // last tile: the diagonal one (key c visible iff c <= r), or without the causal mask the
+        // tile that holds the end of the sequence (keys past it were zero-filled by the loads)
+        const int cmax = d.causal ? r : d.T - 1 - j * 128;
 #pragma unroll
         for (int c = 0; c < 128; ++c)
-          if (c > r) sv[c] = 0xff800000u;                    // -inf
+          if (c > cmax) sv[c] = 0xff800000u;                 // -inf
       }
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll

@@ -11,10 +11,11 @@ from paper_2312_07987_b200 import binding, inputs
 TOL_Y = {inputs.DTYPE_F32: 1e-4, inputs.DTYPE_BF16: 2e-2}
 
 
-def oracle_for(inp, batches=None, rope_base=None, shared_selection=False):
+def oracle_for(inp, batches=None, rope_base=None, shared_selection=False, causal=True):
     x = inp.x if batches is None else inp.x[batches]
     return switchhead_forward(x, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd, inp.cfg.k,
-                              inp.bias_s, inp.bias_d, rope_base=rope_base, shared_selection=shared_selection)
+                              inp.bias_s, inp.bias_d, causal=causal, rope_base=rope_base,
+                              shared_selection=shared_selection)
 
 
 def rel_rms_err(got, ref):

@@ -58,6 +58,7 @@ def test_call_order_and_argument_errors():
     assert lib.sh_debug_buffer(h, 0, ctypes.byref(p), ctypes.byref(n)) == -3
     assert lib.sh_last_status(None, None) == -1
     assert lib.sh_set_rope(None, 10000.0, None) == -1
+    assert lib.sh_set_causal(None, 0) == -1 and lib.sh_set_causal(h, 0) == 0 and lib.sh_set_causal(h, 1) == 0
     assert lib.sh_set_rope(h, 10000.0, None) == -3                   # configured, but no workspace yet
     assert lib.sh_set_rope(h, -1.0, None) in (-3, -1)
     h2 = ctypes.c_void_p(lib.sh_create(128, 2, 32, 4, 2))

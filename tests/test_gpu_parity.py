@@ -199,3 +199,37 @@ def test_shared_selection_rejects_a_destination_gate():
     with pytest.raises(binding.SwitchHeadError):
         L.sh_set_weights(dv(inp.Wq), dv(inp.Wk), dv(inp.Wv), dv(inp.Wo), dv(inp.Ws), dv(inp.Wd))
     L.close()
+
+
+# ---- attention without the autoregressive mask (sh_set_causal(0)) ---------------------------
+def noncausal_check(inp, batches=None):
+    cfg = inp.cfg
+    layer, x, y_causal = pu.run_layer(inp)
+    layer.sh_set_causal(False)
+    y = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0
+    ref = pu.oracle_for(inp, batches, causal=False)
+    pu.check_stages(layer, ref, cfg, batches)
+    yb = y.cpu().numpy() if batches is None else y.cpu().numpy()[batches]
+    err = pu.rel_rms_err(yb, ref["y"])
+    assert err < pu.TOL_Y[cfg.dtype], f"output max-abs error / rms = {err:.3e}"
+    if inp.x.shape[1] > 1:
+        # the last token of a sequence sees the same keys either way; an earlier one does not
+        assert not torch.allclose(y[:, 0], y_causal[:, 0], rtol=1e-3, atol=1e-3)
+    layer.close()
+
+
+def test_noncausal_f32():
+    noncausal_check(inputs.make_inputs(inputs.CONFIGS["tiny_f32"]))
+    noncausal_check(inputs.make_inputs(inputs.LayerConfig("nc_f32", inputs.DTYPE_F32, 2, 131, 128, 2, 64, 4, 2, seed=51)))
+
+
+@pytest.mark.parametrize("T,B,H,D", [(1, 2, 2, 64), (100, 2, 2, 64), (128, 1, 1, 128), (129, 2, 2, 128), (384, 1, 2, 128), (515, 1, 3, 128)])
+def test_noncausal_bf16_shapes(T, B, H, D):
+    cfg = inputs.LayerConfig("nc_bf16", inputs.DTYPE_BF16, B, T, 256, H, D, 4, 2, seed=60 + T)
+    noncausal_check(inputs.make_inputs(cfg))
+
+
+def test_noncausal_c4_262m_sampled():
+    noncausal_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=3))
