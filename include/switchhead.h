@@ -61,8 +61,11 @@ enum {
 };
 
 /* Create a layer description.  Host-only, no CUDA call.
- * Requires 1 <= k <= n_experts <= 32, n_heads >= 1, d_head in {32, 64, 128},
- * d_model a positive multiple of 64.  Returns NULL on error (see sh_last_error). */
+ * Requires 1 <= k <= n_experts <= 32, n_heads >= 1, 1 <= d_head <= 128, d_model a positive
+ * multiple of 64.  d_head is stored padded with zero columns to 64 or 128 (bf16 storage) or
+ * to 32, 64 or 128 (fp32): the padding changes no result (the scale stays 1/sqrt(d_head)),
+ * it costs the time of the padded size, and the Q, K, V, Ahat debug buffers have the padded
+ * width.  Returns NULL on error (see sh_last_error). */
 sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k);
 
 /* The "Shared Selection" variant of the paper's appendix: one gate serves the source and the
@@ -81,8 +84,8 @@ sh_layer* sh_create_dense(int d_model, int n_heads, int d_head);
 
 /* Fix the storage type and the problem size.  dtype SH_F32: x and weights fp32, all
  * arithmetic fp32 on CUDA cores.  dtype SH_BF16: x and weights bf16, tensor-core products
- * with fp32 accumulation, fp16 intermediates (Q, K, V, P, A^h V^h); requires d_head in
- * {64, 128} and d_model a multiple of 128.  `out` is fp32 in both cases.
+ * with fp32 accumulation, fp16 intermediates (Q, K, V, P, A^h V^h); requires d_model a
+ * multiple of 128.  `out` is fp32 in both cases.
  * batch*seq*n_heads*k must be below 2^31.  Invalidates workspace and weights. */
 int sh_configure(sh_layer* layer, int dtype, int batch, int seq);
 

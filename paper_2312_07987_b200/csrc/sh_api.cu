@@ -72,12 +72,13 @@ static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_exper
   g_err[0] = 0;
   if (d_model <= 0 || d_model % 64 != 0) { sh_set_error("d_model must be a positive multiple of 64 (got %d)", d_model); return nullptr; }
   if (n_heads < 1) { sh_set_error("n_heads must be >= 1 (got %d)", n_heads); return nullptr; }
-  if (d_head != 32 && d_head != 64 && d_head != 128) { sh_set_error("d_head must be 32, 64 or 128 (got %d)", d_head); return nullptr; }
+  if (d_head < 1 || d_head > 128) { sh_set_error("d_head must be in 1..128 (got %d)", d_head); return nullptr; }
   if (n_experts < 1 || n_experts > 32) { sh_set_error("n_experts must be in 1..32 (got %d)", n_experts); return nullptr; }
   if (k < 1 || k > n_experts) { sh_set_error("k must be in 1..n_experts (got k=%d, n_experts=%d)", k, n_experts); return nullptr; }
   sh_layer* L = new (std::nothrow) sh_layer();
   if (!L) { sh_set_error("out of host memory"); return nullptr; }
-  L->d.M = d_model; L->d.H = n_heads; L->d.D = d_head; L->d.E = n_experts; L->d.k = k;
+  L->d.M = d_model; L->d.H = n_heads; L->d.Dt = d_head; L->d.E = n_experts; L->d.k = k;
+  L->d.D = d_head <= 32 ? 32 : d_head <= 64 ? 64 : 128;        // sh_configure fixes it for the storage type
   L->d.sides = sides;
   L->d.causal = 1;
   L->d.G = sides * n_heads * n_experts;
@@ -103,10 +104,13 @@ extern "C" int sh_configure(sh_layer* L, int dtype, int batch, int seq) {
   if (dtype != SH_F32 && dtype != SH_BF16) { sh_set_error("dtype must be SH_F32 or SH_BF16 (got %d)", dtype); return SH_ERR_INVALID_ARG; }
   if (batch < 1 || seq < 1) { sh_set_error("batch and seq must be >= 1 (got %d, %d)", batch, seq); return SH_ERR_INVALID_ARG; }
   const ShDims& d0 = L->d;
-  if (dtype == SH_BF16 && (d0.D < 64 || d0.M % 128 != 0)) {
-    sh_set_error("bf16 path needs d_head in {64,128} and d_model %% 128 == 0 (got d_head=%d, d_model=%d)", d0.D, d0.M);
+  if (dtype == SH_BF16 && d0.M % 128 != 0) {
+    sh_set_error("bf16 path needs d_model %% 128 == 0 (got d_model=%d)", d0.M);
     return SH_ERR_UNSUPPORTED;
   }
+  // d_head is stored padded with zero columns: to 64 or 128 on the tensor-core path, to 32, 64 or
+  // 128 on the fp32 path (zero columns of W_Q, W_K, W_V and zero rows of W_O change no result)
+  L->d.D = dtype == SH_BF16 ? (d0.Dt <= 64 ? 64 : 128) : (d0.Dt <= 32 ? 32 : d0.Dt <= 64 ? 64 : 128);
   const long long slots = (long long)batch * seq * d0.H * d0.k;
   if (slots >= (1ll << 31) || (long long)batch * seq * d0.M >= (1ll << 40)) {
     sh_set_error("problem too large: batch*seq*n_heads*k = %lld must be below 2^31", slots);
@@ -159,14 +163,19 @@ static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void
   char* ws = L->ws;
   const long HD = (long)d.H * d.D;
   SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.status, 0, 256, st));
-  // Wq, Wk [H, M, D] -> Wqk[(which*H + h)*D + dd][m]
+  // Wq, Wk [H, M, Dt] -> Wqk[(which*H + h)*D + dd][m]   (rows dd >= Dt stay zero)
   TI* wqk = (TI*)(ws + L->o.wqk);
-  repack<TI, TI>(Wq, wqk, d.H, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
-  repack<TI, TI>(Wk, wqk + HD * d.M, d.H, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
+  if (d.D != d.Dt) {
+    SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wqk, 0, (size_t)(L->dense ? 3 : 2) * HD * d.M * sizeof(TI), st));
+    SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wo, 0, (size_t)HD * d.E * d.M * sizeof(TM), st));
+    if (!L->dense) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wv, 0, (size_t)HD * d.E * d.M * sizeof(TI), st));
+  }
+  repack<TI, TI>(Wq, wqk, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+  repack<TI, TI>(Wk, wqk + HD * d.M, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
   if (L->dense) {
     // Wv [H, 1, M, D] joins the fused projection; Wo [H, 1, D, M] -> Wo_t[m][h*D + dd]
-    repack<TI, TI>(Wv, wqk + 2 * HD * d.M, d.H, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
-    repack<TI, TM>(Wo, ws + L->o.wo, d.H, d.D, d.M, d.D, HD, 1, st);
+    repack<TI, TI>(Wv, wqk + 2 * HD * d.M, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+    repack<TI, TM>(Wo, ws + L->o.wo, d.H, d.Dt, d.M, d.D, HD, 1, st);
   } else {
     // Ws, Wd [H, M, E] -> Wgate[(side*H + h)*E + e][m]
     TI* wg = (TI*)(ws + L->o.wgate);
@@ -181,8 +190,8 @@ static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void
       else SH_CUDA_CHECK(cudaMemsetAsync(gb + d.H * d.E, 0, hb, st));
     }
     // Wv [H, E, M, D] -> [H, E, D, M];  Wo [H, E, D, M] -> [H, E, M, D]
-    repack<TI, TI>(Wv, ws + L->o.wv, d.H * d.E, d.M, d.D, (long)d.D * d.M, d.M, 1, st);
-    repack<TI, TM>(Wo, ws + L->o.wo, d.H * d.E, d.D, d.M, (long)d.D * d.M, d.D, 1, st);
+    repack<TI, TI>(Wv, ws + L->o.wv, d.H * d.E, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+    repack<TI, TM>(Wo, ws + L->o.wo, d.H * d.E, d.Dt, d.M, (long)d.D * d.M, d.D, 1, st);
   }
   SH_CUDA_CHECK(cudaGetLastError());
   return SH_OK;
@@ -248,7 +257,7 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   const ShDims& d = L->d;
   char* ws = L->ws;
   const int HD = d.H * d.D;
-  const float qscale = 1.4426950408889634f / sqrtf((float)d.D);
+  const float qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
   const bool all = stages == SH_STAGE_ALL;
   if (all) sh_mark(L, 0, st);
   if (!L->dense && (stages & SH_STAGE_GATE)) {
@@ -323,12 +332,13 @@ int sh_simt_run_bf16(sh_layer* L, int stages, const void* x, void* out, cudaStre
 // (cos, sin)(t * base^(-2i/D)) for every feature pair i < D/2 and position t < T, computed in
 // double precision, stored as float2 [D/2][T] (positions contiguous: the epilogue threads of a
 // warp hold consecutive tokens and read one pair at a time).
-static __global__ void sh_rope_table_kernel(float2* table, int T, int D, double base) {
+static __global__ void sh_rope_table_kernel(float2* table, int T, int D, int Dt, double base) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   const int half = D / 2;
   if (idx >= T * half) return;
   const int t = idx / half, i = idx % half;
-  const double ang = (double)t * pow(base, -2.0 * (double)i / (double)D);
+  // pairs past the given d_head are zero padding: identity
+  const double ang = 2 * i < Dt ? (double)t * pow(base, -2.0 * (double)i / (double)Dt) : 0.0;
   double s, c;
   sincos(ang, &s, &c);
   table[(size_t)i * T + t] = make_float2((float)c, (float)s);
@@ -347,9 +357,9 @@ extern "C" int sh_set_rope(sh_layer* L, double base, void* stream) {
   if (L->dtype < 0 || !L->ws) { sh_set_error("sh_set_rope needs a configured layer with its workspace"); return SH_ERR_NOT_CONFIGURED; }
   if (!(base >= 0.0) || base != base) { sh_set_error("rotary base must be positive (0 switches it off), got %g", base); return SH_ERR_INVALID_ARG; }
   if (base == 0.0) { L->rope = false; return SH_OK; }
-  if (L->d.D % 2) { sh_set_error("rotary embedding needs an even d_head"); return SH_ERR_UNSUPPORTED; }
+  if (L->d.Dt % 2) { sh_set_error("rotary embedding needs an even d_head (got %d)", L->d.Dt); return SH_ERR_UNSUPPORTED; }
   const int n = L->d.T * (L->d.D / 2);
-  sh_rope_table_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>((float2*)(L->ws + L->o.rope), L->d.T, L->d.D, base);
+  sh_rope_table_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>((float2*)(L->ws + L->o.rope), L->d.T, L->d.D, L->d.Dt, base);
   SH_CUDA_CHECK(cudaGetLastError());
   L->rope = true;
   return SH_OK;

@@ -14,7 +14,8 @@ struct ShTile {            // one row tile of one (head, expert) group
 };
 
 struct ShDims {
-  int M, H, D, E, k;
+  int M, H, D, E, k;       // D: d_head as stored (padded with zero columns to 32, 64 or 128)
+  int Dt;                  // d_head as given (scale 1/sqrt(Dt), rotary angles)
   int B, T;
   int N;                   // B*T tokens
   int sides;               // 2: source and destination gates; 1: shared selection (one gate serves both)

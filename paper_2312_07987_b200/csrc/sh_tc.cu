@@ -329,7 +329,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     TcGemmArgs g{};
     g.d = d; g.K = d.M; g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
     g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
-    g.qscale = 1.4426950408889634f / sqrtf((float)d.D);
+    g.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
     g.status = status;
     g.sched = status + 16;
     g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;

@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 
 
 @pytest.mark.parametrize("args,frag", [((100, 2, 32, 4, 2), "d_model"), ((128, 0, 32, 4, 2), "n_heads"),
-                                       ((128, 2, 48, 4, 2), "d_head"), ((128, 2, 32, 33, 2), "n_experts"),
+                                       ((128, 2, 129, 4, 2), "d_head"), ((128, 2, 32, 33, 2), "n_experts"),
                                        ((128, 2, 32, 4, 0), "k must"), ((128, 2, 32, 4, 5), "k must")])
 def test_create_rejects_bad_dimensions(args, frag):
     h = binding.lib.sh_create(*args)
@@ -43,8 +43,10 @@ def test_call_order_and_argument_errors():
     assert lib.sh_forward(h, None, None, None) == -3                 # not configured
     assert lib.sh_configure(h, 7, 1, 64) == -1
     assert lib.sh_configure(h, binding.SH_F32, 0, 64) == -1
-    assert lib.sh_configure(h, binding.SH_BF16, 1, 64) == -2         # d_head 32 / d_model 128: fp32 only
+    hb = ctypes.c_void_p(lib.sh_create(192, 2, 32, 4, 2))
+    assert lib.sh_configure(hb, binding.SH_BF16, 1, 64) == -2        # d_model 192: not a multiple of 128
     assert "bf16" in binding.sh_last_error()
+    lib.sh_destroy(hb)
     assert lib.sh_configure(h, binding.SH_F32, 1, 64) == 0
     need = lib.sh_workspace_bytes(h)
     assert need > 0

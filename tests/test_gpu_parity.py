@@ -233,3 +233,19 @@ def test_noncausal_bf16_shapes(T, B, H, D):
 
 def test_noncausal_c4_262m_sampled():
     noncausal_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=3))
+
+
+# ---- d_head values that are stored padded (the paper's 76, 112, 100; odd and tiny ones) ------
+@pytest.mark.parametrize("dtype,D,T", [(inputs.DTYPE_F32, 76, 70), (inputs.DTYPE_F32, 5, 33), (inputs.DTYPE_BF16, 76, 200),
+                                       (inputs.DTYPE_BF16, 112, 515), (inputs.DTYPE_BF16, 100, 129), (inputs.DTYPE_BF16, 30, 64)])
+def test_padded_d_head(dtype, D, T):
+    cfg = inputs.LayerConfig("dpad", dtype, 2, T, 256, 2, D, 4, 2, seed=70 + D)
+    full_check(inputs.make_inputs(cfg))
+
+
+def test_padded_d_head_with_rope_and_shared_selection():
+    cfg = inputs.LayerConfig("dpad_rope", inputs.DTYPE_BF16, 2, 300, 256, 2, 100, 5, 3, seed=88)
+    rope_check(inputs.make_inputs(cfg))
+    full_check(inputs.make_inputs(cfg), shared_selection=True)
+    cfg = inputs.LayerConfig("dpad_rope_f32", inputs.DTYPE_F32, 1, 50, 128, 2, 22, 3, 2, seed=89)
+    rope_check(inputs.make_inputs(cfg))
