@@ -397,6 +397,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     } else {
       const int nq = (d.T + 255) / 256;
       const unsigned grid = (unsigned)(nq * d.B * d.H);
+      a.balanced = d.causal && (int)grid <= L->sm_count && !getenv("SH_ATTN_ADJACENT");
       if (d.D == 128) {
         if (!cfg2_128) { if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc; cfg2_128 = true; }
         if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;

@@ -18,6 +18,7 @@ struct TcAttnArgs {
   ShDims d;
   __half* ahat;          // [B*T, H, D]
   int* status;
+  int balanced;          // two-tile kernel: pair query tile p with tile ntile-1-p (grid fits the GPU in one wave)
 };
 
 template <int D>

@@ -4,7 +4,7 @@
 // CUDA cores the tensor pipe works for the other tile.
 //
 // CTA = (batch, head, 256 queries); key/value tiles of 128 up to the diagonal of each query
-// tile (tile 0: steps 0..2*qt, tile 1: steps 0..2*qt+1).
+// tile (tile 0: its steps 0..n0-1, tile 1: its steps 0..n1-1).
 // Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
 // warps 2..5 = softmax of query tile 0, warps 6..9 = softmax of query tile 1 (thread = query
 // row = TMEM lane).  TMEM columns: S0 at 0, S1 at 128, O0 at 256, O1 at 384.
@@ -56,13 +56,22 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = (d.T + 255) / 256;
   const int BH = d.B * d.H;
-  const int qt = nq - 1 - (int)(blockIdx.x / BH);        // heaviest query tiles first
   const int bh = blockIdx.x % BH;
-  const int q0 = qt * 256;
+  // The two 128-query tiles of this CTA.  Saturated grid: adjacent tiles, heaviest pairs first (the
+  // most steps in which both tiles share a K/V stage).  Grid that fits the GPU in one wave
+  // (g.balanced): tile p with tile ntile-1-p, so that under the causal mask every CTA has the same
+  // number of tile-steps and the kernel ends when the average CTA ends, not the heaviest.
+  const int ntile = (d.T + 127) / 128;
+  const int pr = (int)(blockIdx.x / BH);
+  int ta, tb;
+  if (g.balanced) { ta = pr; tb = ntile - 1 - pr; }
+  else { ta = 2 * (nq - 1 - pr); tb = ta + 1; }
+  const bool has_b = tb < ntile && tb != ta;
+  const int qrow[2] = {ta * 128, tb * 128};
   // key tiles each query tile attends to: up to its diagonal tile, or (d.causal == 0) all of them
-  const int nkt = (d.T + 127) / 128;
-  const int n0 = d.causal ? 2 * qt + 1 : nkt;            // steps of query tile 0
-  const int n1 = (q0 + 128 < d.T) ? (d.causal ? 2 * qt + 2 : nkt) : 0;   // steps of query tile 1 (0: no such rows)
+  const int nkt = ntile;
+  const int n0 = d.causal ? ta + 1 : nkt;                // steps of query tile 0
+  const int n1 = has_b ? (d.causal ? tb + 1 : nkt) : 0;  // steps of query tile 1 (0: no such tile)
   const int nsteps = n1 > n0 ? n1 : n0;
   bool dead = false;
 
@@ -93,7 +102,7 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       for (int t = 0; t < (n1 > 0 ? 2 : 1); ++t)
 #pragma unroll
         for (int c = 0; c < DB; ++c)
-          tma_load_3d(sbase + SM::Q_OFF + t * SM::T_BYTES + c * BLK, &mapQ, q_full, c * 64, q0 + t * 128, bh);
+          tma_load_3d(sbase + SM::Q_OFF + t * SM::T_BYTES + c * BLK, &mapQ, q_full, c * 64, qrow[t], bh);
       for (int j = 0; j < nsteps; ++j) {
         const int s = j & 1;
         if (!mbar_wait(&k_empty[s], ((j >> 1) & 1) ^ 1, g.status, dead)) break;
@@ -259,7 +268,7 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     }
     if (ok && n > 0 && mbar_wait(&pv_done[t], (n - 1) & 1, g.status, dead)) {
       tc_fence_after();
-      const int tq = q0 + t * 128 + r;
+      const int tq = qrow[t] + r;
       const float inv = 1.f / l;
       const int bb = bh / d.H, hh = bh % d.H;
       __half* dst = g.ahat + (((size_t)bb * d.T + tq) * d.H + hh) * D;
