@@ -383,7 +383,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   } else {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
-    static bool cfg128 = false, cfg64 = false, cfg2_128 = false, cfg2_64 = false;
+    static bool cfg128 = false, cfg64 = false;
     if (S->attn_single_tile && d.causal) {
       const int nq = (d.T + 127) / 128;
       const unsigned grid = (unsigned)(nq * d.B * d.H);
@@ -398,6 +398,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       const int nq = (d.T + 255) / 256;
       const unsigned grid = (unsigned)(nq * d.B * d.H);
       a.balanced = d.causal && (int)grid <= L->sm_count && !getenv("SH_ATTN_ADJACENT");
+      static bool cfg2_128 = false, cfg2_64 = false;
       if (d.D == 128) {
         if (!cfg2_128) { if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc; cfg2_128 = true; }
         if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;

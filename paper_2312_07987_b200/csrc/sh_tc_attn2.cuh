@@ -1,17 +1,22 @@
-// Causal softmax attention (Eq. 1 with the autoregressive mask) with TWO 128-query tiles per
-// CTA.  Both tiles read the same K/V stages, which halves the bytes pulled from L2 per FLOP -
-// the quantity that bounds the single-tile kernel - and while one tile's softmax runs on the
-// CUDA cores the tensor pipe works for the other tile.
+// Causal softmax attention (Eq. 1 with the autoregressive mask), two 128-query tiles per CTA,
+// with the probabilities P kept in tensor memory.
 //
-// CTA = (batch, head, 256 queries); key/value tiles of 128 up to the diagonal of each query
-// tile (tile 0: its steps 0..n0-1, tile 1: its steps 0..n1-1).
-// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer,
-// warps 2..5 = softmax of query tile 0, warps 6..9 = softmax of query tile 1 (thread = query
-// row = TMEM lane).  TMEM columns: S0 at 0, S1 at 128, O0 at 256, O1 at 384.
-// P (fp16) goes through ONE shared-memory buffer used alternately by the two tiles; the
-// k-th use ("phase") may be written once the UMMAs of phase k-1 have completed (p_free).
-// Running maximum and rescale as in the single-tile kernel (raise only by more than 8 in
-// log2 units; O rescaled in TMEM when that happens).
+// Per query tile: S = Q K^T lands in 128 TMEM columns (fp32); the tile's softmax warps read
+// their rows, and write P = exp2(S - m) back as packed fp16 into the first 64 of the SAME
+// columns (tcgen05.st); the product O += P V then takes its A operand from tensor memory
+// (tcgen05.mma with [a_tmem]).  The next S of the tile is issued right behind that product:
+// the tensor pipe executes in issue order, so it overwrites P only after the product has read
+// it, and no barrier is needed between the two.  Compared with P staged in shared memory
+// (the earlier version of this kernel) this drops 16 shared-memory stores and a proxy fence per thread and step,
+// the UMMA's shared-memory reads of P, and above all the single P buffer the two tiles had to
+// take turns on; the two tiles now interleave freely: while one tile's softmax runs, the pipe
+// works for the other.
+//
+// CTA = (batch, head, two query tiles); key/value tiles of 128 up to the diagonal of each
+// query tile.  Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA
+// issuer, warps 2..5 / 6..9 = softmax of query tile 0 / 1 (thread = query row = TMEM lane).
+// TMEM columns: S0 / P0 at 0, S1 / P1 at 128, O0 at 256, O1 at 384.  Running maximum and
+// rescale: raise only by more than 8 in log2 units; O rescaled in TMEM when that happens.
 #pragma once
 #include "sh_tc_attn.cuh"
 
@@ -20,12 +25,10 @@ namespace shtc {
 template <int D>
 struct Attn2Smem {
   static constexpr int T_BYTES = 128 * D * 2;            // one 128-row tile of Q, K or V
-  static constexpr int P_BYTES = 128 * 128 * 2;
   static constexpr int Q_OFF = 0;                          // 2 tiles
   static constexpr int K_OFF = Q_OFF + 2 * T_BYTES;        // 2 stages
   static constexpr int V_OFF = K_OFF + 2 * T_BYTES;        // 2 stages
-  static constexpr int P_OFF = V_OFF + 2 * T_BYTES;
-  static constexpr int BAR_OFF = P_OFF + P_BYTES;
+  static constexpr int BAR_OFF = V_OFF + 2 * T_BYTES;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;
 };
 
@@ -45,12 +48,10 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   uint64_t* k_empty = bars + 3;   // [2]
   uint64_t* v_full = bars + 5;    // [2]
   uint64_t* v_empty = bars + 7;   // [2]
-  uint64_t* s_full = bars + 9;    // [2] per query tile
-  uint64_t* s_empty = bars + 11;  // [2] per query tile
-  uint64_t* pv_done = bars + 13;  // [2] per query tile
-  uint64_t* p_full = bars + 15;
-  uint64_t* p_free = bars + 16;
-  uint32_t* tmem_slot = (uint32_t*)(bars + 17);
+  uint64_t* s_full = bars + 9;    // [2] per query tile: S of the step is in TMEM
+  uint64_t* p_full = bars + 11;   // [2] per query tile: P of the step is in TMEM (one arrival per softmax warp)
+  uint64_t* pv_done = bars + 13;  // [2] per query tile: the step's P V product has completed
+  uint32_t* tmem_slot = (uint32_t*)(bars + 15);
 
   const ShDims& d = g.d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -80,11 +81,9 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
-      mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 128);
+      mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4);
       mbar_init(&pv_done[i], 1);
     }
-    mbar_init(p_full, 128);
-    mbar_init(p_free, 1);
     fence_barrier_init();
     tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV);
   }
@@ -122,7 +121,7 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       constexpr uint32_t idesc_s = make_idesc_f16(128, 128, 0, 0, 0);
       constexpr uint32_t idesc_pv = make_idesc_f16(128, D, 0, 0, 1);
       const uint32_t q_lo0 = desc_lo_k(sbase + SM::Q_OFF), k_lo0 = desc_lo_k(sbase + SM::K_OFF);
-      const uint32_t p_lo = desc_lo_k(sbase + SM::P_OFF), v_lo0 = desc_lo_mn(sbase + SM::V_OFF, BLK);
+      const uint32_t v_lo0 = desc_lo_mn(sbase + SM::V_OFF, BLK);
       const int nt[2] = {n0, n1};
       auto issue_s = [&](int t, int j) {                     // S_t = Q_t K_j^T
         const uint32_t q_lo = q_lo0 + t * (SM::T_BYTES >> 4), k_lo = k_lo0 + (j & 1) * (SM::T_BYTES >> 4);
@@ -140,53 +139,38 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         if (n1 > 0) issue_s(1, 0);
         umma_commit(&k_empty[0]);
       }
-      uint32_t pp = 0;                                       // phase counter of the shared P buffer
       for (int j = 0; ok && j < nsteps; ++j) {
         const int s = j & 1;
-        // S of the NEXT step first: it only needs K(j+1) and the softmax warps to have read S(j) out
-        // of TMEM, so the next softmax can start while this step's P V products are still queued
-        if (j + 1 < nsteps) {
-          if (!mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, g.status, dead)) break;
-          for (int t = 0; t < 2 && ok; ++t) {
-            if (j + 1 >= nt[t]) continue;
-            if (!mbar_wait(&s_empty[t], j & 1, g.status, dead)) { ok = false; break; }
-            tc_fence_after();
-            issue_s(t, j + 1);
-          }
-          if (!ok) break;
-          umma_commit(&k_empty[(j + 1) & 1]);
-        }
+        const bool more = j + 1 < nsteps;
+        if (more && !mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, g.status, dead)) break;
         if (!mbar_wait(&v_full[s], (j >> 1) & 1, g.status, dead)) break;
         const uint32_t v_lo = v_lo0 + s * (SM::T_BYTES >> 4);
         for (int t = 0; t < 2 && ok; ++t) {
           if (j >= nt[t]) continue;
-          if (!mbar_wait(p_full, pp & 1, g.status, dead)) { ok = false; break; }
+          if (!mbar_wait(&p_full[t], j & 1, g.status, dead)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {                     // 128 keys in steps of 16
-            const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
-            umma_f16(tmem + 256 + t * 128, desc_pack(p_lo + koff), desc_pack(v_lo + k * (2048 >> 4)), idesc_pv, (j | k) != 0);
-          }
-          umma_commit(p_free);
+          for (int k = 0; k < 8; ++k)                       // 128 keys in steps of 16: A = P_t from tensor memory
+            umma_f16_tmem_a(tmem + 256 + t * 128, tmem + t * 128 + 8 * k, desc_pack(v_lo + k * (2048 >> 4)), idesc_pv, (j | k) != 0);
           umma_commit(&pv_done[t]);
-          ++pp;
+          // the tile's next S goes right behind: executed in issue order, it overwrites P_t only
+          // after the product above has read it
+          if (j + 1 < nt[t]) issue_s(t, j + 1);
         }
         if (!ok) break;
         umma_commit(&v_empty[s]);
+        if (more) umma_commit(&k_empty[(j + 1) & 1]);
       }
     }
   } else {
     // ---- softmax: warps 2..5 own query tile 0, warps 6..9 query tile 1; thread = query row ------
     const int t = (warp - 2) >> 2;
     const int n = t == 0 ? n0 : n1;
-    const int other = t == 0 ? n1 : n0;
     const int q = warp & 3;
     const int r = q * 32 + lane;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t tmem_s = tmem + t * 128, tmem_o = tmem + 256 + t * 128;
     float m = -INFINITY, l = 0.f;
-    const uint32_t prow = sbase + SM::P_OFF + r * 128;
-    const uint32_t sw = (uint32_t)(r & 7);
     bool ok = true;
     for (int j = 0; j < n; ++j) {
       if (!mbar_wait(&s_full[t], j & 1, g.status, dead)) { ok = false; break; }
@@ -195,8 +179,6 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + lane_off + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
-      tc_fence_before();
-      mbar_arrive(&s_empty[t]);
       if (j == n - 1) {
         // last tile: the diagonal one (key c visible iff c <= r), or without the causal mask the
         // tile that holds the end of the sequence (keys past it were zero-filled by the loads)
@@ -221,30 +203,22 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         m = mx;
         raise = j > 0;
       }
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 negm = make_float2(-m, -m);
       uint32_t pk[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) {
-        const float p0 = fast_exp2(__uint_as_float(sv[2 * c]) - m);
-        const float p1 = fast_exp2(__uint_as_float(sv[2 * c + 1]) - m);
-        sum4[c & 3] += p0 + p1;
-        __half2 h = __floats2half2_rn(p0, p1);
+        const float2 x = __fadd2_rn(make_float2(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1])), negm);
+        float2 pr;
+        pr.x = fast_exp2(x.x);
+        pr.y = fast_exp2(x.y);
+        sum2[c & 1] = __fadd2_rn(sum2[c & 1], pr);
+        __half2 h = __floats2half2_rn(pr.x, pr.y);
         pk[c] = *reinterpret_cast<uint32_t*>(&h);
       }
-      l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-      // phase of the shared P buffer this write is: tile 0 step j comes after min(j, n1) writes of
-      // tile 1; tile 1 step j after min(j + 1, n0) writes of tile 0
-      const int phase = j + (t == 0 ? (j < other ? j : other) : (j + 1 < other ? j + 1 : other));
-      // This group's own previous P V product first: a parity wait cannot tell phase p from phase
-      // p - 2, and without this the group could reach the p_free wait below while p_free is still
-      // two phases back (the issuer queues the next S before this step's P V), pass it on the stale
-      // phase and overwrite P under a running product.
-      if (j > 0 && !mbar_wait(&pv_done[t], (j - 1) & 1, g.status, dead)) { ok = false; break; }
-      if (phase > 0) {
-        if (!mbar_wait(p_free, (phase - 1) & 1, g.status, dead)) { ok = false; break; }
-        tc_fence_after();
-      }
+      l = l * alpha + ((sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y));
       if (j > 0 && __any_sync(0xffffffffu, raise)) {         // rescale this warp's 32 rows of O
+        // (S of this step was issued behind the previous P V product, so that product has completed)
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t ov[32];
@@ -254,17 +228,14 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
           tmem_st32(tmem_o + lane_off + c * 32, ov);
         }
-        tmem_st_wait();
       }
-#pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        const uint32_t addr = prow + (ch >> 3) * BLK + (((uint32_t)(ch & 7) ^ sw) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]),
-                     "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3]) : "memory");
-      }
-      fence_proxy_async_smem();
+      // P (packed fp16 pairs) over the first 64 columns of this row's S
+      tmem_st32(tmem_s + lane_off, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tmem_st32(tmem_s + lane_off + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(p_full);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[t]);
     }
     if (ok && n > 0 && mbar_wait(&pv_done[t], (n - 1) & 1, g.status, dead)) {
       tc_fence_after();
