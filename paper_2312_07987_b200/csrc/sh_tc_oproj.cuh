@@ -186,9 +186,9 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
       }
       mbar_arrive(sel_ready);
       if (!mbar_wait(sel_ready, wpar, g.status, dead)) { ok = false; break; }
-      float acc[128];
+      float2 acc2[64];                                     // packed fp32 pairs: one FFMA2 per two features
 #pragma unroll
-      for (int f = 0; f < 128; ++f) acc[f] = 0.f;
+      for (int f = 0; f < 64; ++f) acc2[f] = make_float2(0.f, 0.f);
       for (int h = 0; h < d.H && ok; ++h) {
         const int sel = (tok * d.H + h) * d.k;               // this token's selections for head h
         for (int e = 0; e < d.E; ++e, ++ge) {
@@ -209,8 +209,10 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
               __syncwarp();                                  // one arrival per warp: 256 arrivals on one barrier
               if (lane == 0) mbar_arrive(&d_empty[buf]);     // word would serialise in the LSU
             }
+            const float2 g2 = make_float2(gv, gv);
 #pragma unroll
-            for (int f = 0; f < 32; ++f) acc[c * 32 + f] = fmaf(gv, __uint_as_float(v[f]), acc[c * 32 + f]);
+            for (int f = 0; f < 16; ++f)
+              acc2[c * 16 + f] = __ffma2_rn(g2, make_float2(__uint_as_float(v[2 * f]), __uint_as_float(v[2 * f + 1])), acc2[c * 16 + f]);
           }
         }
       }
@@ -227,7 +229,7 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch)                     // 16-byte chunk ch of row `lane` sits at chunk ch ^ (lane & 7)
             *reinterpret_cast<float4*>(stg + lane * 32 + ((ch ^ (lane & 7)) << 2)) =
-                make_float4(acc[c * 32 + 4 * ch], acc[c * 32 + 4 * ch + 1], acc[c * 32 + 4 * ch + 2], acc[c * 32 + 4 * ch + 3]);
+                make_float4(acc2[c * 16 + 2 * ch].x, acc2[c * 16 + 2 * ch].y, acc2[c * 16 + 2 * ch + 1].x, acc2[c * 16 + 2 * ch + 1].y);
           __syncwarp();
           // 8 lanes cover one row's 128 bytes, a warp instruction four rows
 #pragma unroll
