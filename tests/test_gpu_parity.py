@@ -249,3 +249,13 @@ def test_padded_d_head_with_rope_and_shared_selection():
     full_check(inputs.make_inputs(cfg), shared_selection=True)
     cfg = inputs.LayerConfig("dpad_rope_f32", inputs.DTYPE_F32, 1, 50, 128, 2, 22, 3, 2, seed=89)
     rope_check(inputs.make_inputs(cfg))
+
+
+# ---- launch-structure switches (A/B aids): same numbers with ordinary launches on one stream ----
+@pytest.mark.parametrize("env", [{"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
+                                 {"SH_ATTN_ADJACENT": "1"}])
+def test_launch_structure_switches_keep_the_result(env, monkeypatch):
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)                           # read when the weights are set / at launch
+    full_check(inputs.make_inputs(inputs.CONFIGS["small_bf16"]))
+    full_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=3), check_stage_buffers=False)
