@@ -239,11 +239,9 @@ static int launch_gate_sort(sh_layer* L, const void* x, cudaStream_t st) {
       (const float*)(ws + L->o.gbias), (int*)(ws + L->o.idx), (float*)(ws + L->o.gate),
       (int*)(ws + L->o.blockcnt), d);
   const size_t ssm = sh_sort_smem_bytes(d);
-  static size_t sort_cfg = 48 * 1024;
-  if (ssm > sort_cfg) {
+  // (set on every call that needs it: the attribute belongs to the current device's copy of the function)
+  if (ssm > 48 * 1024)
     SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
-    sort_cfg = ssm;
-  }
   sh_sort_kernel<<<d.nblk, sh_sort_threads(d), ssm, st>>>((const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate),
       (const int*)(ws + L->o.blockcnt), (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists),
       (float*)(ws + L->o.lgate), (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), d);

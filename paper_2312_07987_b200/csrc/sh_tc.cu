@@ -106,13 +106,31 @@ static int launch_k(bool pdl, void (*kern)(P...), dim3 grid, dim3 block, size_t 
   return SH_OK;
 }
 
+// Dynamic shared memory limit and carve-out of a kernel, set once per (kernel, device, size): the
+// attributes belong to the device's copy of the function, so a process that drives several GPUs
+// must set them on each.  Always the largest shared-memory carve-out: kernels of one forward pass
+// share SMs (a sort block beside a GEMM CTA; the next kernel's CTAs arriving while this one
+// drains), and an SM set up with a smaller carve-out has to run empty before it can be set up again.
+struct SmemAttr { const void* fn; int dev; int bytes; };
+static SmemAttr g_smem_attr[128];
+static int g_smem_attr_n = 0;
+
 template <typename K>
 static int set_smem(K kernel, int bytes) {
-  SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  // Always the largest shared-memory carve-out: kernels of one forward pass share SMs (a sort block
-  // beside a GEMM CTA; the next kernel's CTAs arriving while this one drains), and an SM set up
-  // with a smaller carve-out has to run empty before it can be set up again.
-  SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  int dev = 0;
+  SH_CUDA_CHECK(cudaGetDevice(&dev));
+  const void* fn = (const void*)kernel;
+  SmemAttr* slot = nullptr;
+  for (int i = 0; i < g_smem_attr_n; ++i)
+    if (g_smem_attr[i].fn == fn && g_smem_attr[i].dev == dev) slot = &g_smem_attr[i];
+  if (slot && slot->bytes >= bytes) return SH_OK;
+  if (bytes > 48 * 1024 || !slot)
+    SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes > 48 * 1024 ? bytes : 48 * 1024));
+  if (!slot) {
+    SH_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    if (g_smem_attr_n < 128) slot = &g_smem_attr[g_smem_attr_n++];
+  }
+  if (slot) { slot->fn = fn; slot->dev = dev; slot->bytes = bytes; }
   return SH_OK;
 }
 
@@ -226,27 +244,12 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.status = (int*)(ws + L->o.status);
   const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
   const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
-  static int configured[2] = {0, 0};
-  if (configured[deep] < smem) {
-    if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
-    configured[deep] = smem;
-  }
+  if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
   if (deep) sh_tc_gate_kernel<8><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
   else sh_tc_gate_kernel<4><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
   const size_t ssm = sh_sort_smem_bytes(d);
-  static size_t sort_cfg = 48 * 1024;
-  static bool sort_carveout = false;
-  if (!sort_carveout) {
-    // Sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow: ask for
-    // the largest shared-memory carve-out, or an SM that a sort block configured would have to
-    // drain before such a CTA could join it.
-    SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
-    sort_carveout = true;
-  }
-  if (ssm > sort_cfg) {
-    SH_CUDA_CHECK(cudaFuncSetAttribute(sh_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
-    sort_cfg = ssm;
-  }
+  // (sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow)
+  if ((rc = set_smem(sh_sort_kernel, (int)ssm))) return rc;
   // In a forward pass only the value experts read sorted lists (the output projection works from
   // idx / gate, token tile by token tile), so only the source side is sorted there -- unless the
   // scatter-add or CUDA-core output projection (debugging paths) is selected.  The histogram stride
@@ -271,12 +274,7 @@ template <int BN, int STAGES, int MODE, int MT>
 static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, unsigned grid, cudaStream_t st, bool pdl) {
   auto kern = sh_tc_pgemm_kernel<BN, STAGES, MODE, MT>;
   constexpr int smem = PGemmSmem<BN, STAGES, MT>::TOTAL;
-  static bool configured = false;
-  if (!configured) {
-    int rc = set_smem(kern, smem);
-    if (rc != SH_OK) return rc;
-    configured = true;
-  }
+  if (int rc = set_smem(kern, smem)) return rc;
   return launch_k(pdl, kern, dim3(grid), dim3(320), smem, st, mapA, mapB, g);
 }
 
@@ -284,12 +282,7 @@ template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>
 static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, dim3 grid, cudaStream_t st) {
   auto kern = sh_tc_gemm_kernel<BN, STAGES, MODE, A_BF16, B_BF16, MT>;
   constexpr int smem = GemmSmem<BN, STAGES, MT>::TOTAL;
-  static bool configured = false;
-  if (!configured) {
-    int rc = set_smem(kern, smem);
-    if (rc != SH_OK) return rc;
-    configured = true;
-  }
+  if (int rc = set_smem(kern, smem)) return rc;
   kern<<<grid, 192, smem, st>>>(mapA, mapB, g);
   return SH_OK;
 }
@@ -383,27 +376,25 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   } else {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
-    static bool cfg128 = false, cfg64 = false;
     if (S->attn_single_tile && d.causal) {
       const int nq = (d.T + 127) / 128;
       const unsigned grid = (unsigned)(nq * d.B * d.H);
       if (d.D == 128) {
-        if (!cfg128) { if ((rc = set_smem(sh_tc_attention_kernel<128>, AttnSmem<128>::TOTAL))) return rc; cfg128 = true; }
+        if ((rc = set_smem(sh_tc_attention_kernel<128>, AttnSmem<128>::TOTAL))) return rc;
         sh_tc_attention_kernel<128><<<grid, 192, AttnSmem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
       } else {
-        if (!cfg64) { if ((rc = set_smem(sh_tc_attention_kernel<64>, AttnSmem<64>::TOTAL))) return rc; cfg64 = true; }
+        if ((rc = set_smem(sh_tc_attention_kernel<64>, AttnSmem<64>::TOTAL))) return rc;
         sh_tc_attention_kernel<64><<<grid, 192, AttnSmem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
       }
     } else {
       const int nq = (d.T + 255) / 256;
       const unsigned grid = (unsigned)(nq * d.B * d.H);
       a.balanced = d.causal && (int)grid <= L->sm_count && !getenv("SH_ATTN_ADJACENT");
-      static bool cfg2_128 = false, cfg2_64 = false;
       if (d.D == 128) {
-        if (!cfg2_128) { if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc; cfg2_128 = true; }
+        if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc;
         if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
       } else {
-        if (!cfg2_64) { if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc; cfg2_64 = true; }
+        if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc;
         if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<64>, dim3(grid), dim3(320), Attn2Smem<64>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
       }
     }
@@ -439,7 +430,6 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
     }
     const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
-    static int cfg_smem128 = 0, cfg_smem64 = 0;
     int as = 3, smem = 0;
     for (; as >= 2; --as) {
       smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.k) : OprojSmem<64>::total(as, d.H, d.k);
@@ -448,10 +438,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     if (as < 2) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
     a.a_slots = as;
     if (d.D == 128) {
-      if (cfg_smem128 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc; cfg_smem128 = smem; }
+      if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc;
       if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<128>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
     } else {
-      if (cfg_smem64 < smem) { if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc; cfg_smem64 = smem; }
+      if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc;
       if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<64>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
     }
     L->launches += 1;
