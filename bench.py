@@ -236,20 +236,25 @@ def main():
         stage += np.array(layer.sh_forward_timed(x, out))
     stage /= reps
 
-    # ---- end to end through the C ABI with host buffers ----
-    xh = x.cpu().pin_memory()
-    outh = torch.empty(inp.x.shape, dtype=torch.float32).pin_memory()
-    xd = torch.empty_like(x)
-    for _ in range(2):
-        xd.copy_(xh, non_blocking=True); layer.sh_forward(xd, out); outh.copy_(out, non_blocking=True)
+    # ---- end to end with host buffers: every step copies x in from pinned host memory and the
+    # result back out; the three run as a pipeline on three streams (pipeline.HostFedLayer), as a
+    # host-fed caller would run them ----
+    from paper_2312_07987_b200 import pipeline
+    xh = [x.cpu().pin_memory() for _ in range(2)]
+    outh = [torch.empty(inp.x.shape, dtype=torch.float32).pin_memory() for _ in range(2)]
+    pipe = pipeline.HostFedLayer(layer, x)
+    for i in range(4):
+        pipe.step(xh[i & 1], outh[i & 1])
+    pipe.wait()
+    assert torch.equal(outh[1], out.cpu()) or float((outh[1] - out.cpu()).abs().max()) < 1e-2 * float(out.abs().max()), \
+        "pipelined result differs from the direct one"
     barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for _ in range(args.steps):
-        xd.copy_(xh, non_blocking=True)
-        layer.sh_forward(xd, out)
-        outh.copy_(out, non_blocking=True)
-    b.record(stream)
+    a.record(pipe.s_in)
+    for i in range(args.steps):
+        pipe.step(xh[i & 1], outh[i & 1])
+    b.record(pipe.s_out)
+    pipe.wait()
     barrier()
     e2e_ms = a.elapsed_time(b)
     assert layer.sh_last_status() == 0, "device status word set during the timed region"
