@@ -10,7 +10,7 @@
 #include "sh_tc_attn.cuh"
 #include "sh_tc_attn2.cuh"
 #include "sh_tc_gate.cuh"
-#include "sh_tc_oproj.cuh"
+#include "sh_tc_oproj2.cuh"
 
 using namespace shtc;
 
@@ -77,6 +77,7 @@ struct TcState {
   CUtensorMap map_wqk, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
   int qk_bn, o_bn, qk_variant;
+  int o_pair, o_pairs_max;       // output projection on CTA pairs; clusters the device holds at once
   int persistent;       // 1 = persistent Q/K and value-expert GEMMs (default); 0 = one CTA per tile (experiment switch)
   int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
   int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
@@ -104,6 +105,35 @@ static int launch_k(bool pdl, void (*kern)(P...), dim3 grid, dim3 block, size_t 
   cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
   SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...));
   return SH_OK;
+}
+
+// The same for a kernel that runs as clusters of two CTAs (grid.x even).
+template <typename... P, typename... A>
+static int launch_k_pairs(bool pdl, void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl ? 2 : 1;
+  SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...));
+  return SH_OK;
+}
+
+// How many two-CTA clusters of a kernel the device holds at once (0 on error).
+template <typename K>
+static int max_pairs(K kern, int block, size_t smem) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n;
 }
 
 // Dynamic shared memory limit and carve-out of a kernel, set once per (kernel, device, size): the
@@ -173,6 +203,8 @@ int sh_tc_prepare(sh_layer* L) {
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_join, cudaEventDisableTiming));
   }
   S->o_bn = 128;
+  S->o_pair = getenv("SH_O_SINGLE") == nullptr;     // CTA-pair output projection unless switched off
+  S->o_pairs_max = 0;
   const char* env = getenv("SH_SIMT_STAGES");
   S->simt_mask = env ? atoi(env) : 0;
   if (L->sm_count == 0) {
@@ -428,6 +460,34 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       int dev = 0;
       SH_CUDA_CHECK(cudaGetDevice(&dev));
       SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    // The CTA-pair kernel rounds the gate-scaled token rows to fp16 once more than the single-CTA
+    // kernel; with k >= 4 the k-way fp16 sum of the value stage already uses most of the output
+    // tolerance, so those shapes keep the single-CTA kernel (as does a device that cannot hold a
+    // two-CTA cluster of this size).
+    bool pair = S->o_pair && d.k <= 3;
+    if (pair) {
+      const int psm = d.D == 128 ? OprojPairSmem<128>::TOTAL : OprojPairSmem<64>::TOTAL;
+      if (d.D == 128) { if ((rc = set_smem(sh_tc_oproj_pair_kernel<128>, psm))) return rc; }
+      else if ((rc = set_smem(sh_tc_oproj_pair_kernel<64>, psm))) return rc;
+      if (S->o_pairs_max == 0) {
+        S->o_pairs_max = d.D == 128 ? max_pairs(sh_tc_oproj_pair_kernel<128>, 480, psm) : max_pairs(sh_tc_oproj_pair_kernel<64>, 480, psm);
+        if (S->o_pairs_max <= 0) S->o_pairs_max = -1;
+      }
+      if (S->o_pairs_max < 0) pair = false;
+      else {
+        // 256 tokens x 256 features per unit, gates folded into the A operand
+        a.nwork = ((d.N + 255) / 256) * ((d.M + 255) / 256);
+        const unsigned pgrid = 2u * (unsigned)(a.nwork < S->o_pairs_max ? a.nwork : S->o_pairs_max);
+        const __half* ahat = (const __half*)(ws + L->o.ahat);
+        if (d.D == 128) rc = launch_k_pairs(pdl && (S->pdl_mask & 16), sh_tc_oproj_pair_kernel<128>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
+        else rc = launch_k_pairs(pdl && (S->pdl_mask & 16), sh_tc_oproj_pair_kernel<64>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
+        if (rc) return rc;
+        L->launches += 1;
+        sh_mark(L, 5, st);
+        SH_CUDA_CHECK(cudaGetLastError());
+        return SH_OK;
+      }
     }
     const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
     int as = 3, smem = 0;

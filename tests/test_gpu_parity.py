@@ -253,9 +253,16 @@ def test_padded_d_head_with_rope_and_shared_selection():
 
 # ---- launch-structure switches (A/B aids): same numbers with ordinary launches on one stream ----
 @pytest.mark.parametrize("env", [{"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
-                                 {"SH_ATTN_ADJACENT": "1"}])
+                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}])
 def test_launch_structure_switches_keep_the_result(env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)                           # read when the weights are set / at launch
     full_check(inputs.make_inputs(inputs.CONFIGS["small_bf16"]))
     full_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=3), check_stage_buffers=False)
+
+
+def test_pair_output_projection_ragged_tokens_and_features():
+    # CTA-pair output projection: N = 300 is not a multiple of the pair's 256 tokens (the second CTA of
+    # the last pair owns 44 tokens, and with N = 100 none at all), d_model = 384 or 128 not of its 256 features
+    full_check(inputs.make_inputs(inputs.LayerConfig("pair_ragged", inputs.DTYPE_BF16, 2, 150, 384, 2, 64, 4, 2, seed=90)))
+    full_check(inputs.make_inputs(inputs.LayerConfig("pair_half_empty", inputs.DTYPE_BF16, 1, 100, 128, 3, 128, 3, 1, seed=91)))
