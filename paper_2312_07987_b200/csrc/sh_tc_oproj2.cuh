@@ -11,21 +11,25 @@
 // accumulate into ONE tensor-memory buffer; the pipe runs without a per-expert hand-over, and the
 // other buffer is read out and stored by separate epilogue warps while the next unit accumulates.
 // The sum still never leaves the SM, out is written exactly once, and the result does not depend on
-// timing (one issuing thread, fixed order).
+// timing (the UMMAs are issued in a fixed order).  The price is one more fp16 rounding (of gate x
+// Ahat) than the single-CTA kernel makes.
 //
 // CTA pair (cluster of two, tcgen05 cta_group::2): work unit = 256 consecutive tokens x 256 output
 // features; each CTA owns 128 of the tokens (its scaled tiles, its accumulators, its stores) and
 // loads only its half of every expert's 256 weight rows - the pair's tensor cores read both halves.
 //
 // Roles per CTA (480 threads): warp 0 lane 0 = TMA producer (weights), warp 1 = TMEM allocation; in
-// the leader (even CTA) lane 0 of warps 1 and 14 = UMMA issuers for the pair; warps 2..9 = builders (thread = one
-// token x half of the head's D columns: Ahat row from global memory into registers one head ahead,
-// per expert a scaled copy into the stage's 128-byte-swizzled K-major tile); warps 10..13 =
-// epilogue (thread = one token, TMEM -> transpose in shared memory -> 16-byte coalesced stores).
-// Two rings: weights in 64-column blocks of this CTA's 128 feature rows (16 KB, seven stages: a TMA
-// load from L2 takes ~1 us, two experts' worth of tensor work, so three experts are kept in flight)
-// and scaled token tiles (128 x D, three stages: a tile is rebuilt ~1000 cycles after the UMMAs that
-// read it complete).  The issuing thread waits for each weight block (leader's barrier: the pair's
+// the leader (even CTA) lane 0 of warps 1 and 14 = UMMA issuers for the pair (they alternate, see
+// below); warps 2..9 = builders (thread = one token x half of the head's D columns: Ahat row from
+// global memory into registers one head ahead, per expert a scaled copy into the stage's
+// 128-byte-swizzled K-major tile); warps 10..13 = epilogue (thread = one token, TMEM -> transpose
+// in shared memory -> 16-byte coalesced stores).
+// Two rings: weights in 64-column blocks of this CTA's 128 feature rows (16 KB, five stages: a TMA
+// load from L2 takes ~1 us, two experts' worth of tensor work) and scaled token tiles (128 x D, four
+// stages: a tile is rebuilt ~1000 cycles after the UMMAs that read it complete, and those may wait
+// in the pipe's queue behind the expert before).  Together with the epilogue's staging that is all
+// of the 227 KB; of the splits that fit (7 + 3, 5 + 4, four 32 KB weight stages + 2 tiles) this one
+// measured best.  An issuing thread waits for each weight block (leader's barrier: the pair's
 // bytes) and once per expert for the tile (leader's barrier: one arrival per builder warp of both
 // CTAs), and commits each to the empty barrier of both CTAs (multicast).
 #pragma once
@@ -39,10 +43,33 @@ template <int D>
 struct OprojPairSmem {
   static constexpr int W_BYTES = 128 * 64 * 2;           // one 64-column block of this CTA's 128 feature rows of an expert
   static constexpr int P_BYTES = 128 * D * 2;            // scaled token tile: this CTA's 128 tokens x D
-  static constexpr int WST = 7, PST = 3;                 // ring depths
+  static constexpr int WST = 5, PST = 4;                 // ring depths
   static constexpr int STAGING = 4 * 32 * 32 * 4;        // per epilogue warp a 32 x 32 fp32 transpose tile
   static constexpr int TOTAL = WST * W_BYTES + PST * P_BYTES + STAGING + 512 + 1024;
 };
+
+// One 32-column chunk of a unit's accumulator: TMEM -> registers -> 32 x 32 transpose in shared
+// memory (token-per-lane -> 128-byte row segments) -> 16-byte coalesced stores.  One warp; stg = its
+// 4 KB of staging; obase = out + (first of the warp's 32 tokens) * M + the unit's first feature.
+__device__ __forceinline__ void oproj_store_chunk(uint32_t taddr, int c, float* stg, float* obase, int M, int rows_here, bool cols_live, int lane) {
+  uint32_t v[32];
+  tmem_ld32(taddr + c * 32, v);
+  tmem_ld_wait();
+  __syncwarp();
+#pragma unroll
+  for (int ch = 0; ch < 8; ++ch)                           // 16-byte chunk ch of row `lane` sits at chunk ch ^ (lane & 7)
+    *reinterpret_cast<uint4*>(stg + lane * 32 + ((ch ^ (lane & 7)) << 2)) = make_uint4(v[4 * ch], v[4 * ch + 1], v[4 * ch + 2], v[4 * ch + 3]);
+  __syncwarp();
+  if (cols_live) {
+#pragma unroll
+    for (int r4 = 0; r4 < 32; r4 += 4) {
+      const int r = r4 + (lane >> 3), ch = lane & 7;
+      if (r < rows_here)
+        *reinterpret_cast<float4*>(obase + (size_t)r * M + c * 32 + 4 * ch) =
+            *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2));
+    }
+  }
+}
 
 template <int D>
 __global__ void __launch_bounds__(480, 1)
@@ -50,6 +77,7 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
   using SM = OprojPairSmem<D>;
   constexpr int DB = D / 64;                             // 64-column (128-byte) blocks per row
   constexpr int WST = SM::WST, PST = SM::PST;
+  static_assert(WST <= 8 && PST <= 4, "barrier slots");
   constexpr uint32_t TBLK = 128 * 128;                   // one 64-column block of a 128-row tile
   constexpr int CH = D / 16;                             // 16-byte chunks per builder thread (half a row)
   extern __shared__ unsigned char smem_raw[];
@@ -58,10 +86,10 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
   const ShDims& d = g.d;
   constexpr uint32_t w_off = 0, p_off = WST * SM::W_BYTES, stg_off = p_off + PST * SM::P_BYTES, misc_off = stg_off + SM::STAGING;
   uint64_t* bars = (uint64_t*)(sgen + misc_off);
-  uint64_t* w_full = bars;               // [7] leader's: the pair's bytes of one weight block
-  uint64_t* w_empty = bars + 8;          // [7] both CTAs (multicast commit)
-  uint64_t* p_full = bars + 16;          // [3] leader's: 16 arrivals (builder warps of both CTAs)
-  uint64_t* p_empty = bars + 20;         // [3] both CTAs (multicast commit)
+  uint64_t* w_full = bars;               // [WST] leader's: the pair's bytes of one weight block
+  uint64_t* w_empty = bars + 8;          // [WST] both CTAs (multicast commit)
+  uint64_t* p_full = bars + 16;          // [PST] leader's: 16 arrivals (builder warps of both CTAs)
+  uint64_t* p_empty = bars + 20;         // [PST] both CTAs (multicast commit)
   uint64_t* d_full = bars + 24;          // [2] both CTAs (multicast commit): a unit's accumulator is complete
   uint64_t* d_empty = bars + 26;         // [2] leader's: 8 arrivals (epilogue warps of both CTAs)
   uint64_t* turn = bars + 28;            // [2] leader's: the token of the two issuing threads
@@ -242,28 +270,11 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
       float* obase = g.out + (size_t)(row0 + q * 32) * d.M + fc * 256;
 #pragma unroll 1
       for (int c = 0; c < 8; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_off + buf * 256 + c * 32, v);
-        tmem_ld_wait();
-        if (c == 7) {                                      // everything is in registers: hand the accumulator back
+        oproj_store_chunk(tmem + lane_off + buf * 256, c, stg, obase, d.M, rows_here, fc * 256 + c * 32 < d.M, lane);
+        if (c == 7) {                                      // everything has been read: hand the accumulator back
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_leader(&d_empty[buf]);
-        }
-        // 32 x 32 transpose through shared memory: token-per-lane -> 128-byte row segments
-        __syncwarp();
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch)                     // 16-byte chunk ch of row `lane` sits at chunk ch ^ (lane & 7)
-          *reinterpret_cast<uint4*>(stg + lane * 32 + ((ch ^ (lane & 7)) << 2)) = make_uint4(v[4 * ch], v[4 * ch + 1], v[4 * ch + 2], v[4 * ch + 3]);
-        __syncwarp();
-        if (fc * 256 + c * 32 < d.M) {
-#pragma unroll
-          for (int r4 = 0; r4 < 32; r4 += 4) {
-            const int r = r4 + (lane >> 3), ch = lane & 7;
-            if (r < rows_here)
-              *reinterpret_cast<float4*>(obase + (size_t)r * d.M + c * 32 + 4 * ch) =
-                  *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2));
-          }
         }
       }
     }
