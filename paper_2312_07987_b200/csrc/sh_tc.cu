@@ -11,6 +11,7 @@
 #include "sh_tc_attn2.cuh"
 #include "sh_tc_gate.cuh"
 #include "sh_tc_oproj2.cuh"
+#include "sh_tc_qkpair.cuh"
 
 using namespace shtc;
 
@@ -74,10 +75,11 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
-  CUtensorMap map_wqk, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
+  CUtensorMap map_wqk, map_wqk128, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
   int qk_bn, o_bn, qk_variant;
   int o_pair, o_pairs_max;       // output projection on CTA pairs; clusters the device holds at once
+  int qk_pair, qk_pairs_max;     // the same for the dense Q/K projection
   int persistent;       // 1 = persistent Q/K and value-expert GEMMs (default); 0 = one CTA per tile (experiment switch)
   int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
   int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
@@ -87,7 +89,8 @@ struct TcState {
   bool pdl = true;
   int pdl_mask = 31;
   cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_join2 = nullptr;
+  cudaStream_t side2 = nullptr;   // second grid of a split Q/K projection
 };
 
 constexpr int QK_STAGES = 4;
@@ -170,6 +173,8 @@ void sh_tc_release(sh_layer* L) {
     if (S->ev_fork) cudaEventDestroy(S->ev_fork);
     if (S->ev_join) cudaEventDestroy(S->ev_join);
     if (S->side) cudaStreamDestroy(S->side);
+    if (S->ev_join2) cudaEventDestroy(S->ev_join2);
+    if (S->side2) cudaStreamDestroy(S->side2);
     delete S;
     L->tc = nullptr;
   }
@@ -201,10 +206,14 @@ int sh_tc_prepare(sh_layer* L) {
     SH_CUDA_CHECK(cudaStreamCreateWithFlags(&S->side, cudaStreamNonBlocking));
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_fork, cudaEventDisableTiming));
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_join, cudaEventDisableTiming));
+    SH_CUDA_CHECK(cudaStreamCreateWithFlags(&S->side2, cudaStreamNonBlocking));
+    SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_join2, cudaEventDisableTiming));
   }
   S->o_bn = 128;
   S->o_pair = getenv("SH_O_SINGLE") == nullptr;     // CTA-pair output projection unless switched off
   S->o_pairs_max = 0;
+  S->qk_pair = getenv("SH_QK_SINGLE") == nullptr;
+  S->qk_pairs_max = 0;
   const char* env = getenv("SH_SIMT_STAGES");
   S->simt_mask = env ? atoi(env) : 0;
   if (L->sm_count == 0) {
@@ -222,6 +231,7 @@ int sh_tc_prepare(sh_layer* L) {
   L->d.tile_rows_src = (L->dense || (S->simt_mask & SH_STAGE_V) || getenv("SH_V_TILE128") || !big || dst_reads_src_tiles) ? 128 : 256;
   int rc;
   if ((rc = sh_tc_encode_2d(&S->map_wqk, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, S->qk_bn))) return rc;
+  if ((rc = sh_tc_encode_2d(&S->map_wqk128, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, 128))) return rc;
   if (!L->dense) {
     if ((rc = sh_tc_encode_2d(&S->map_wv, 0, ws + L->o.wv, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, S->o_bn))) return rc;
@@ -339,15 +349,61 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     SH_CUDA_CHECK(cudaStreamWaitEvent(S->side, S->ev_fork, 0));
     qst = S->side;
   }
+  CUtensorMap map_x;
+  if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
+  // Split Q/K projection.  A grid whose CTAs cannot all start at once (the gate kernel holds SMs)
+  // keeps every kernel launched after it, in any stream, from starting: the sort kernel, launched to
+  // become resident while the gate kernel runs, then starts ~4 us after the gate kernel has ended.
+  // And launched after gate and sort, the projection starts two launch latencies late when the
+  // host is not running ahead (a single forward pass: ~100 us instead of ~107).  So the projection goes
+  // out as two grids of CTA pairs that claim tiles from one counter: grid A, launched BEFORE the
+  // gate kernel, sized for the SMs the gate kernel does not need; grid B, launched AFTER the sort
+  // kernel on a stream of its own, takes over the gate kernel's SMs when they come free.
+  int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
+  TcGemmArgs qg{};
+  if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_variant == 2 && S->persistent && S->qk_pair && S->side2 &&
+      !getenv("SH_QK_ONE_GRID")) {
+    using PS = QkPairSmem<6>;
+    if ((rc = set_smem(sh_tc_qk_pair_kernel<6>, PS::TOTAL))) return rc;
+    if (S->qk_pairs_max == 0) {
+      S->qk_pairs_max = max_pairs(sh_tc_qk_pair_kernel<6>, 320, PS::TOTAL);
+      if (S->qk_pairs_max <= 0) S->qk_pairs_max = -1;
+    }
+    if (S->qk_pairs_max > 0) {
+      const int ptiles = ((d.N + 255) / 256) * ((2 * HD + 255) / 256);
+      const int pairs = ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max;
+      // (one gate CTA per SM; running two per SM with half the stages, to leave grid A more SMs when
+      //  there are more gate CTAs than half the SMs, made the gate kernel 2.4 us slower and the layer
+      //  8-10 us slower at 16384 tokens)
+      int gate_sms = d.nblk;
+      if (gate_sms > L->sm_count - 8) gate_sms = L->sm_count - 8;
+      qkA = (L->sm_count - gate_sms) / 2;
+      if (qkA > pairs) qkA = pairs;
+      qkB = pairs - qkA;
+      qg.d = d; qg.K = d.M; qg.ncols = 2 * HD; qg.nrows = d.N;
+      qg.out0 = ws + L->o.q; qg.out1 = ws + L->o.k; qg.out2 = ws + L->o.v;
+      qg.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+      qg.status = status; qg.sched = status + 16; qg.claimers = qkA + qkB;
+      qg.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
+      if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkA), dim3(320), PS::TOTAL, S->side, map_x, S->map_wqk128, qg))) return rc;
+      L->launches += 1;
+    }
+  }
   if (!L->dense) {
     if ((rc = tc_gate_sort(L, x, out, true, st))) return rc;
   }
   sh_mark(L, 1, st);
-  CUtensorMap map_x;
-  if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
-
+  if (qkA > 0 && qkB > 0) {
+    using PS = QkPairSmem<6>;
+    SH_CUDA_CHECK(cudaStreamWaitEvent(S->side2, S->ev_fork, 0));
+    if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkB), dim3(320), PS::TOTAL, S->side2, map_x, S->map_wqk128, qg))) return rc;
+    SH_CUDA_CHECK(cudaEventRecord(S->ev_join2, S->side2));
+    L->launches += 1;
+  }
   // ---- Q, K (and V for the dense comparator) ------------------------------------------------
-  if (simt & SH_STAGE_QK) {
+  if (qkA > 0) {
+    // (launched above, as two grids)
+  } else if (simt & SH_STAGE_QK) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_QK, x, out, st))) return rc;
   } else {
     cudaStream_t st = qst;                                  // Q/K projection: side stream when overlapping
@@ -362,6 +418,21 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     switch (S->qk_variant) {
       case 1: rc = launch_gemm<128, 3, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
       case 2: {
+        if (S->persistent && S->qk_pair) {
+          // CTA pairs: 256 x 256 tiles, each CTA loads half of the weight rows
+          using PS = QkPairSmem<6>;
+          if ((rc = set_smem(sh_tc_qk_pair_kernel<6>, PS::TOTAL))) return rc;
+          if (S->qk_pairs_max == 0) {
+            S->qk_pairs_max = max_pairs(sh_tc_qk_pair_kernel<6>, 320, PS::TOTAL);
+            if (S->qk_pairs_max <= 0) S->qk_pairs_max = -1;
+          }
+          if (S->qk_pairs_max > 0) {
+            const int ptiles = ((d.N + 255) / 256) * ((g.ncols + 255) / 256);
+            const unsigned pgrid = 2u * (unsigned)(ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max);
+            rc = launch_k_pairs(pdl && !overlap && (S->pdl_mask & 2), sh_tc_qk_pair_kernel<6>, dim3(pgrid), dim3(320), PS::TOTAL, st, map_x, S->map_wqk128, g);
+            break;
+          }
+        }
         const unsigned tiles = (unsigned)(d.nblk * ((g.ncols + 255) / 256));
         rc = S->persistent ? launch_pgemm<256, 4, PG_QKV, 1>(map_x, S->map_wqk, g, tiles < (unsigned)L->sm_count ? tiles : (unsigned)L->sm_count, st, pdl && !overlap && (S->pdl_mask & 2))
                            : launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st);
@@ -401,6 +472,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     }
   }
   if (overlap) SH_CUDA_CHECK(cudaStreamWaitEvent(st, S->ev_join, 0));
+  if (qkA > 0 && qkB > 0) SH_CUDA_CHECK(cudaStreamWaitEvent(st, S->ev_join2, 0));
   sh_mark(L, 3, st);
   // ---- attention ---------------------------------------------------------------------------------
   if (simt & SH_STAGE_ATTN) {

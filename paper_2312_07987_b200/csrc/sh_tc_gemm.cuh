@@ -32,6 +32,7 @@ struct TcGemmArgs {
   const float2* rope;    // dense Q/K mode: (cos, sin) table [D/2, T] of the rotary embedding, or nullptr
   int* status;
   int* sched;            // persistent dense mode: {next tile, CTAs that made their final claim}, both 0 between launches
+  int claimers;          // claiming CTAs (or CTA pairs) over all grids that share sched; 0: this grid's own
 };
 
 // Rotary embedding of the 16 adjacent feature pairs held in v[0..31] (fp32 bit patterns): pair i of

@@ -166,6 +166,47 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
 __device__ __forceinline__ void mbar_arrive_leader(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(smem_u32(bar) & PAIR_LEADER_MASK) : "memory");
 }
+// The address of `p`'s offset in the shared memory of CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_map(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// Arrival on a barrier of another CTA of the cluster that publishes this thread's earlier writes to
+// that CTA (a few hundred cycles: for once-per-tile messages, not for per-stage traffic).
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bounded wait that also acquires what another CTA of the cluster published before its arrival.
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, int* status, bool& dead) {
+  if (dead) return false;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.b32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((++spins & 63u) == 0) {
+      if (global_timer_ns() - t0 > SH_WAIT_LIMIT_NS || *(volatile int*)status != 0) {
+        if (atomicCAS(status, 0, SH_ERR_TIMEOUT) == 0) {
+          status[1] = (int)blockIdx.x; status[2] = (int)threadIdx.x; status[3] = (int)smem_u32(bar);
+          status[4] = (int)parity; status[5] = (int)gridDim.x; status[6] = (int)blockDim.x;
+        }
+        dead = true;
+        return false;
+      }
+    }
+  }
+}
 // ---- programmatic dependent launch -------------------------------------------------------------------
 // A kernel launched with the programmatic-stream-serialization attribute may become resident while
 // the kernel before it in the stream still runs: pdl_trigger() in the earlier kernel (once every

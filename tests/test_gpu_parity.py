@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2312_07987_b200 import inputs
+from paper_2312_07987_b200 import binding, inputs
 from tests import parity_util as pu
 
 pytestmark = pytest.mark.gpu
@@ -253,7 +253,7 @@ def test_padded_d_head_with_rope_and_shared_selection():
 
 # ---- launch-structure switches (A/B aids): same numbers with ordinary launches on one stream ----
 @pytest.mark.parametrize("env", [{"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
-                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}])
+                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"}])
 def test_launch_structure_switches_keep_the_result(env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)                           # read when the weights are set / at launch
@@ -266,3 +266,22 @@ def test_pair_output_projection_ragged_tokens_and_features():
     # the last pair owns 44 tokens, and with N = 100 none at all), d_model = 384 or 128 not of its 256 features
     full_check(inputs.make_inputs(inputs.LayerConfig("pair_ragged", inputs.DTYPE_BF16, 2, 150, 384, 2, 64, 4, 2, seed=90)))
     full_check(inputs.make_inputs(inputs.LayerConfig("pair_half_empty", inputs.DTYPE_BF16, 1, 100, 128, 3, 128, 3, 1, seed=91)))
+
+
+def test_back_to_back_forward_passes_share_the_tile_counter_cleanly():
+    # the two grids of the split Q/K projection claim tiles from one counter that the last claimer of a
+    # pass puts back: many passes in a row, with and without a host synchronisation between them
+    inp = inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=5)
+    layer = binding.layer_from_inputs(inp)
+    x = binding.to_device(inp.x, inp.cfg.dtype)
+    first = layer.sh_forward(x).clone()
+    torch.cuda.synchronize()
+    for i in range(12):
+        y = layer.sh_forward(x)
+        if i % 3 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0
+    # k = 2: no sum in the layer depends on arrival order, so the passes agree bit for bit
+    assert torch.equal(y, first), float((y - first).abs().max())
+    layer.close()

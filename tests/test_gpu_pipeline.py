@@ -10,7 +10,9 @@ pytestmark = pytest.mark.gpu
 
 
 def test_host_fed_steps_match_direct_forward():
-    inp = inputs.make_inputs(inputs.CONFIGS["small_bf16"])
+    # k = 2: the two-way fp16 sums of the value stage do not depend on arrival order, so every pass
+    # over the same input gives the same bits
+    inp = inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=2)
     layer = binding.layer_from_inputs(inp)
     x0 = binding.to_device(inp.x, inp.cfg.dtype)
     xs = [x0, (x0.float() * 0.5).to(x0.dtype), (x0.float().flip(1)).to(x0.dtype).contiguous()]
@@ -26,7 +28,5 @@ def test_host_fed_steps_match_direct_forward():
     assert layer.sh_last_status() == 0
     for i in range(n_steps):
         ref = want[i % 3]
-        # (the k-way V sums are vector reductions in arrival order: not bit for bit)
-        err = float((outh[i] - ref).abs().max() / ref.pow(2).mean().sqrt())
-        assert err < 1e-2, f"step {i}: {err:.3e}"
+        assert torch.equal(outh[i], ref), f"step {i}: max abs difference {float((outh[i] - ref).abs().max()):.3e}"
     layer.close()
