@@ -287,8 +287,8 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
   const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
   if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
-  if (deep) sh_tc_gate_kernel<8><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
-  else sh_tc_gate_kernel<4><<<d.nblk, 224, smem, st>>>(map_x, S->map_wgate, g);
+  if (deep) sh_tc_gate_kernel<8><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
+  else sh_tc_gate_kernel<4><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
   const size_t ssm = sh_sort_smem_bytes(d);
   // (sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow)
   if ((rc = set_smem(sh_sort_kernel, (int)ssm))) return rc;
@@ -351,18 +351,21 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   }
   CUtensorMap map_x;
   if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
-  // Split Q/K projection.  A grid whose CTAs cannot all start at once (the gate kernel holds SMs)
-  // keeps every kernel launched after it, in any stream, from starting: the sort kernel, launched to
-  // become resident while the gate kernel runs, then starts ~4 us after the gate kernel has ended.
-  // And launched after gate and sort, the projection starts two launch latencies late when the
-  // host is not running ahead (a single forward pass: ~100 us instead of ~107).  So the projection goes
-  // out as two grids of CTA pairs that claim tiles from one counter: grid A, launched BEFORE the
-  // gate kernel, sized for the SMs the gate kernel does not need; grid B, launched AFTER the sort
-  // kernel on a stream of its own, takes over the gate kernel's SMs when they come free.
+  // Split Q/K projection (opt-in: SH_QK_SPLIT).  A grid whose CTAs cannot all start at once (the gate
+  // kernel holds SMs) keeps every kernel launched after it, in any stream, from starting: the sort
+  // kernel, launched to become resident while the gate kernel runs, then starts ~4 us after the gate
+  // kernel has ended.  And launched after gate and sort, the projection starts two launch latencies
+  // late when the host is not running ahead (a single forward pass at the 262M-scale shape: ~102 us
+  // instead of ~107).  With the switch the projection goes out as two grids of CTA pairs that claim
+  // tiles from one counter: grid A, launched BEFORE the gate kernel, sized for the SMs the gate
+  // kernel does not need; grid B, launched AFTER the sort kernel on a stream of its own, takes over
+  // the gate kernel's SMs when they come free.  Not the default: with the launches queued ahead
+  // (back-to-back passes) it gains 1 us of 112, and about one process in six ran every pass 8 us
+  // slower (the third stream presumably sharing a hardware queue with the main one).
   int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
   TcGemmArgs qg{};
   if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_variant == 2 && S->persistent && S->qk_pair && S->side2 &&
-      !getenv("SH_QK_ONE_GRID")) {
+      getenv("SH_QK_SPLIT")) {
     using PS = QkPairSmem<6>;
     if ((rc = set_smem(sh_tc_qk_pair_kernel<6>, PS::TOTAL))) return rc;
     if (S->qk_pairs_max == 0) {

@@ -6,9 +6,11 @@
 // runs, the otherwise idle epilogue warps clear the V and out rows of the CTA's tokens (both
 // are accumulated into later).
 //
-// Warp roles (224 threads): warps 0 and 6 = TMA producers (x boxes / gate-weight boxes: one
-// thread issues a box only every ~150 ns), warp 1 = TMEM owner + UMMA issuer, warps 2..5 =
-// zero-fill, then selection epilogue.
+// Warp roles (608 threads): warps 0 and 6 = TMA producers (x boxes / gate-weight boxes), warp 1 = TMEM owner + UMMA issuer, warps 2..5 and
+// 7..18 = zero-fill, then selection: warps 2..5 (one per TMEM lane quarter) move the logits to
+// shared memory, then four threads share a token's (side, head) groups - the selection is a
+// chain of dependent compares, exp and stores per group (~600 cycles), and with one thread per
+// token it alone took 5.6 us of the kernel's 14.
 #pragma once
 #include "sh_tc_prims.cuh"
 
@@ -25,8 +27,10 @@ struct TcGateArgs {
   int* status;
 };
 
+constexpr int GATE_THREADS = 608;
+
 template <int STAGES>
-__global__ void __launch_bounds__(224)
+__global__ void __launch_bounds__(GATE_THREADS)
 sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, TcGateArgs g) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -40,7 +44,8 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   uint64_t* full_bar = (uint64_t*)(sgen + bar_off);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* tmem_full = empty_bar + STAGES;
-  uint32_t* tmem_slot = (uint32_t*)(tmem_full + 1);
+  uint64_t* logits_ready = tmem_full + 1;               // the logits tile is in shared memory (4 warp arrivals)
+  uint32_t* tmem_slot = (uint32_t*)(logits_ready + 1);
   int* s_hist = (int*)(sgen + bar_off + 256);           // [G]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -54,6 +59,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
     mbar_init(tmem_full, 1);
+    mbar_init(logits_ready, 4);
     fence_barrier_init();
     tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapW);
   }
@@ -66,6 +72,8 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   pdl_trigger();                                        // the sort kernel may become resident (it waits for this grid)
 
   if (warp == 0 || warp == 6) {
+    // (the boxes of consecutive stages arrive ~290 ns apart however many lanes issue them: with x
+    //  coming from HBM, 8 stages x 20 KB in flight over a ~2 us round trip is ~70 GB/s per SM)
     if (lane == 0) {
       for (int kb = 0; kb < KB; ++kb) {
         const int s = kb % STAGES;
@@ -96,18 +104,20 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       umma_commit(tmem_full);
     }
   } else {
-    const int et = threadIdx.x - 64;                    // 0..127
+    // selection threads: 0..127 = warps 2..5, 128..511 = warps 7..18
+    const int et = warp < 6 ? threadIdx.x - 64 : threadIdx.x - 96;
+    constexpr int NSEL = GATE_THREADS - 96;             // 512
     // ---- clear the rows this CTA's tokens own in V and out (accumulated into later) -----------
     if (g.zero_out) {
       const int n4 = d.M / 4;                           // float4 per row
       float4* base = reinterpret_cast<float4*>(g.zero_out + (size_t)row0 * d.M);
       const long total = (long)nrows * n4;
-      for (long i = et; i < total; i += 128) base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (long i = et; i < total; i += NSEL) base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (g.zero_v) {
       const int sh = d.D == 128 ? 4 : 3;                // 16-byte chunks per (token, head) row: D / 8
       const int ch = et & ((1 << sh) - 1);
-      for (int tl = et >> sh; tl < nrows; tl += 128 >> sh) {
+      for (int tl = et >> sh; tl < nrows; tl += NSEL >> sh) {
         const int tok = row0 + tl;
         const int bb = tok / d.T, tt = tok % d.T;
         __half* p = g.zero_v + ((size_t)bb * d.H * d.T + tt) * d.D + ch * 8;
@@ -115,37 +125,46 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
           *reinterpret_cast<uint4*>(p + (size_t)hh * d.T * d.D) = make_uint4(0, 0, 0, 0);
       }
     }
-    // ---- selection epilogue: thread = token = TMEM lane ---------------------------------------
-    const int q = warp & 3;
-    const int r = q * 32 + lane;
-    float* srow = reinterpret_cast<float*>(sgen) + (size_t)r * (Gp + 1);
-    if (mbar_wait(tmem_full, 0, g.status, dead)) {
-      tc_fence_after();
-      const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
-      // logits row -> shared memory (the pipeline buffers are idle now); up to four TMEM loads
-      // are issued per wait because the load latency, not its bandwidth, bounds this loop
-      for (int c0 = 0; c0 < Gp; c0 += 64) {
-        uint32_t v[64];
+    // ---- logits tile -> shared memory: warps 2..5, thread = token = TMEM lane -----------------
+    if (warp < 6) {
+      const int q = warp & 3;
+      const int r = q * 32 + lane;
+      float* srow = reinterpret_cast<float*>(sgen) + (size_t)r * (Gp + 1);
+      if (mbar_wait(tmem_full, 0, g.status, dead)) {
+        tc_fence_after();
+        const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
+        // (the pipeline buffers are idle now); up to four TMEM loads are issued per wait because
+        // the load latency, not its bandwidth, bounds this loop
+        for (int c0 = 0; c0 < Gp; c0 += 64) {
+          uint32_t v[64];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (c0 + 16 * u < Gp) {
-            uint32_t* w = &v[16 * u];
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]),
-                  "=r"(w[8]), "=r"(w[9]), "=r"(w[10]), "=r"(w[11]), "=r"(w[12]), "=r"(w[13]), "=r"(w[14]), "=r"(w[15])
-                : "r"(trow + c0 + 16 * u)
-                : "memory");
+          for (int u = 0; u < 4; ++u) {
+            if (c0 + 16 * u < Gp) {
+              uint32_t* w = &v[16 * u];
+              asm volatile(
+                  "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                  : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]),
+                    "=r"(w[8]), "=r"(w[9]), "=r"(w[10]), "=r"(w[11]), "=r"(w[12]), "=r"(w[13]), "=r"(w[14]), "=r"(w[15])
+                  : "r"(trow + c0 + 16 * u)
+                  : "memory");
+            }
           }
-        }
-        tmem_ld_wait();
+          tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (c0 + i < d.G) srow[c0 + i] = __uint_as_float(v[i]) + g.gbias[c0 + i];
+          for (int i = 0; i < 64; ++i)
+            if (c0 + i < d.G) srow[c0 + i] = __uint_as_float(v[i]) + g.gbias[c0 + i];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(logits_ready);
       }
+    }
+    // ---- selection: thread = (token r, group slice sub): groups sub, sub + 4, ... ----------------
+    if (mbar_wait(logits_ready, 0, g.status, dead)) {
+      const int r = et & 127, sub = et >> 7;
+      const float* srow = reinterpret_cast<const float*>(sgen) + (size_t)r * (Gp + 1);
       const int t = row0 + r;
       if (r < nrows) {
-        for (int grp = 0; grp < d.sides * d.H; ++grp) {
+        for (int grp = sub; grp < d.sides * d.H; grp += NSEL / 128) {
           const float* z = srow + grp * d.E;
           const int side = grp / d.H, h = grp % d.H;
           const size_t o = (((size_t)side * d.N + t) * d.H + h) * d.k;
