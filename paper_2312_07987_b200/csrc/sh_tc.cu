@@ -360,8 +360,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   // tiles from one counter: grid A, launched BEFORE the gate kernel, sized for the SMs the gate
   // kernel does not need; grid B, launched AFTER the sort kernel on a stream of its own, takes over
   // the gate kernel's SMs when they come free.  Not the default: with the launches queued ahead
-  // (back-to-back passes) it gains 1 us of 112, and about one process in six ran every pass 8 us
-  // slower (the third stream presumably sharing a hardware queue with the main one).
+  // (back-to-back passes) it gains 1-1.5 us of 112 (0-4 of 273 at 16384 tokens, depending on the
+  // GPU of the pool), and about one process in six ran every pass 6-8 us slower - as every process
+  // does when grid B's stream is given a higher priority than the caller's, so the slow mode is
+  // grid B's CTAs being placed ahead of the sort and value-expert kernels' CTAs.
   int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
   TcGemmArgs qg{};
   if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_variant == 2 && S->persistent && S->qk_pair && S->side2 &&
