@@ -317,7 +317,7 @@ static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const 
   auto kern = sh_tc_pgemm_kernel<BN, STAGES, MODE, MT>;
   constexpr int smem = PGemmSmem<BN, STAGES, MT>::TOTAL;
   if (int rc = set_smem(kern, smem)) return rc;
-  return launch_k(pdl, kern, dim3(grid), dim3(320), smem, st, mapA, mapB, g);
+  return launch_k(pdl, kern, dim3(grid), dim3(352), smem, st, mapA, mapB, g);
 }
 
 template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>

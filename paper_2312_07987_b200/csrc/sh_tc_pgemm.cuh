@@ -31,7 +31,7 @@ struct PGemmSmem {
 };
 
 template <int BN, int STAGES, int MODE, int MT>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(352, 1)
 sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcGemmArgs g) {
   using SM = PGemmSmem<BN, STAGES, MT>;
   static_assert(MT * BN <= 256, "two accumulators must fit the 512 TMEM columns");
@@ -58,8 +58,9 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
   bool dead = false;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 129 : 2); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    // (MT == 2: one issuing thread per 128-row half of the tile, each committing on its own)
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], GATHER ? 129 : 2); mbar_init(&empty_bar[s], MT); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], MT); mbar_init(&acc_empty[b], 128); }
     for (int j = 0; j < TQ; ++j) { mbar_init(&tq_full[j], 1); mbar_init(&tq_empty[j], 130); }   // A producer + issuer + 128 epilogue threads
     fence_barrier_init();
     tma_prefetch_desc(&mapB);
@@ -144,27 +145,28 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || (MT == 2 && warp == 10)) {
+    // With two 128-row halves per tile (MT == 2, N = 128) a stage is eight UMMAs of 64 cycles, and
+    // issuing one costs a thread about as long: each half has its own issuing thread (warp 1 / 10),
+    // its own accumulator columns and its own commits.
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_f16(128, BN, 1, 1, 0);
-      const uint32_t a_lo0 = desc_lo_k(sbase), b_lo0 = desc_lo_k(sbase + SM::A_BYTES);
+      const int mt = warp == 1 ? 0 : 1;
+      const uint32_t a_lo0 = desc_lo_k(sbase) + mt * (128 * 64 * 2 >> 4), b_lo0 = desc_lo_k(sbase + SM::A_BYTES);
       int s = 0, it = 0;
       uint32_t par = 0;
       for (; !dead; ++it) {
         if (next_tile(it) < 0) break;
         const int b = it & 1;
         if (!mbar_wait(&acc_empty[b], ((it >> 1) & 1) ^ 1, g.status, dead)) break;
-        const uint32_t td = tmem + b * ACC_COLS;
+        const uint32_t td = tmem + b * ACC_COLS + mt * BN;
         for (int kb = 0; kb < KB; ++kb) {
           if (!mbar_wait(&full_bar[s], par, g.status, dead)) break;
           tc_fence_after();
           const uint32_t a_lo = a_lo0 + s * (SM::STAGE_BYTES >> 4), b_lo = b_lo0 + s * (SM::STAGE_BYTES >> 4);
 #pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_f16(td + mt * BN, desc_pack(a_lo + mt * (128 * 64 * 2 >> 4) + 2 * k), desc_pack(b_lo + 2 * k), idesc, (kb | k) != 0);
-          }
+          for (int k = 0; k < 4; ++k)
+            umma_f16(td, desc_pack(a_lo + 2 * k), desc_pack(b_lo + 2 * k), idesc, (kb | k) != 0);
           umma_commit(&empty_bar[s]);
           if (++s == STAGES) { s = 0; par ^= 1; }
         }
@@ -172,7 +174,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         umma_commit(&acc_full[b]);
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 6 && warp < 10) {
     if (GATHER) {
       // thread -> 16-byte chunk c of rows rb, rb + 16, ... (8 threads cover one 128-byte row)
       const int et = threadIdx.x - 192;                    // 0..127
@@ -220,7 +222,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
           if (++s_arr == STAGES) s_arr = 0;
         }
     }
-  } else {
+  } else if (warp < 6) {
     // ---- epilogue: thread = accumulator row = TMEM lane -----------------------------------------
     const int q = warp & 3;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
