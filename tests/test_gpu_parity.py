@@ -288,3 +288,24 @@ def test_back_to_back_forward_passes_share_the_tile_counter_cleanly(split, monke
     # k = 2: no sum in the layer depends on arrival order, so the passes agree bit for bit
     assert torch.equal(y, first), float((y - first).abs().max())
     layer.close()
+
+
+def _random_bf16_configs(n, seed):
+    # seeded draws over the shape space the bf16 path accepts: ragged token counts (tile tails, a CTA
+    # pair whose second half is empty), d_model any multiple of 128, both stored head widths and
+    # padded ones, 1..8 experts, every k up to E and 4, with and without a skewed gate bias
+    rng = np.random.default_rng(seed)
+    cfgs = []
+    for i in range(n):
+        E = int(rng.integers(1, 9))
+        k = int(rng.integers(1, min(E, 4) + 1))
+        cfgs.append(inputs.LayerConfig(
+            f"rand{seed}_{i}", inputs.DTYPE_BF16, int(rng.integers(1, 4)), int(rng.integers(1, 700)),
+            128 * int(rng.integers(1, 7)), int(rng.integers(1, 5)), int(rng.choice([40, 64, 100, 128])), E, k,
+            seed=1000 * seed + i, zipf_bias=float(rng.choice([0.0, 1.2]))))
+    return cfgs
+
+
+@pytest.mark.parametrize("cfg", _random_bf16_configs(10, 7), ids=lambda c: f"B{c.batch}T{c.seq}M{c.d_model}H{c.n_heads}D{c.d_head}E{c.n_experts}k{c.k}")
+def test_random_bf16_shapes(cfg):
+    full_check(inputs.make_inputs(cfg), check_stage_buffers=False)
