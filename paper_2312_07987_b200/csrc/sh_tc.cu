@@ -261,7 +261,7 @@ static int gate_smem_bytes(int Gp, int G, int stages) {
 }
 
 // Gate + top-k + bucket sort.  With zero_for_forward the fused kernel also clears V and out.
-static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_forward, cudaStream_t st) {
+static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_forward, cudaStream_t st, bool sort_apart = false) {
   TcState* S = (TcState*)L->tc;
   const ShDims& d = L->d;
   char* ws = L->ws;
@@ -289,7 +289,11 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
   if (deep) sh_tc_gate_kernel<8><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
   else sh_tc_gate_kernel<4><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
-  const size_t ssm = sh_sort_smem_bytes(d);
+  size_t ssm = sh_sort_smem_bytes(d);
+  // sort_apart: ask for enough shared memory that a sort block fits beside a gate CTA but not beside a
+  // ~198 KB GEMM CTA: next to the Q/K projection's CTAs (whose waiting warps poll) a block takes
+  // 11 us instead of 4.7
+  if (sort_apart && ssm < 40 * 1024) ssm = 40 * 1024;
   // (sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow)
   if ((rc = set_smem(sh_sort_kernel, (int)ssm))) return rc;
   // In a forward pass only the value experts read sorted lists (the output projection works from
@@ -351,23 +355,23 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   }
   CUtensorMap map_x;
   if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
-  // Split Q/K projection (opt-in: SH_QK_SPLIT).  A grid whose CTAs cannot all start at once (the gate
-  // kernel holds SMs) keeps every kernel launched after it, in any stream, from starting: the sort
-  // kernel, launched to become resident while the gate kernel runs, then starts ~4 us after the gate
-  // kernel has ended.  And launched after gate and sort, the projection starts two launch latencies
-  // late when the host is not running ahead (a single forward pass at the 262M-scale shape: ~102 us
-  // instead of ~107).  With the switch the projection goes out as two grids of CTA pairs that claim
-  // tiles from one counter: grid A, launched BEFORE the gate kernel, sized for the SMs the gate
-  // kernel does not need; grid B, launched AFTER the sort kernel on a stream of its own, takes over
-  // the gate kernel's SMs when they come free.  Not the default: with the launches queued ahead
-  // (back-to-back passes) it gains 1-1.5 us of 112 (0-4 of 273 at 16384 tokens, depending on the
-  // GPU of the pool), and about one process in six ran every pass 6-8 us slower - as every process
-  // does when grid B's stream is given a higher priority than the caller's, so the slow mode is
-  // grid B's CTAs being placed ahead of the sort and value-expert kernels' CTAs.
+  // Split Q/K projection (SH_QK_ONE_GRID switches it off).  A grid whose CTAs cannot all start at
+  // once (the gate kernel holds SMs) keeps every kernel launched after it, in any stream, from
+  // starting: the sort kernel, launched to become resident while the gate kernel runs, then starts
+  // 4-8 us after the gate kernel has ended.  And launched after gate and sort, the projection starts
+  // two launch latencies late when the host is not running ahead (a single forward pass at the
+  // 262M-scale shape: ~102 us instead of ~107).  So the projection goes out as two grids of CTA pairs
+  // that claim tiles from one counter: grid A, launched BEFORE the gate kernel, sized for the SMs the
+  // gate kernel does not need; grid B, launched AFTER the sort kernel on a stream of its own, takes
+  // over the gate kernel's SMs when they come free.  The sort blocks are kept off the SMs of grid A
+  // (see tc_gate_sort): without that, about one process in six ran every pass 6-8 us slower (as every
+  // process does when grid B's stream is given a higher priority than the caller's: grid B's CTAs
+  // placed ahead of the sort and value-expert kernels' CTAs); with it, ten processes in a row ran
+  // 109.8-111.9 us per pass against 111.7-114.7 with one grid, and 265 against 270.5 at 16384 tokens.
   int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
   TcGemmArgs qg{};
   if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_variant == 2 && S->persistent && S->qk_pair && S->side2 &&
-      getenv("SH_QK_SPLIT")) {
+      !getenv("SH_QK_ONE_GRID")) {
     using PS = QkPairSmem<6>;
     if ((rc = set_smem(sh_tc_qk_pair_kernel<6>, PS::TOTAL))) return rc;
     if (S->qk_pairs_max == 0) {
@@ -395,7 +399,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     }
   }
   if (!L->dense) {
-    if ((rc = tc_gate_sort(L, x, out, true, st))) return rc;
+    if ((rc = tc_gate_sort(L, x, out, true, st, qkA > 0))) return rc;
   }
   sh_mark(L, 1, st);
   if (qkA > 0 && qkB > 0) {

@@ -253,7 +253,7 @@ def test_padded_d_head_with_rope_and_shared_selection():
 
 # ---- launch-structure switches (A/B aids): same numbers with ordinary launches on one stream ----
 @pytest.mark.parametrize("env", [{"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
-                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_SPLIT": "1"}])
+                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"}])
 def test_launch_structure_switches_keep_the_result(env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)                           # read when the weights are set / at launch
@@ -270,9 +270,9 @@ def test_pair_output_projection_ragged_tokens_and_features():
 
 @pytest.mark.parametrize("split", [False, True])
 def test_back_to_back_forward_passes_share_the_tile_counter_cleanly(split, monkeypatch):
-    if split:
-        monkeypatch.setenv("SH_QK_SPLIT", "1")
-    # the CTA pairs of the Q/K projection (one grid, or two with SH_QK_SPLIT) claim tiles from one counter
+    if not split:
+        monkeypatch.setenv("SH_QK_ONE_GRID", "1")
+    # the CTA pairs of the Q/K projection (two grids, or one with SH_QK_ONE_GRID) claim tiles from one counter
     # that the last claimer of a pass puts back: many passes in a row, with and without a host synchronisation between them
     inp = inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=5)
     layer = binding.layer_from_inputs(inp)
