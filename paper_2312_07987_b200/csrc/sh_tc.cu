@@ -366,7 +366,8 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   // over the gate kernel's SMs when they come free.  The sort blocks are kept off the SMs of grid A
   // (see tc_gate_sort): without that, about one process in six ran every pass 6-8 us slower (as every
   // process does when grid B's stream is given a higher priority than the caller's: grid B's CTAs
-  // placed ahead of the sort and value-expert kernels' CTAs); with it, ten processes in a row ran
+  // placed ahead of the sort and value-expert kernels' CTAs, and as happens with a five-stage grid
+  // B, whose CTAs fit beside the sort blocks and slow them down); with it, ten processes in a row ran
   // 109.8-111.9 us per pass against 111.7-114.7 with one grid, and 265 against 270.5 at 16384 tokens.
   int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
   TcGemmArgs qg{};
