@@ -96,13 +96,15 @@ sh_gate_topk_kernel(const T* __restrict__ x, const T* __restrict__ Wg, const flo
 // Dynamic shared memory: 128*H*k*2*8 bytes (the block's idx and gate values, both sides)
 // + (6*G + 8) * 4 bytes.
 // ---------------------------------------------------------------------------------------
-// Threads: 128 * GS, thread = (token tid % 128, group slice tid / 128); slice gs handles the
-// (side, head) groups gs, gs + GS, ...
-static __global__ void __launch_bounds__(1024)
-sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, const int* __restrict__ blockcnt,
-               int* __restrict__ offsets, int* __restrict__ lists, float* __restrict__ lgate,
-               ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
-  extern __shared__ int s_sort[];
+// The block's part of the sort, for `nthreads` = 128 * GS threads numbered tid; `sync` is a barrier
+// over exactly those threads.  have_sel: the block's idx / gate values are already in the
+// shared-memory arrays (the fused gate kernel put them there), otherwise they are copied from idx /
+// gate.  blockcnt must be complete for ALL blocks.
+template <class Sync>
+static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx, const float* __restrict__ gate, const int* __restrict__ blockcnt,
+                                                     int* __restrict__ offsets, int* __restrict__ lists, float* __restrict__ lgate,
+                                                     ShTile* __restrict__ tiles, int* __restrict__ ntiles, const ShDims& d,
+                                                     int* s_sort, int tid, int nthreads, int blk, bool have_sel, Sync sync) {
   const int nb = d.G;
   const int per_tok = d.H * d.k;
   int* s_pre = s_sort;                 // [nb] selections of this bucket in earlier blocks
@@ -112,23 +114,18 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
   int* s_wcnt = s_tbase + nb;          // [nb][4] per-warp counts of this block's tokens
   int* s_idx = s_wcnt + 4 * nb;        // [2][128*per_tok]
   float* s_gt = (float*)(s_idx + 2 * 128 * per_tok);
-  const int tid = threadIdx.x, lane = tid & 31;
-  const int tl = tid & 127, gs = tid >> 7, GS = blockDim.x >> 7;
+  const int lane = tid & 31;
+  const int tl = tid & 127, gs = tid >> 7, GS = nthreads >> 7;
   const int twarp = tl >> 5;           // warp index among the 4 warps of a slice
-  const int blk = blockIdx.x;
   const int tok0 = blk * SH_TILE_ROWS;
   const int nrows = min(SH_TILE_ROWS, d.N - tok0);
-  for (int i = tid; i < 2 * nb; i += blockDim.x) s_pre[i] = 0;   // s_pre and s_tot
-  // programmatic dependent launch (no-ops in an ordinary launch): let the next kernel in the
-  // stream become resident, then wait for the gate kernel's selections to be complete and visible
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  for (int i = tid; i < 2 * nb; i += nthreads) s_pre[i] = 0;   // s_pre and s_tot
   // bucket b = tid % nb; the thread sums the blocks part, part + parts, ... in registers.  These
   // loads do not depend on the selections copy below, so both are in flight together.
   int my_b = -1, my_tot = 0, my_pre = 0;
   {
-    const int parts = max(1, (int)blockDim.x / nb);
-    if (nb <= (int)blockDim.x) {
+    const int parts = max(1, nthreads / nb);
+    if (nb <= nthreads) {
       if (tid / nb < parts) {
         my_b = tid % nb;
         const int part = tid / nb;
@@ -141,19 +138,19 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
       }
     }
   }
-  for (int side = 0; side < d.sides; ++side) {                    // this block's selections
+  for (int side = 0; side < (have_sel ? 0 : d.sides); ++side) {  // this block's selections
     const size_t base = ((size_t)side * d.N + tok0) * per_tok;
-    for (int i = tid; i < nrows * per_tok; i += blockDim.x) {
+    for (int i = tid; i < nrows * per_tok; i += nthreads) {
       s_idx[side * 128 * per_tok + i] = idx[base + i];
       s_gt[side * 128 * per_tok + i] = gate[base + i];
     }
   }
-  __syncthreads();
+  sync();
   if (my_b >= 0) {
     if (my_tot) atomicAdd(&s_tot[my_b], my_tot);
     if (my_pre) atomicAdd(&s_pre[my_b], my_pre);
-  } else if (nb > (int)blockDim.x) {                              // more buckets than threads: plain loop
-    for (int b = tid; b < nb; b += blockDim.x) {
+  } else if (nb > nthreads) {                              // more buckets than threads: plain loop
+    for (int b = tid; b < nb; b += nthreads) {
       int tot = 0, pre = 0;
       for (int bk = 0; bk < d.nblk; ++bk) {
         const int c = blockcnt[(size_t)bk * nb + b];
@@ -164,8 +161,8 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
       s_pre[b] = pre;
     }
   }
-  __syncthreads();
-  for (int g = tid; g < d.sides * d.H; g += blockDim.x) {
+  sync();
+  for (int g = tid; g < d.sides * d.H; g += nthreads) {
     int run = 0;
     for (int e = 0; e < d.E; ++e) {
       s_off[g * d.E + e] = run;
@@ -182,7 +179,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
       if (lane == 0) s_wcnt[(grp * d.E + e) * 4 + twarp] = __popc(bal);
     }
   }
-  __syncthreads();
+  sync();
   {
     const int t = tok0 + tl;
     for (int grp = gs; grp < d.sides * d.H; grp += GS) {
@@ -209,7 +206,7 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     }
   }
   if (blk != 0) return;
-  for (int g = tid; g < d.sides * d.H; g += blockDim.x) {
+  for (int g = tid; g < d.sides * d.H; g += nthreads) {
     for (int e = 0; e < d.E; ++e) offsets[g * (d.E + 1) + e] = s_off[g * d.E + e];
     offsets[g * (d.E + 1) + d.E] = s_off[g * d.E + d.E - 1] + s_tot[g * d.E + d.E - 1];
   }
@@ -223,8 +220,8 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
     }
     ntiles[side] = run;
   }
-  __syncthreads();
-  for (int i = tid; i < d.sides * d.H * d.E * 32; i += blockDim.x) {   // 32 threads share a bucket's tiles
+  sync();
+  for (int i = tid; i < d.sides * d.H * d.E * 32; i += nthreads) {   // 32 threads share a bucket's tiles
     const int b = i >> 5;
     const int side = b / (d.H * d.E), h = (b / d.E) % d.H, e = b % d.E;
     const int cnt = s_tot[b];
@@ -237,6 +234,21 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
       tp[ti] = tl2;
     }
   }
+}
+
+// Threads: 128 * GS, thread = (token tid % 128, group slice tid / 128); slice gs handles the
+// (side, head) groups gs, gs + GS, ...
+static __global__ void __launch_bounds__(1024)
+sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, const int* __restrict__ blockcnt,
+               int* __restrict__ offsets, int* __restrict__ lists, float* __restrict__ lgate,
+               ShTile* __restrict__ tiles, int* __restrict__ ntiles, ShDims d) {
+  extern __shared__ int s_sort[];
+  // programmatic dependent launch (no-ops in an ordinary launch): let the next kernel in the
+  // stream become resident, then wait for the gate kernel's selections to be complete and visible
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  sh_sort_block(idx, gate, blockcnt, offsets, lists, lgate, tiles, ntiles, d, s_sort, (int)threadIdx.x, (int)blockDim.x, (int)blockIdx.x,
+                false, [] { __syncthreads(); });
 }
 
 static inline int sh_sort_threads(const ShDims& d) {
