@@ -80,6 +80,7 @@ struct TcState {
   int qk_bn, o_bn, qk_variant;
   int o_pair, o_pairs_max;       // output projection on CTA pairs; clusters the device holds at once
   int qk_pair, qk_pairs_max;     // the same for the dense Q/K projection
+  int gate_coop;                 // 1: the gate kernel can be launched cooperatively (fused sort), -1: it cannot
   int persistent;       // 1 = persistent Q/K and value-expert GEMMs (default); 0 = one CTA per tile (experiment switch)
   int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
   int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
@@ -214,6 +215,7 @@ int sh_tc_prepare(sh_layer* L) {
   S->o_pairs_max = 0;
   S->qk_pair = getenv("SH_QK_SINGLE") == nullptr;
   S->qk_pairs_max = 0;
+  S->gate_coop = 0;
   const char* env = getenv("SH_SIMT_STAGES");
   S->simt_mask = env ? atoi(env) : 0;
   if (L->sm_count == 0) {
@@ -287,6 +289,52 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
   const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
   if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
+  // In a forward pass only the value experts read sorted lists (the output projection works from
+  // idx / gate, token tile by token tile), so only the source side is sorted there -- unless the
+  // scatter-add or CUDA-core output projection (debugging paths) is selected.  The histogram stride
+  // stays G; the sort's loops run over sides * H groups.
+  ShDims ds = d;
+  if (zero_for_forward && !S->o_scatter && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
+  // Fused sort: when every CTA of the gate kernel can be resident at once (cooperative launch) and the
+  // sort's scratch fits behind the logits tile in the idle operand ring, the gate kernel places the
+  // tokens itself and there is no sort kernel.  Used when the gate kernel needs at most half of the SMs:
+  // 114.8 -> 110.7 us per forward at 8192 tokens (64 CTAs), but 270.7 -> 273.3 at 16384 (128 CTAs that
+  // must all find a free SM before any of them starts).
+  if (L->sm_count == 0) {
+    int dev = 0;
+    SH_CUDA_CHECK(cudaGetDevice(&dev));
+    SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
+  {
+    const int stage = 128 * 64 * 2 + ((S->gate_gp * 128 + 1023) & ~1023);
+    const int pipe = (deep ? 8 : 4) * stage, stag = 128 * (S->gate_gp + 1) * 4;
+    g.fused = !getenv("SH_SORT_SEPARATE") && 2 * d.nblk <= L->sm_count && ((stag + 15) & ~15) + (int)sh_sort_smem_bytes(d) <= pipe;
+    if (g.fused && S->gate_coop == 0) {
+      int dev = 0, coop = 0, per_sm = 0;
+      SH_CUDA_CHECK(cudaGetDevice(&dev));
+      SH_CUDA_CHECK(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+      if (deep) SH_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sh_tc_gate_kernel<8>, GATE_THREADS, smem));
+      else SH_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sh_tc_gate_kernel<4>, GATE_THREADS, smem));
+      S->gate_coop = (coop && per_sm >= 1) ? 1 : -1;
+    }
+    if (S->gate_coop < 0) g.fused = 0;
+  }
+  g.sort_sides = ds.sides; g.tile_rows_src = d.tile_rows_src; g.max_tiles = d.max_tiles;
+  g.offsets = (int*)(ws + L->o.offsets); g.lists = (int*)(ws + L->o.lists); g.lgate = (float*)(ws + L->o.lgate);
+  g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
+  g.gridbar = (int*)(ws + L->o.status) + 24;
+  if (g.fused) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(d.nblk); cfg.blockDim = dim3(GATE_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (deep) SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, sh_tc_gate_kernel<8>, map_x, S->map_wgate, g));
+    else SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, sh_tc_gate_kernel<4>, map_x, S->map_wgate, g));
+    L->launches += 1;
+    return SH_OK;
+  }
   if (deep) sh_tc_gate_kernel<8><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
   else sh_tc_gate_kernel<4><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
   size_t ssm = sh_sort_smem_bytes(d);
@@ -296,12 +344,6 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   if (sort_apart && ssm < 40 * 1024) ssm = 40 * 1024;
   // (sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow)
   if ((rc = set_smem(sh_sort_kernel, (int)ssm))) return rc;
-  // In a forward pass only the value experts read sorted lists (the output projection works from
-  // idx / gate, token tile by token tile), so only the source side is sorted there -- unless the
-  // scatter-add or CUDA-core output projection (debugging paths) is selected.  The histogram stride
-  // stays G; the kernel's loops run over sides * H groups.
-  ShDims ds = d;
-  if (zero_for_forward && !S->o_scatter && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
   if ((rc = launch_k(S->pdl && !L->ev && (S->pdl_mask & 1), sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(ds)), ssm, st,
                      (const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate), (const int*)(ws + L->o.blockcnt),
                      (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists), (float*)(ws + L->o.lgate),

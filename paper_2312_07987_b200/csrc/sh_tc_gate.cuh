@@ -6,6 +6,12 @@
 // runs, the otherwise idle epilogue warps clear the V and out rows of the CTA's tokens (both
 // are accumulated into later).
 //
+// Fused sort (g.fused, cooperative launch): when the whole grid is resident at once, the CTAs meet
+// at a grid-wide barrier (a counter in global memory, bounded wait) once their histograms are
+// published, and each then places its own tokens in the sorted lists (sh_sort_block, the body of the
+// stand-alone sort kernel, run by the 512 selection threads on the selections still in shared
+// memory): no second kernel, no second trip of the selections through L2.
+//
 // Warp roles (608 threads): warps 0 and 6 = TMA producers (x boxes / gate-weight boxes), warp 1 = TMEM owner + UMMA issuer, warps 2..5 and
 // 7..18 = zero-fill, then selection: warps 2..5 (one per TMEM lane quarter) move the logits to
 // shared memory, then four threads share a token's (side, head) groups - the selection is a
@@ -13,6 +19,7 @@
 // token it alone took 5.6 us of the kernel's 14.
 #pragma once
 #include "sh_tc_prims.cuh"
+#include "sh_simt.cuh"
 
 namespace shtc {
 
@@ -25,6 +32,13 @@ struct TcGateArgs {
   __half* zero_v;            // [B, H, T, D] or nullptr
   float* zero_out;           // [N, M] or nullptr
   int* status;
+  // fused sort (cooperative launch only)
+  int fused;                 // 1: place the tokens in the sorted lists at the end of this kernel
+  int sort_sides;            // sides the sort covers (1: source side only)
+  int tile_rows_src;         // rows per tile of the source-side tile table
+  int max_tiles;
+  int* offsets; int* lists; float* lgate; ShTile* tiles; int* ntiles;
+  int* gridbar;              // {arrived, departed}, both 0 between launches
 };
 
 constexpr int GATE_THREADS = 608;
@@ -159,7 +173,13 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       }
     }
     // ---- selection: thread = (token r, group slice sub): groups sub, sub + 4, ... ----------------
-    if (mbar_wait(logits_ready, 0, g.status, dead)) {
+    // fused sort: its scratch sits behind the logits rows; the selections go there as well
+    int* s_sort = reinterpret_cast<int*>(sgen + ((stag_bytes + 15) & ~15));
+    const int per_tok = d.H * d.k;
+    int* s_idx = s_sort + 8 * d.G;                        // [2][128 * per_tok], as sh_sort_block lays it out
+    float* s_gt = reinterpret_cast<float*>(s_idx + 2 * 128 * per_tok);
+    const bool sel_ok = mbar_wait(logits_ready, 0, g.status, dead);
+    if (sel_ok) {
       const int r = et & 127, sub = et >> 7;
       const float* srow = reinterpret_cast<const float*>(sgen) + (size_t)r * (Gp + 1);
       const int t = row0 + r;
@@ -178,11 +198,46 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
               if (best < 0 || ze > bz) { best = e; bz = ze; }
             }
             taken |= 1u << best;
+            const float gv = 1.f / (1.f + expf(-bz));
             g.idx[o + j] = best;
-            g.gate[o + j] = 1.f / (1.f + expf(-bz));
+            g.gate[o + j] = gv;
+            if (g.fused) {
+              s_idx[side * 128 * per_tok + (r * d.H + h) * d.k + j] = best;
+              s_gt[side * 128 * per_tok + (r * d.H + h) * d.k + j] = gv;
+            }
             atomicAdd(&s_hist[grp * d.E + best], 1);
           }
         }
+      }
+    }
+    if (g.fused) {
+      // ---- publish the histogram, meet the other CTAs, place this CTA's tokens ----------------------
+      auto sel_sync = [] { asm volatile("bar.sync 1, 512;" ::: "memory"); };
+      sel_sync();                                           // s_hist, s_idx, s_gt complete
+      for (int i = et; i < d.G; i += NSEL) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
+      __threadfence();
+      sel_sync();
+      int* s_flag = s_hist + d.G;                           // (the histogram area is 3 G words)
+      if (et == 0) {
+        bool ok = sel_ok;
+        atomicAdd(g.gridbar, 1);
+        const uint64_t t0 = global_timer_ns();
+        while (ok && *(volatile int*)g.gridbar < (int)gridDim.x) {
+          if (global_timer_ns() - t0 > SH_WAIT_LIMIT_NS || *(volatile int*)g.status != 0) {
+            atomicCAS(g.status, 0, SH_ERR_TIMEOUT);
+            ok = false;
+          }
+        }
+        __threadfence();
+        // the CTA that leaves last puts the counters back for the next launch
+        if (atomicAdd(g.gridbar + 1, 1) == (int)gridDim.x - 1) { g.gridbar[0] = 0; g.gridbar[1] = 0; }
+        *s_flag = ok ? 1 : 0;
+      }
+      sel_sync();
+      if (*(volatile int*)s_flag) {
+        ShDims ds = d;
+        ds.sides = g.sort_sides;
+        sh_sort_block(g.idx, g.gate, g.blockcnt, g.offsets, g.lists, g.lgate, g.tiles, g.ntiles, ds, s_sort, et, NSEL, (int)blockIdx.x, true, sel_sync);
       }
     }
   }
@@ -193,7 +248,8 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     tmem_dealloc(tmem_d, tmem_cols);
   }
   // ---- publish this CTA's selection histogram (the sort kernel scans them) ------------------
-  for (int i = threadIdx.x; i < d.G; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
+  if (!g.fused)
+    for (int i = threadIdx.x; i < d.G; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
 }
 
 }  // namespace shtc

@@ -253,7 +253,7 @@ def test_padded_d_head_with_rope_and_shared_selection():
 
 # ---- launch-structure switches (A/B aids): same numbers with ordinary launches on one stream ----
 @pytest.mark.parametrize("env", [{"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
-                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"}])
+                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"}, {"SH_SORT_SEPARATE": "1"}])
 def test_launch_structure_switches_keep_the_result(env, monkeypatch):
     for k, v in env.items():
         monkeypatch.setenv(k, v)                           # read when the weights are set / at launch
