@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 DEFAULT_CONFIG = "c4_262m_bf16"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's main kernel, from the ncu
 # capture summarised in profiles/c4_262m_bf16_forward_kernels.md (MB, workload c4_262m_bf16)
-DRAM_TRAFFIC_MB = {"c4_262m_bf16": {"gate_topk_sort": 16.87 + 0.56, "qk_proj": 18.92, "v_experts": 29.92,
+DRAM_TRAFFIC_MB = {"c4_262m_bf16": {"gate_topk_sort": 16.92, "qk_proj": 18.91, "v_experts": 29.92,
                                     "attention": 25.22, "o_experts": 13.23}}
 STAGES = ["gate_topk_sort", "qk_proj", "v_experts", "attention", "o_experts"]
 
