@@ -115,7 +115,9 @@ def test_forward_is_repeatable_and_selection_deterministic():
     for a, b in zip(r0, r1):
         assert torch.equal(a, b)
     rms = y0.double().pow(2).mean().sqrt().item()
-    assert (y0 - y1).abs().max().item() / rms < 1e-2
+    # (k = 3: the value stage's fp16 sums come in arrival order; both passes are within the tolerance of
+    #  the oracle, their difference has been seen at 1.2e-2 * RMS)
+    assert (y0 - y1).abs().max().item() / rms < 4e-2
     layer.close()
 
 
@@ -155,8 +157,13 @@ def rope_check(inp, base=10000.0, batches=None):
     layer.sh_set_rope(0.0)                                   # off again: the plain layer
     y_off = layer.sh_forward(x)
     torch.cuda.synchronize()
-    # (not bit for bit: the k-way V sums are atomic / vector reductions in arrival order)
-    assert pu.rel_rms_err(y_off.cpu().numpy(), y_plain.cpu().numpy()) < (1e-5 if cfg.dtype == inputs.DTYPE_F32 else 1e-2)
+    # (k >= 3: not bit for bit, the k-way V sums are atomic / vector reductions in arrival order; two
+    #  passes have been seen 1.2e-2 * RMS apart at k = 3, and a rotation left on would be of order 1)
+    diff = pu.rel_rms_err(y_off.cpu().numpy(), y_plain.cpu().numpy())
+    if cfg.dtype == inputs.DTYPE_BF16 and cfg.k <= 2:
+        assert torch.equal(y_off, y_plain), diff
+    else:
+        assert diff < (1e-5 if cfg.dtype == inputs.DTYPE_F32 else 4e-2), diff
     layer.close()
 
 
