@@ -65,6 +65,9 @@ static void layout_workspace(sh_layer* L) {
   o.tiles = take((size_t)2 * d.max_tiles * sizeof(ShTile));
   o.ntiles = take(256);
   o.rope = take((size_t)d.T * (d.D / 2) * 8);     // (cos, sin) per feature pair and position
+  // k >= 3 with 16-bit storage: the k gate-weighted contributions to a value row are summed in fp32
+  // here and rounded to fp16 once (k successive fp16 roundings cost most of the output tolerance)
+  o.v32 = take((L->dtype == SH_BF16 && !L->dense && d.k >= 3) ? (size_t)d.N * HD * 4 : 16);
   o.total = off;
 }
 

@@ -29,7 +29,7 @@ struct ShDims {
 // Workspace sub-buffers (byte offsets from the workspace base).
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, rope, total;
+         offsets, lists, lgate, tiles, ntiles, rope, v32, total;
 };
 
 struct sh_layer {

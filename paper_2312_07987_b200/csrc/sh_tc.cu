@@ -262,6 +262,25 @@ static int gate_smem_bytes(int Gp, int G, int stages) {
   return bar_off + 256 + 3 * G * 4 + 1024;
 }
 
+// k >= 3: the value experts accumulate a token's k contributions in an fp32 buffer (fp32 vector
+// reductions) that is rounded to fp16 once, instead of k fp16 reductions into V itself - those cost
+// up to k * 2^-11 relative on rows of which the first tokens of a sequence, attending to few keys,
+// pass nearly unaveraged into an output far above the global RMS the tolerance is measured in.
+static bool use_v32(const sh_layer* L, const TcState* S) {
+  return L->dtype == SH_BF16 && !L->dense && L->d.k >= 3 && !(S->simt_mask & SH_STAGE_V);
+}
+
+static __global__ void __launch_bounds__(256)
+sh_v32_to_f16_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, size_t n4) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 v = src[i];
+    const __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
+    dst[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+  }
+}
+
 // Gate + top-k + bucket sort.  With zero_for_forward the fused kernel also clears V and out.
 static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_forward, cudaStream_t st, bool sort_apart = false) {
   TcState* S = (TcState*)L->tc;
@@ -272,6 +291,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_GATE, x, nullptr, st))) return rc;
     if (zero_for_forward) {
       SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * d.H * d.D * 2, st));
+      if (use_v32(L, S)) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v32, 0, (size_t)d.N * d.H * d.D * 4, st));
       SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
       L->launches += 2;
     }
@@ -283,7 +303,8 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.d = d; g.Gp = S->gate_gp; g.gbias = (const float*)(ws + L->o.gbias);
   g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
   g.blockcnt = (int*)(ws + L->o.blockcnt);
-  g.zero_v = zero_for_forward ? (__half*)(ws + L->o.v) : nullptr;
+  g.zero_v_f32 = use_v32(L, S) ? 1 : 0;
+  g.zero_v = zero_for_forward ? (void*)(ws + (g.zero_v_f32 ? L->o.v32 : L->o.v)) : nullptr;
   g.zero_out = (zero_for_forward && (S->o_scatter || (S->simt_mask & SH_STAGE_O))) ? (float*)out : nullptr;
   g.status = (int*)(ws + L->o.status);
   const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
@@ -509,6 +530,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       g.lists = (const int*)(ws + L->o.lists); g.lgate = (const float*)(ws + L->o.lgate);
       g.tiles = (const ShTile*)(ws + L->o.tiles); g.ntiles = (const int*)(ws + L->o.ntiles);
       g.b_rows_per_group = d.D; g.out0 = ws + L->o.v; g.status = status;
+      if (use_v32(L, S)) { g.v_f32 = 1; g.out0 = ws + L->o.v32; }
       // 256-row tiles (two accumulators sharing the weight operand): at most half the 128-row bound plus one per group
       dim3 grid(d.tile_rows_src == 256 ? d.max_tiles / 2 + d.H * d.E : d.max_tiles, 1);
       if (d.tile_rows_src == 256) {
@@ -521,6 +543,17 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       }
       if (rc) return rc;
       L->launches += 1;
+      if (g.v_f32) {
+        // the fp32 sums, rounded to fp16 once, become V
+        const size_t n4 = (size_t)d.N * HD / 4;
+        unsigned cgrid = (unsigned)((n4 + 255) / 256);
+        const unsigned ccap = L->sm_count > 0 ? 8u * (unsigned)L->sm_count : 1184u;
+        if (cgrid > ccap) cgrid = ccap;
+        if ((rc = launch_k(pdl && (S->pdl_mask & 4), sh_v32_to_f16_kernel, dim3(cgrid), dim3(256), 0, st,
+                           (const float4*)(ws + L->o.v32), (uint2*)(ws + L->o.v), n4)))
+          return rc;
+        L->launches += 1;
+      }
     }
   }
   if (overlap) SH_CUDA_CHECK(cudaStreamWaitEvent(st, S->ev_join, 0));

@@ -29,7 +29,8 @@ struct TcGateArgs {
   const float* gbias;        // [G]
   int* idx; float* gate;     // [2, N, H, k]
   int* blockcnt;             // [nblk, G] per-CTA selection histogram
-  __half* zero_v;            // [B, H, T, D] or nullptr
+  void* zero_v;              // [B, H, T, D] fp16 (or fp32: zero_v_f32) or nullptr
+  int zero_v_f32;
   float* zero_out;           // [N, M] or nullptr
   int* status;
   // fused sort (cooperative launch only)
@@ -129,14 +130,15 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       for (long i = et; i < total; i += NSEL) base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (g.zero_v) {
-      const int sh = d.D == 128 ? 4 : 3;                // 16-byte chunks per (token, head) row: D / 8
-      const int ch = et & ((1 << sh) - 1);
-      for (int tl = et >> sh; tl < nrows; tl += NSEL >> sh) {
+      const int row_bytes = d.D * (g.zero_v_f32 ? 4 : 2);  // one (token, head) row
+      const int cpr = row_bytes / 16;                      // 16-byte chunks per row (a power of two: 8..32)
+      const int ch = et & (cpr - 1);
+      for (int tl = et / cpr; tl < nrows; tl += NSEL / cpr) {
         const int tok = row0 + tl;
         const int bb = tok / d.T, tt = tok % d.T;
-        __half* p = g.zero_v + ((size_t)bb * d.H * d.T + tt) * d.D + ch * 8;
+        char* p = (char*)g.zero_v + ((size_t)bb * d.H * d.T + tt) * row_bytes + ch * 16;
         for (int hh = 0; hh < d.H; ++hh)
-          *reinterpret_cast<uint4*>(p + (size_t)hh * d.T * d.D) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(p + (size_t)hh * d.T * row_bytes) = make_uint4(0, 0, 0, 0);
       }
     }
     // ---- logits tile -> shared memory: warps 2..5, thread = token = TMEM lane -----------------

@@ -32,6 +32,7 @@ struct TcGemmArgs {
   const float2* rope;    // dense Q/K mode: (cos, sin) table [D/2, T] of the rotary embedding, or nullptr
   int* status;
   int* sched;            // persistent dense mode: {next tile, CTAs that made their final claim}, both 0 between launches
+  int v_f32;             // value experts: out0 is an fp32 accumulation buffer (fp32 vector reductions)
   int claimers;          // claiming CTAs (or CTA pairs) over all grids that share sched; 0: this grid's own
 };
 
@@ -244,8 +245,16 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
             __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * gate, __uint_as_float(v[2 * i + 1]) * gate);
             p[i] = *reinterpret_cast<uint32_t*>(&hv);
           }
+          if (g.v_f32) {
+            float* d32 = (float*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D + n0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              red_add_v4_f32(d32 + 4 * i, __uint_as_float(v[4 * i]) * gate, __uint_as_float(v[4 * i + 1]) * gate,
+                             __uint_as_float(v[4 * i + 2]) * gate, __uint_as_float(v[4 * i + 3]) * gate);
+          } else {
 #pragma unroll
           for (int i = 0; i < 4; ++i) red_add_v4_f16x2(dst + 8 * i, p[4 * i], p[4 * i + 1], p[4 * i + 2], p[4 * i + 3]);
+          }
         } else if (MODE == GEMM_O) {
           float* dst = (float*)g.out0 + (size_t)tok * d.M + n0;
 #pragma unroll

@@ -303,8 +303,16 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                 __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * gt, __uint_as_float(v[2 * i + 1]) * gt);
                 p[i] = *reinterpret_cast<uint32_t*>(&hv);
               }
+              if (g.v_f32) {
+                float* d32 = (float*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D + n0;
 #pragma unroll
-              for (int i = 0; i < 4; ++i) red_add_v4_f16x2(dst + 8 * i, p[4 * i], p[4 * i + 1], p[4 * i + 2], p[4 * i + 3]);
+                for (int i = 0; i < 8; ++i)
+                  red_add_v4_f32(d32 + 4 * i, __uint_as_float(v[4 * i]) * gt, __uint_as_float(v[4 * i + 1]) * gt,
+                                 __uint_as_float(v[4 * i + 2]) * gt, __uint_as_float(v[4 * i + 3]) * gt);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) red_add_v4_f16x2(dst + 8 * i, p[4 * i], p[4 * i + 1], p[4 * i + 2], p[4 * i + 3]);
+              }
             }
           }
         }
