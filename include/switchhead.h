@@ -14,8 +14,14 @@
  * Conventions
  *   - Every pointer is a DEVICE pointer unless the comment says "host".
  *   - Arrays are dense, row-major, in the layouts stated per argument.
- *   - `stream` is a cudaStream_t passed as void*; NULL is the default stream.  All device
- *     work of a call is enqueued on that stream; no call synchronises the device.
+ *   - `stream` is a cudaStream_t passed as void*; NULL is the default stream.  The device work
+ *     of a call is ordered on that stream: it starts after everything enqueued there before
+ *     the call and is complete before anything enqueued there after it.  The bf16 forward pass
+ *     also uses two non-blocking streams the layer owns (the dense Q/K projection runs on them
+ *     beside the gate and sort kernels, forked from and joined back into `stream` with
+ *     events), which matters to a caller that captures `stream` into a graph or gives it a
+ *     priority.  No call synchronises the device unless its comment says so.
+ *   - The release library reads nothing from the environment.
  *   - Functions returning int give SH_OK (0) or a negative SH_ERR_* code; sh_last_error()
  *     then holds a readable reason (thread-local, host string owned by the library).
  *   - The library owns only the handle.  x, out, the source weights and the workspace
@@ -45,7 +51,8 @@ enum {
   SH_ERR_WORKSPACE = -4,
   SH_ERR_CUDA = -5,
   SH_ERR_TIMEOUT = -6, /* a bounded device-side wait ran out (reported by sh_last_status) */
-  SH_ERR_BOUNDS = -7   /* a device-side index check failed (reported by sh_last_status)  */
+  SH_ERR_BOUNDS = -7   /* an index check of the debug library failed (sh_last_status), or
+                          sh_check_guards found a guard behind a workspace buffer overwritten */
 };
 
 /* Identifiers for sh_debug_buffer. */
@@ -134,10 +141,35 @@ int sh_set_rope(sh_layer* layer, double base, void* stream);
  * SH_ERR_INVALID_ARG).  out is fully overwritten.  Enqueues kernels only. */
 int sh_forward(sh_layer* layer, const void* x, void* out, void* stream);
 
+/* Kernel slots of sh_forward_stamped. */
+enum {
+  SH_STAMP_GATE = 0,   /* gate logits + top-k (+ the bucket sort when it is fused into this kernel) */
+  SH_STAMP_SORT = 1,   /* bucket sort as a kernel of its own                                        */
+  SH_STAMP_QK_A = 2,   /* dense Q/K projection: the grid launched ahead of the gate kernel (or the only grid) */
+  SH_STAMP_QK_B = 3,   /* ... the grid launched behind the sort, when the projection is split        */
+  SH_STAMP_V = 4,      /* value experts                                                              */
+  SH_STAMP_ATTN = 5,   /* attention                                                                  */
+  SH_STAMP_O = 6,      /* output experts + gate-weighted sum                                         */
+  SH_STAMP_COUNT = 7
+};
+
+/* Measurement aid: sh_forward, launched exactly as sh_forward launches it (same kernels, streams
+ * and launch attributes), with every kernel of the bf16 path writing three device-clock stamps
+ * (%globaltimer, nanoseconds): `resident` = its first CTA running, `start` = its first CTA past
+ * the wait for the kernel it depends on, `end` = its last CTA done.  Waits for `stream`, then
+ * fills the HOST array stamps[3][SH_STAMP_COUNT] = {resident[], start[], end[]}.  A kernel that
+ * did not run in this pass (and every kernel of the fp32 configuration, whose CUDA-core kernels
+ * carry no stamps) leaves resident = start = UINT64_MAX and end = 0.  The spans of kernels that
+ * overlap in time may be subtracted from one another: they share one clock. */
+int sh_forward_stamped(sh_layer* layer, const void* x, void* out, void* stream, uint64_t* stamps);
+
 /* Measurement aid: sh_forward with CUDA events recorded on `stream` at the stage boundaries;
  * waits for the stream, then writes to the HOST array stage_ms[6] the milliseconds of
  * {gate + top-k + sort, Q/K projection, value experts, attention, output experts, whole
- * pass}.  Creates and destroys its events, so unlike sh_forward it must not be stream-captured. */
+ * pass}.  To give the boundaries a meaning this call serialises the pass: ordinary launches on
+ * one stream, no kernel overlapping the next, so the stage times add up to MORE than a
+ * sh_forward takes; sh_forward_stamped shows what each kernel costs inside the real pass.
+ * Creates and destroys its events, so unlike sh_forward it must not be stream-captured. */
 int sh_forward_timed(sh_layer* layer, const void* x, void* out, void* stream, float* stage_ms);
 
 /* Gate stage alone, with its results exposed (any output pointer may be NULL):
@@ -188,6 +220,42 @@ int sh_debug_buffer(sh_layer* layer, int which, void** dev_ptr, size_t* bytes);
  * 0 if every kernel so far completed normally, else the first SH_ERR_TIMEOUT / SH_ERR_BOUNDS
  * code recorded by a kernel that gave up a bounded wait or skipped a bad index. */
 int sh_last_status(sh_layer* layer, void* stream);
+
+/* The first 16 words of the device status block, copied to the HOST array words[16] (drains
+ * `stream`): [0] the status word; [1..6] where the first bounded wait gave up - block, thread,
+ * shared-memory address of the barrier, parity waited for, grid size, block size; [8..11] the
+ * first failed index check of the debug library - site, value, limit, block. */
+int sh_status_block(sh_layer* layer, int32_t* words, void* stream);
+
+/* Clears the status block (asynchronously on `stream`): the status word, the diagnostics, and
+ * the tile and grid-barrier counters that a kernel which gave up may have left half-way.  After
+ * a non-zero sh_last_status, call this before the next sh_forward. */
+int sh_clear_status(sh_layer* layer, void* stream);
+
+/* Every sub-buffer of the workspace is followed by 256 guard bytes that sh_set_weights fills
+ * with a pattern.  Checks them all (one small kernel; drains `stream`): SH_OK, or SH_ERR_BOUNDS
+ * with the number of damaged words in sh_last_error() when some kernel wrote past the end of
+ * its buffer.  A testing aid that costs nothing in sh_forward. */
+int sh_check_guards(sh_layer* layer, void* stream);
+
+/* Self-tests of the error paths; neither touches memory outside the status block.
+ *   which = 0: a one-thread kernel waits, through the bounded wait every kernel of the library
+ *              uses, on a barrier that nothing signals, with a limit of `arg` nanoseconds
+ *              (at most 1e9).  It gives up, records SH_ERR_TIMEOUT and the diagnostics words, and
+ *              returns; the context stays usable.  sh_clear_status afterwards.
+ *   which = 1: (debug library only, else SH_ERR_UNSUPPORTED) runs the index check on the value
+ *              `arg` against the limit 10; a value outside records SH_ERR_BOUNDS and its
+ *              diagnostics.
+ * Enqueues one kernel on `stream`. */
+int sh_selftest(sh_layer* layer, int which, uint64_t arg, void* stream);
+
+/* 1 if the library was built with -DSH_DEBUG: every token-list entry, tile-table field and expert
+ * index read from memory is range-checked before it is used (a failed check records SH_ERR_BOUNDS
+ * and the access is skipped), and launch-structure switches are read from the environment when the
+ * weights are set (SH_NO_PDL, SH_NO_OVERLAP, SH_QK_ONE_GRID, SH_QK_SINGLE, SH_O_SINGLE,
+ * SH_NO_PERSISTENT, SH_SORT_SEPARATE, SH_ATTN_ADJACENT, SH_SIMT_STAGES: A/B and test aids).
+ * 0 for the release library, which has neither. */
+int sh_is_debug_build(void);
 
 /* Number of kernel launches the last sh_forward enqueued. */
 int sh_launch_count(const sh_layer* layer);

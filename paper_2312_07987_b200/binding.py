@@ -22,8 +22,10 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
 EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
-           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_gate_topk", "sh_debug_buffer", "sh_last_status",
-           "sh_launch_count", "sh_last_error", "sh_destroy"]
+           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
+           "sh_noalloc_gate_topk", "sh_debug_buffer", "sh_last_status", "sh_status_block", "sh_clear_status", "sh_check_guards",
+           "sh_selftest", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
+STAMP_KERNELS = ["gate", "sort", "qk_a", "qk_b", "v", "attn", "o"]
 
 
 def _load() -> ctypes.CDLL:
@@ -50,6 +52,18 @@ def _load() -> ctypes.CDLL:
     lib.sh_forward.argtypes = [vp, vp, vp, vp]
     lib.sh_forward_timed.restype = i32
     lib.sh_forward_timed.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float)]
+    lib.sh_forward_stamped.restype = i32
+    lib.sh_forward_stamped.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ctypes.c_uint64)]
+    lib.sh_status_block.restype = i32
+    lib.sh_status_block.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+    lib.sh_clear_status.restype = i32
+    lib.sh_clear_status.argtypes = [vp, vp]
+    lib.sh_check_guards.restype = i32
+    lib.sh_check_guards.argtypes = [vp, vp]
+    lib.sh_selftest.restype = i32
+    lib.sh_selftest.argtypes = [vp, i32, ctypes.c_uint64, vp]
+    lib.sh_is_debug_build.restype = i32
+    lib.sh_is_debug_build.argtypes = []
     lib.sh_gate_topk.restype = i32
     lib.sh_gate_topk.argtypes = [vp] * 7
     lib.sh_noalloc_gate_topk.restype = i32
@@ -153,6 +167,28 @@ class Layer:
         ms = (ctypes.c_float * 6)()
         _check(lib.sh_forward_timed(self.handle, _ptr(x), _ptr(out), _stream(), ms))
         return list(ms)
+
+    def sh_forward_stamped(self, x: torch.Tensor, out: torch.Tensor):
+        """One forward pass launched as sh_forward launches it; returns {kernel: (resident, start, end)} in
+        nanoseconds of the device clock for the kernels that ran (see STAMP_KERNELS)."""
+        n = len(STAMP_KERNELS)
+        buf = (ctypes.c_uint64 * (3 * n))()
+        _check(lib.sh_forward_stamped(self.handle, _ptr(x), _ptr(out), _stream(), buf))
+        return {name: (buf[i], buf[n + i], buf[2 * n + i]) for i, name in enumerate(STAMP_KERNELS) if buf[2 * n + i] != 0}
+
+    def sh_status_block(self):
+        w = (ctypes.c_int32 * 16)()
+        _check(lib.sh_status_block(self.handle, w, _stream()))
+        return list(w)
+
+    def sh_clear_status(self) -> None:
+        _check(lib.sh_clear_status(self.handle, _stream()))
+
+    def sh_check_guards(self) -> None:
+        _check(lib.sh_check_guards(self.handle, _stream()))
+
+    def sh_selftest(self, which: int, arg: int) -> None:
+        _check(lib.sh_selftest(self.handle, which, arg, _stream()))
 
     def sh_gate_topk(self, x: torch.Tensor):
         d_model, H, D, E, k = self.dims

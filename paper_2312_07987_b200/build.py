@@ -8,6 +8,10 @@ import subprocess
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libswitchhead.so")
+# The debug library: same sources with -DSH_DEBUG (index checks before every list / tile-table /
+# expert-index use, and launch-structure switches read from the environment).  Tests load it through
+# SWITCHHEAD_LIB; the release library reads nothing from the environment.
+DEBUG_LIB_PATH = os.path.join(PKG_DIR, "libswitchhead_debug.so")
 SOURCES = ["sh_api.cu", "sh_tc.cu", "sh_static.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-shared", "-Xcompiler", "-fPIC"]
@@ -20,19 +24,20 @@ def _nvcc() -> str:
     return exe
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def is_stale(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps.append(os.path.join(PKG_DIR, "..", "include", "switchhead.h"))
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not is_stale():
-        return LIB_PATH
-    cmd = [_nvcc(), *NVCC_FLAGS, "-o", LIB_PATH, *[os.path.join(CSRC, s) for s in SOURCES]]
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    out = DEBUG_LIB_PATH if debug else LIB_PATH
+    if not force and not is_stale(out):
+        return out
+    cmd = [_nvcc(), *NVCC_FLAGS, *(["-DSH_DEBUG"] if debug else []), "-o", out, *[os.path.join(CSRC, s) for s in SOURCES]]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -41,8 +46,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         print(res.stderr)
-    return LIB_PATH
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    import sys
+    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

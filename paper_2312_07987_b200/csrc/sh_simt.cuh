@@ -173,7 +173,10 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
     const int side = grp / d.H, h = grp % d.H;
     unsigned mask = 0;
     if (tl < nrows)
-      for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[side * 128 * per_tok + (tl * d.H + h) * d.k + j];
+      for (int j = 0; j < d.k; ++j) {
+        const int ev = s_idx[side * 128 * per_tok + (tl * d.H + h) * d.k + j];
+        if (SH_INDEX_OK(ev, d.E, d.status, SH_SITE_SORT_EXPERT)) mask |= 1u << ev;
+      }
     for (int e = 0; e < d.E; ++e) {
       const unsigned bal = __ballot_sync(0xffffffffu, (mask >> e) & 1u);
       if (lane == 0) s_wcnt[(grp * d.E + e) * 4 + twarp] = __popc(bal);
@@ -187,7 +190,10 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
       const int sel = side * 128 * per_tok + (tl * d.H + h) * d.k;
       unsigned mask = 0;
       if (tl < nrows)
-        for (int j = 0; j < d.k; ++j) mask |= 1u << s_idx[sel + j];
+        for (int j = 0; j < d.k; ++j) {
+          const int ev = s_idx[sel + j];
+          if (SH_INDEX_OK(ev, d.E, d.status, SH_SITE_SORT_EXPERT)) mask |= 1u << ev;
+        }
       for (int e = 0; e < d.E; ++e) {
         const bool mine = (mask >> e) & 1u;
         const unsigned bal = __ballot_sync(0xffffffffu, mine);
@@ -199,8 +205,10 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
           for (int j = 0; j < d.k; ++j)
             if (s_idx[sel + j] == e) gv = s_gt[sel + j];
           const size_t dst = (size_t)grp * d.N * d.k + s_off[b] + s_pre[b] + pos;
-          lists[dst] = t;
-          lgate[dst] = gv;
+          if (SH_INDEX_OK(s_off[b] + s_pre[b] + pos, (long long)d.N * d.k, d.status, SH_SITE_SORT_SLOT)) {
+            lists[dst] = t;
+            lgate[dst] = gv;
+          }
         }
       }
     }
@@ -246,9 +254,15 @@ sh_sort_kernel(const int* __restrict__ idx, const float* __restrict__ gate, cons
   // programmatic dependent launch (no-ops in an ordinary launch): let the next kernel in the
   // stream become resident, then wait for the gate kernel's selections to be complete and visible
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_SORT);
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_SORT);
   sh_sort_block(idx, gate, blockcnt, offsets, lists, lgate, tiles, ntiles, d, s_sort, (int)threadIdx.x, (int)blockDim.x, (int)blockIdx.x,
                 false, [] { __syncthreads(); });
+  if (d.stamps) {
+    __syncthreads();
+    if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_SORT);
+  }
 }
 
 static inline int sh_sort_threads(const ShDims& d) {

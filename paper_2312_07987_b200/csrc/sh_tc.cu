@@ -1,5 +1,6 @@
 // Tensor-core (tcgen05) path of the bf16 configuration: tensor maps and launch sequence.
 #include <cstdlib>
+#include <mutex>
 #include <new>
 #include <utility>
 
@@ -7,7 +8,6 @@
 #include "sh_simt.cuh"
 #include "sh_tc_gemm.cuh"
 #include "sh_tc_pgemm.cuh"
-#include "sh_tc_attn.cuh"
 #include "sh_tc_attn2.cuh"
 #include "sh_tc_gate.cuh"
 #include "sh_tc_oproj2.cuh"
@@ -76,22 +76,27 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
   CUtensorMap map_wqk, map_wqk128, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
-  int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel
-  int qk_bn, o_bn, qk_variant;
-  int o_pair, o_pairs_max;       // output projection on CTA pairs; clusters the device holds at once
-  int qk_pair, qk_pairs_max;     // the same for the dense Q/K projection
-  int gate_coop;                 // 1: the gate kernel can be launched cooperatively (fused sort), -1: it cannot
-  int persistent;       // 1 = persistent Q/K and value-expert GEMMs (default); 0 = one CTA per tile (experiment switch)
-  int attn_single_tile; // 1 = one 128-query tile per CTA (experiment switch)
-  int o_scatter;        // 1 = grouped GEMM with scatter-add epilogue instead of the on-chip sum (experiment switch)
-  int simt_mask;        // stages forced onto the CUDA-core kernels (testing aid)
-  // fork/join: the Q/K projection does not depend on the gate and sort kernels, so it runs on a
-  // side stream between two events recorded on the caller's stream
-  bool pdl = true;
-  int pdl_mask = 31;
-  cudaStream_t side = nullptr;
+  CUtensorMap map_x;             // tensor map of the last x pointer seen (x_cached)
+  const void* x_cached = nullptr;
+  int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel (more than 256 gate columns)
+  int qk_bn;            // column tile of the dense projection: 256 (CTA pairs / persistent) when 2*H*D allows, else 128
+  int o_pairs_max;      // clusters of the CTA-pair output projection the device holds at once (0: not asked yet, -1: none)
+  int qk_pairs_max;     // the same for the dense Q/K projection
+  int gate_coop;        // 1: the gate kernel can be launched cooperatively (fused sort), -1: it cannot
+  // Launch-structure switches.  The release library fixes them here; a library built with SH_DEBUG
+  // reads them from the environment once, in sh_tc_prepare, for A/B runs and for the tests that
+  // drive the less-travelled launch paths.
+  bool pdl = true;          // kernels of the caller's stream chained by programmatic dependent launch
+  bool overlap = true;      // Q/K projection on a side stream beside gate + sort
+  bool qk_two_grids = true; // ... as two grids around the gate kernel
+  bool qk_pair = true;      // CTA-pair Q/K kernel (else single-CTA persistent)
+  bool o_pair = true;       // CTA-pair output projection for k <= 3 (else single-CTA)
+  bool persistent = true;   // persistent Q/K and value-expert GEMMs (else one CTA per tile)
+  bool fused_sort = true;   // sort fused into the gate kernel when it needs at most half of the SMs
+  bool attn_balanced = true;
+  int simt_mask = 0;        // SH_DEBUG only: stages forced onto the CUDA-core kernels
+  cudaStream_t side = nullptr, side2 = nullptr;   // Q/K grids A and B
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_join2 = nullptr;
-  cudaStream_t side2 = nullptr;   // second grid of a split Q/K projection
 };
 
 constexpr int QK_STAGES = 4;
@@ -148,9 +153,11 @@ static int max_pairs(K kern, int block, size_t smem) {
 struct SmemAttr { const void* fn; int dev; int bytes; };
 static SmemAttr g_smem_attr[128];
 static int g_smem_attr_n = 0;
+static std::mutex g_smem_attr_mutex;     // layers may be driven from several host threads
 
 template <typename K>
 static int set_smem(K kernel, int bytes) {
+  std::lock_guard<std::mutex> lock(g_smem_attr_mutex);
   int dev = 0;
   SH_CUDA_CHECK(cudaGetDevice(&dev));
   const void* fn = (const void*)kernel;
@@ -190,34 +197,35 @@ int sh_tc_prepare(sh_layer* L) {
   char* ws = L->ws;
   const int HD = d.H * d.D;
   const int nproj = L->dense ? 3 : 2;
-  S->attn_single_tile = getenv("SH_ATTN_SINGLE") ? 1 : 0;
-  S->persistent = getenv("SH_NO_PERSISTENT") ? 0 : 1;
-  const char* ov = getenv("SH_O_SCATTER");
-  S->o_scatter = ov ? atoi(ov) : 0;
-  const char* qv = getenv("SH_QK_VARIANT");
-  S->qk_variant = qv ? atoi(qv) : (((L->dense ? 3 : 2) * d.H * d.D) % 256 == 0 ? 2 : 0);
-  S->qk_bn = (S->qk_variant == 2) ? 256 : 128;
-  // Default: the kernels of the caller's stream are chained by programmatic dependent launch (each
-  // becomes resident while the one before it drains, and waits on the device for its results);
-  // the dense Q/K projection, which needs nothing from the gate and sort kernels, is launched the
-  // ordinary way on a side stream so that it runs beside them.  SH_NO_PDL=1: ordinary launches only.
+#ifdef SH_DEBUG
+  // A/B switches of the debug library (read once, here)
   S->pdl = !getenv("SH_NO_PDL");
-  if (const char* m = getenv("SH_PDL_MASK")) S->pdl_mask = atoi(m);   // debugging: bit 0 sort, 1 Q/K, 2 V, 3 attention, 4 O
-  if (!L->dense && !getenv("SH_NO_OVERLAP")) {
+  S->overlap = !getenv("SH_NO_OVERLAP");
+  S->qk_two_grids = !getenv("SH_QK_ONE_GRID");
+  S->qk_pair = !getenv("SH_QK_SINGLE");
+  S->o_pair = !getenv("SH_O_SINGLE");
+  S->persistent = !getenv("SH_NO_PERSISTENT");
+  S->fused_sort = !getenv("SH_SORT_SEPARATE");
+  S->attn_balanced = !getenv("SH_ATTN_ADJACENT");
+  if (const char* env = getenv("SH_SIMT_STAGES")) S->simt_mask = atoi(env);   // bit mask gate=1, qk=2, v=4, attention=8, o=16
+#endif
+  // 256-column tiles (CTA pairs, or the persistent single-CTA kernel) need the projection's width to
+  // be a multiple of 256; other widths take the one-CTA-per-tile kernel with 128-column tiles
+  S->qk_bn = (nproj * HD) % 256 == 0 ? 256 : 128;
+  // The kernels of the caller's stream are chained by programmatic dependent launch (each becomes
+  // resident while the one before it drains, and waits on the device for its results); the dense
+  // Q/K projection, which needs nothing from the gate and sort kernels, is launched the ordinary way
+  // on side streams so that it runs beside them.
+  if (!L->dense && S->overlap) {
     SH_CUDA_CHECK(cudaStreamCreateWithFlags(&S->side, cudaStreamNonBlocking));
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_fork, cudaEventDisableTiming));
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_join, cudaEventDisableTiming));
     SH_CUDA_CHECK(cudaStreamCreateWithFlags(&S->side2, cudaStreamNonBlocking));
     SH_CUDA_CHECK(cudaEventCreateWithFlags(&S->ev_join2, cudaEventDisableTiming));
   }
-  S->o_bn = 128;
-  S->o_pair = getenv("SH_O_SINGLE") == nullptr;     // CTA-pair output projection unless switched off
   S->o_pairs_max = 0;
-  S->qk_pair = getenv("SH_QK_SINGLE") == nullptr;
   S->qk_pairs_max = 0;
   S->gate_coop = 0;
-  const char* env = getenv("SH_SIMT_STAGES");
-  S->simt_mask = env ? atoi(env) : 0;
   if (L->sm_count == 0) {
     int dev = 0;
     SH_CUDA_CHECK(cudaGetDevice(&dev));
@@ -227,19 +235,19 @@ int sh_tc_prepare(sh_layer* L) {
   // enough of them to fill the SMs one and a half times
   const long long slots = (long long)d.N * d.H * d.k;
   const bool big = slots / 256 >= (3ll * L->sm_count) / 2;
-  // (with a shared selection the destination-side consumers of the tile table -- the CUDA-core and
-  //  scatter-add output projections, debugging paths here -- read the source side's 128-row tiles)
-  const bool dst_reads_src_tiles = L->d.sides == 1 && ((S->simt_mask & SH_STAGE_O) || getenv("SH_O_SCATTER"));
-  L->d.tile_rows_src = (L->dense || (S->simt_mask & SH_STAGE_V) || getenv("SH_V_TILE128") || !big || dst_reads_src_tiles) ? 128 : 256;
+  // (the CUDA-core stages of the debug library read 128-row tiles; with a shared selection its output
+  //  projection reads the source side's table)
+  const bool simt_tiles = (S->simt_mask & SH_STAGE_V) || (L->d.sides == 1 && (S->simt_mask & SH_STAGE_O));
+  L->d.tile_rows_src = (L->dense || simt_tiles || !big) ? 128 : 256;
   int rc;
   if ((rc = sh_tc_encode_2d(&S->map_wqk, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, S->qk_bn))) return rc;
   if ((rc = sh_tc_encode_2d(&S->map_wqk128, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, 128))) return rc;
   if (!L->dense) {
     if ((rc = sh_tc_encode_2d(&S->map_wv, 0, ws + L->o.wv, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
-    if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, S->o_bn))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 128))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo256, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 256))) return rc;
   } else {
-    if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, S->o_bn))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, 128))) return rc;
   }
   S->gate_gp = 0;
   if (!L->dense && (d.G + 15) / 16 * 16 <= 256) {
@@ -253,6 +261,19 @@ int sh_tc_prepare(sh_layer* L) {
   return SH_OK;
 }
 
+// The tensor map of x [N, M] (128-token x 64-column boxes); kept for the pointer last seen, since a
+// caller usually passes the same one or two buffers pass after pass.
+static int x_map(sh_layer* L, const void* x, const CUtensorMap** out) {
+  TcState* S = (TcState*)L->tc;
+  if (S->x_cached != x) {
+    const ShDims& d = L->d;
+    if (int rc = sh_tc_encode_2d(&S->map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128)) return rc;
+    S->x_cached = x;
+  }
+  *out = &S->map_x;
+  return SH_OK;
+}
+
 // The gate kernel's x stream comes cold from HBM (~1.2 us per box round trip), so what bounds its
 // main loop is the bytes in flight per CTA: 8 stages when they fit, else 4.
 static int gate_smem_bytes(int Gp, int G, int stages) {
@@ -262,74 +283,49 @@ static int gate_smem_bytes(int Gp, int G, int stages) {
   return bar_off + 256 + 3 * G * 4 + 1024;
 }
 
-// k >= 3: the value experts accumulate a token's k contributions in an fp32 buffer (fp32 vector
-// reductions) that is rounded to fp16 once, instead of k fp16 reductions into V itself - those cost
-// up to k * 2^-11 relative on rows of which the first tokens of a sequence, attending to few keys,
-// pass nearly unaveraged into an output far above the global RMS the tolerance is measured in.
-static bool use_v32(const sh_layer* L, const TcState* S) {
-  return L->dtype == SH_BF16 && !L->dense && L->d.k >= 3 && !(S->simt_mask & SH_STAGE_V);
-}
-
-static __global__ void __launch_bounds__(256)
-sh_v32_to_f16_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, size_t n4) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
-    const float4 v = src[i];
-    const __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
-    dst[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
-  }
-}
-
-// Gate + top-k + bucket sort.  With zero_for_forward the fused kernel also clears V and out.
+// Gate + top-k + bucket sort.  With zero_for_forward the gate kernel also clears the value buffer.
 static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_forward, cudaStream_t st, bool sort_apart = false) {
   TcState* S = (TcState*)L->tc;
   const ShDims& d = L->d;
   char* ws = L->ws;
   int rc;
   if (!S->gate_gp || (S->simt_mask & SH_STAGE_GATE)) {
+    // more than 256 gate columns (or the debug library's switch): the CUDA-core gate kernel
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_GATE, x, nullptr, st))) return rc;
     if (zero_for_forward) {
       SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * d.H * d.D * 2, st));
-      if (use_v32(L, S)) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v32, 0, (size_t)d.N * d.H * d.D * 4, st));
-      SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
+      if (S->simt_mask & SH_STAGE_O) SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
       L->launches += 2;
     }
     return SH_OK;
   }
-  CUtensorMap map_x;
-  if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
+  const CUtensorMap* map_x;
+  if ((rc = x_map(L, x, &map_x))) return rc;
   TcGateArgs g{};
   g.d = d; g.Gp = S->gate_gp; g.gbias = (const float*)(ws + L->o.gbias);
   g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
   g.blockcnt = (int*)(ws + L->o.blockcnt);
-  g.zero_v_f32 = use_v32(L, S) ? 1 : 0;
-  g.zero_v = zero_for_forward ? (void*)(ws + (g.zero_v_f32 ? L->o.v32 : L->o.v)) : nullptr;
-  g.zero_out = (zero_for_forward && (S->o_scatter || (S->simt_mask & SH_STAGE_O))) ? (float*)out : nullptr;
+  g.zero_v = zero_for_forward ? (void*)(ws + L->o.v) : nullptr;
+  g.zero_out = (zero_for_forward && (S->simt_mask & SH_STAGE_O)) ? (float*)out : nullptr;
   g.status = (int*)(ws + L->o.status);
   const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
   const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
   if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
   // In a forward pass only the value experts read sorted lists (the output projection works from
   // idx / gate, token tile by token tile), so only the source side is sorted there -- unless the
-  // scatter-add or CUDA-core output projection (debugging paths) is selected.  The histogram stride
-  // stays G; the sort's loops run over sides * H groups.
+  // debug library's CUDA-core output projection is selected.  The histogram stride stays G; the
+  // sort's loops run over sides * H groups.
   ShDims ds = d;
-  if (zero_for_forward && !S->o_scatter && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
+  if (zero_for_forward && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
   // Fused sort: when every CTA of the gate kernel can be resident at once (cooperative launch) and the
   // sort's scratch fits behind the logits tile in the idle operand ring, the gate kernel places the
   // tokens itself and there is no sort kernel.  Used when the gate kernel needs at most half of the SMs:
   // 114.8 -> 110.7 us per forward at 8192 tokens (64 CTAs), but 270.7 -> 273.3 at 16384 (128 CTAs that
   // must all find a free SM before any of them starts).
-  if (L->sm_count == 0) {
-    int dev = 0;
-    SH_CUDA_CHECK(cudaGetDevice(&dev));
-    SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
-  }
   {
     const int stage = 128 * 64 * 2 + ((S->gate_gp * 128 + 1023) & ~1023);
     const int pipe = (deep ? 8 : 4) * stage, stag = 128 * (S->gate_gp + 1) * 4;
-    g.fused = !getenv("SH_SORT_SEPARATE") && 2 * d.nblk <= L->sm_count && ((stag + 15) & ~15) + (int)sh_sort_smem_bytes(d) <= pipe;
+    g.fused = S->fused_sort && 2 * d.nblk <= L->sm_count && ((stag + 15) & ~15) + (int)sh_sort_smem_bytes(d) <= pipe;
     if (g.fused && S->gate_coop == 0) {
       int dev = 0, coop = 0, per_sm = 0;
       SH_CUDA_CHECK(cudaGetDevice(&dev));
@@ -343,7 +339,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.sort_sides = ds.sides; g.tile_rows_src = d.tile_rows_src; g.max_tiles = d.max_tiles;
   g.offsets = (int*)(ws + L->o.offsets); g.lists = (int*)(ws + L->o.lists); g.lgate = (float*)(ws + L->o.lgate);
   g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
-  g.gridbar = (int*)(ws + L->o.status) + 24;
+  g.gridbar = (int*)(ws + L->o.status) + SH_ST_GRIDBAR;
   if (g.fused) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(d.nblk); cfg.blockDim = dim3(GATE_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
@@ -351,21 +347,20 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    if (deep) SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, sh_tc_gate_kernel<8>, map_x, S->map_wgate, g));
-    else SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, sh_tc_gate_kernel<4>, map_x, S->map_wgate, g));
+    if (deep) SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, sh_tc_gate_kernel<8>, *map_x, S->map_wgate, g));
+    else SH_CUDA_CHECK(cudaLaunchKernelEx(&cfg, sh_tc_gate_kernel<4>, *map_x, S->map_wgate, g));
     L->launches += 1;
     return SH_OK;
   }
-  if (deep) sh_tc_gate_kernel<8><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
-  else sh_tc_gate_kernel<4><<<d.nblk, GATE_THREADS, smem, st>>>(map_x, S->map_wgate, g);
+  if (deep) sh_tc_gate_kernel<8><<<d.nblk, GATE_THREADS, smem, st>>>(*map_x, S->map_wgate, g);
+  else sh_tc_gate_kernel<4><<<d.nblk, GATE_THREADS, smem, st>>>(*map_x, S->map_wgate, g);
   size_t ssm = sh_sort_smem_bytes(d);
   // sort_apart: ask for enough shared memory that a sort block fits beside a gate CTA but not beside a
   // ~198 KB GEMM CTA: next to the Q/K projection's CTAs (whose waiting warps poll) a block takes
   // 11 us instead of 4.7
   if (sort_apart && ssm < 40 * 1024) ssm = 40 * 1024;
-  // (sort blocks become resident early and share SMs with the 190 KB GEMM CTAs that follow)
   if ((rc = set_smem(sh_sort_kernel, (int)ssm))) return rc;
-  if ((rc = launch_k(S->pdl && !L->ev && (S->pdl_mask & 1), sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(ds)), ssm, st,
+  if ((rc = launch_k(S->pdl && !L->ev, sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(ds)), ssm, st,
                      (const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate), (const int*)(ws + L->o.blockcnt),
                      (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists), (float*)(ws + L->o.lgate),
                      (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), ds)))
@@ -396,6 +391,22 @@ static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const T
   return SH_OK;
 }
 
+using QkPS = QkPairSmem<6>;
+
+// Clusters of the CTA-pair Q/K kernel the device holds at once (looked up once per layer; -1: none).
+static int qk_pairs_max(TcState* S) {
+  if (S->qk_pairs_max == 0) {
+    if (set_smem(sh_tc_qk_pair_kernel<6>, QkPS::TOTAL) != SH_OK) return S->qk_pairs_max = -1;
+    S->qk_pairs_max = max_pairs(sh_tc_qk_pair_kernel<6>, 320, QkPS::TOTAL);
+    if (S->qk_pairs_max <= 0) S->qk_pairs_max = -1;
+  }
+  return S->qk_pairs_max;
+}
+
+// The launches of one forward pass after grid A of a split Q/K projection is out (see sh_tc_forward).
+static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t st, const CUtensorMap& map_x, bool overlap,
+                           int qkA, int qkB, TcGemmArgs& qg);
+
 int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   TcState* S = (TcState*)L->tc;
   if (!S) { sh_set_error("tensor-core state missing: call sh_set_weights first"); return SH_ERR_NOT_CONFIGURED; }
@@ -405,71 +416,84 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   int rc;
   const int simt = S->simt_mask;
   int* status = (int*)(ws + L->o.status);
-  const bool pdl = S->pdl && !L->ev;                       // stage-timed runs use ordinary launches
 
   sh_mark(L, 0, st);
-  // stage-timed runs stay serial so that the stage boundaries mean something
+  // stage-timed runs (sh_forward_timed) stay serial so that the stage boundaries mean something
   const bool overlap = S->side && !L->ev && !(simt & SH_STAGE_QK);
-  cudaStream_t qst = st;
   if (overlap) {
     SH_CUDA_CHECK(cudaEventRecord(S->ev_fork, st));
     SH_CUDA_CHECK(cudaStreamWaitEvent(S->side, S->ev_fork, 0));
-    qst = S->side;
   }
-  CUtensorMap map_x;
-  if ((rc = sh_tc_encode_2d(&map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128))) return rc;
-  // Split Q/K projection (SH_QK_ONE_GRID switches it off).  A grid whose CTAs cannot all start at
-  // once (the gate kernel holds SMs) keeps every kernel launched after it, in any stream, from
-  // starting: the sort kernel, launched to become resident while the gate kernel runs, then starts
-  // 4-8 us after the gate kernel has ended.  And launched after gate and sort, the projection starts
-  // two launch latencies late when the host is not running ahead (a single forward pass at the
-  // 262M-scale shape: ~102 us instead of ~107).  So the projection goes out as two grids of CTA pairs
-  // that claim tiles from one counter: grid A, launched BEFORE the gate kernel, sized for the SMs the
-  // gate kernel does not need; grid B, launched AFTER the sort kernel on a stream of its own, takes
-  // over the gate kernel's SMs when they come free.  The sort blocks are kept off the SMs of grid A
-  // (see tc_gate_sort): without that, about one process in six ran every pass 6-8 us slower (as every
-  // process does when grid B's stream is given a higher priority than the caller's: grid B's CTAs
-  // placed ahead of the sort and value-expert kernels' CTAs, and as happens with a five-stage grid
-  // B, whose CTAs fit beside the sort blocks and slow them down); with it, ten processes in a row ran
-  // 109.8-111.9 us per pass against 111.7-114.7 with one grid, and 265 against 270.5 at 16384 tokens.
+  const CUtensorMap* map_x;
+  if ((rc = x_map(L, x, &map_x))) return rc;
+  // Split Q/K projection.  A grid whose CTAs cannot all start at once (the gate kernel holds SMs)
+  // keeps every kernel launched after it, in any stream, from starting: the sort kernel, launched to
+  // become resident while the gate kernel runs, then starts 4-8 us after the gate kernel has ended.
+  // And launched after gate and sort, the projection starts two launch latencies late when the host
+  // is not running ahead (a single forward pass at the 262M-scale shape: ~102 us instead of ~107).
+  // So the projection goes out as two grids of CTA pairs that claim tiles from one counter: grid A,
+  // launched BEFORE the gate kernel, sized for the SMs the gate kernel does not need; grid B, launched
+  // AFTER the sort kernel on a stream of its own, takes over the gate kernel's SMs when they come
+  // free.  The sort blocks are kept off the SMs of grid A (see tc_gate_sort): without that, about one
+  // process in six ran every pass 6-8 us slower (as every process does when grid B's stream is given
+  // a higher priority than the caller's: grid B's CTAs placed ahead of the sort and value-expert
+  // kernels' CTAs, and as happens with a five-stage grid B, whose CTAs fit beside the sort blocks and
+  // slow them down); with it, ten processes in a row ran 109.8-111.9 us per pass against 111.7-114.7
+  // with one grid, and 265 against 270.5 at 16384 tokens.
   int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
   TcGemmArgs qg{};
-  if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_variant == 2 && S->persistent && S->qk_pair && S->side2 &&
-      !getenv("SH_QK_ONE_GRID")) {
-    using PS = QkPairSmem<6>;
-    if ((rc = set_smem(sh_tc_qk_pair_kernel<6>, PS::TOTAL))) return rc;
-    if (S->qk_pairs_max == 0) {
-      S->qk_pairs_max = max_pairs(sh_tc_qk_pair_kernel<6>, 320, PS::TOTAL);
-      if (S->qk_pairs_max <= 0) S->qk_pairs_max = -1;
-    }
-    if (S->qk_pairs_max > 0) {
-      const int ptiles = ((d.N + 255) / 256) * ((2 * HD + 255) / 256);
-      const int pairs = ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max;
-      // (one gate CTA per SM; running two per SM with half the stages, to leave grid A more SMs when
-      //  there are more gate CTAs than half the SMs, made the gate kernel 2.4 us slower and the layer
-      //  8-10 us slower at 16384 tokens)
-      int gate_sms = d.nblk;
-      if (gate_sms > L->sm_count - 8) gate_sms = L->sm_count - 8;
-      qkA = (L->sm_count - gate_sms) / 2;
-      if (qkA > pairs) qkA = pairs;
-      qkB = pairs - qkA;
-      qg.d = d; qg.K = d.M; qg.ncols = 2 * HD; qg.nrows = d.N;
-      qg.out0 = ws + L->o.q; qg.out1 = ws + L->o.k; qg.out2 = ws + L->o.v;
-      qg.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
-      qg.status = status; qg.sched = status + 16; qg.claimers = qkA + qkB;
-      qg.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
-      if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkA), dim3(320), PS::TOTAL, S->side, map_x, S->map_wqk128, qg))) return rc;
-      L->launches += 1;
-    }
+  if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_bn == 256 && S->persistent && S->qk_pair &&
+      S->qk_two_grids && qk_pairs_max(S) > 0) {
+    const int ptiles = ((d.N + 255) / 256) * ((2 * HD + 255) / 256);
+    const int pairs = ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max;
+    // (one gate CTA per SM; running two per SM with half the stages, to leave grid A more SMs when
+    //  there are more gate CTAs than half the SMs, made the gate kernel 2.4 us slower and the layer
+    //  8-10 us slower at 16384 tokens)
+    int gate_sms = d.nblk;
+    if (gate_sms > L->sm_count - 8) gate_sms = L->sm_count - 8;
+    qkA = (L->sm_count - gate_sms) / 2;
+    if (qkA > pairs) qkA = pairs;
+    qkB = pairs - qkA;
+    qg.d = d; qg.K = d.M; qg.ncols = 2 * HD; qg.nrows = d.N;
+    qg.out0 = ws + L->o.q; qg.out1 = ws + L->o.k; qg.out2 = ws + L->o.v;
+    qg.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+    qg.status = status; qg.sched = status + SH_ST_SCHED; qg.claimers = qkA + qkB;
+    qg.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
+    qg.stamp_id = SH_K_QK_A;
+    if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkA), dim3(320), QkPS::TOTAL, S->side, *map_x, S->map_wqk128, qg))) return rc;
+    L->launches += 1;
   }
+  rc = tc_forward_rest(L, x, out, st, *map_x, overlap, qkA, qkB, qg);
+  if (rc != SH_OK && qkA > 0) {
+    // Grid A is out and something after it could not be launched: the tile counter it shares with
+    // grid B would keep this pass's claims, and the caller's stream would never join the side
+    // streams.  Put both right, so that a later pass starts from a clean state.
+    cudaMemsetAsync(status + SH_ST_SCHED, 0, 8, S->side);
+    cudaEventRecord(S->ev_join, S->side);
+    cudaStreamWaitEvent(st, S->ev_join, 0);
+    cudaGetLastError();
+  }
+  return rc;
+}
+
+static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t st, const CUtensorMap& map_x, bool overlap,
+                           int qkA, int qkB, TcGemmArgs& qg) {
+  TcState* S = (TcState*)L->tc;
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const int HD = d.H * d.D;
+  int rc;
+  const int simt = S->simt_mask;
+  int* status = (int*)(ws + L->o.status);
+  const bool pdl = S->pdl && !L->ev;                       // stage-timed runs use ordinary launches
   if (!L->dense) {
     if ((rc = tc_gate_sort(L, x, out, true, st, qkA > 0))) return rc;
   }
   sh_mark(L, 1, st);
   if (qkA > 0 && qkB > 0) {
-    using PS = QkPairSmem<6>;
     SH_CUDA_CHECK(cudaStreamWaitEvent(S->side2, S->ev_fork, 0));
-    if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkB), dim3(320), PS::TOTAL, S->side2, map_x, S->map_wqk128, qg))) return rc;
+    qg.stamp_id = SH_K_QK_B;
+    if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkB), dim3(320), QkPS::TOTAL, S->side2, map_x, S->map_wqk128, qg))) return rc;
     SH_CUDA_CHECK(cudaEventRecord(S->ev_join2, S->side2));
     L->launches += 1;
   }
@@ -479,40 +503,32 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   } else if (simt & SH_STAGE_QK) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_QK, x, out, st))) return rc;
   } else {
-    cudaStream_t st = qst;                                  // Q/K projection: side stream when overlapping
+    cudaStream_t qst = overlap ? S->side : st;              // side stream when overlapping
     TcGemmArgs g{};
     g.d = d; g.K = d.M; g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
     g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
     g.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
     g.status = status;
-    g.sched = status + 16;
+    g.sched = status + SH_ST_SCHED;
     g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
+    g.stamp_id = SH_K_QK_A;
     dim3 grid(d.nblk, (g.ncols + S->qk_bn - 1) / S->qk_bn);
-    switch (S->qk_variant) {
-      case 1: rc = launch_gemm<128, 3, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
-      case 2: {
-        if (S->persistent && S->qk_pair) {
-          // CTA pairs: 256 x 256 tiles, each CTA loads half of the weight rows
-          using PS = QkPairSmem<6>;
-          if ((rc = set_smem(sh_tc_qk_pair_kernel<6>, PS::TOTAL))) return rc;
-          if (S->qk_pairs_max == 0) {
-            S->qk_pairs_max = max_pairs(sh_tc_qk_pair_kernel<6>, 320, PS::TOTAL);
-            if (S->qk_pairs_max <= 0) S->qk_pairs_max = -1;
-          }
-          if (S->qk_pairs_max > 0) {
-            const int ptiles = ((d.N + 255) / 256) * ((g.ncols + 255) / 256);
-            const unsigned pgrid = 2u * (unsigned)(ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max);
-            rc = launch_k_pairs(pdl && !overlap && (S->pdl_mask & 2), sh_tc_qk_pair_kernel<6>, dim3(pgrid), dim3(320), PS::TOTAL, st, map_x, S->map_wqk128, g);
-            break;
-          }
-        }
+    if (S->qk_bn == 256) {
+      if (S->persistent && S->qk_pair && qk_pairs_max(S) > 0) {
+        // CTA pairs: 256 x 256 tiles, each CTA loads half of the weight rows
+        const int ptiles = ((d.N + 255) / 256) * ((g.ncols + 255) / 256);
+        const unsigned pgrid = 2u * (unsigned)(ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max);
+        rc = launch_k_pairs(pdl && !overlap, sh_tc_qk_pair_kernel<6>, dim3(pgrid), dim3(320), QkPS::TOTAL, qst, map_x, S->map_wqk128, g);
+      } else if (S->persistent) {
+        // a device that cannot hold such a cluster: single-CTA persistent kernel, 128 x 256 tiles
         const unsigned tiles = (unsigned)(d.nblk * ((g.ncols + 255) / 256));
-        rc = S->persistent ? launch_pgemm<256, 4, PG_QKV, 1>(map_x, S->map_wqk, g, tiles < (unsigned)L->sm_count ? tiles : (unsigned)L->sm_count, st, pdl && !overlap && (S->pdl_mask & 2))
-                           : launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st);
-        break;
+        rc = launch_pgemm<256, 4, PG_QKV, 1>(map_x, S->map_wqk, g, tiles < (unsigned)L->sm_count ? tiles : (unsigned)L->sm_count, qst, pdl && !overlap);
+      } else {
+        rc = launch_gemm<256, 4, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, qst);
       }
-      case 3: rc = launch_gemm<128, 6, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
-      default: rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, st); break;
+    } else {
+      // projection width not a multiple of 256: one CTA per 128 x 128 tile
+      rc = launch_gemm<128, QK_STAGES, GEMM_QKV, 1, 1>(map_x, S->map_wqk, g, grid, qst);
     }
     if (rc) return rc;
     L->launches += 1;
@@ -530,11 +546,12 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       g.lists = (const int*)(ws + L->o.lists); g.lgate = (const float*)(ws + L->o.lgate);
       g.tiles = (const ShTile*)(ws + L->o.tiles); g.ntiles = (const int*)(ws + L->o.ntiles);
       g.b_rows_per_group = d.D; g.out0 = ws + L->o.v; g.status = status;
-      if (use_v32(L, S)) { g.v_f32 = 1; g.out0 = ws + L->o.v32; }
+      g.stamp_id = SH_K_V;
+      g.v_early = (float*)(ws + L->o.vearly); g.v_early_cnt = (int*)(ws + L->o.vearly_cnt);
       // 256-row tiles (two accumulators sharing the weight operand): at most half the 128-row bound plus one per group
       dim3 grid(d.tile_rows_src == 256 ? d.max_tiles / 2 + d.H * d.E : d.max_tiles, 1);
       if (d.tile_rows_src == 256) {
-        if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 2>(map_x, S->map_wv, g, grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count, st, pdl && (S->pdl_mask & 4))
+        if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 2>(map_x, S->map_wv, g, grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count, st, pdl)
                                            : launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
         else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
       } else {
@@ -543,17 +560,6 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
       }
       if (rc) return rc;
       L->launches += 1;
-      if (g.v_f32) {
-        // the fp32 sums, rounded to fp16 once, become V
-        const size_t n4 = (size_t)d.N * HD / 4;
-        unsigned cgrid = (unsigned)((n4 + 255) / 256);
-        const unsigned ccap = L->sm_count > 0 ? 8u * (unsigned)L->sm_count : 1184u;
-        if (cgrid > ccap) cgrid = ccap;
-        if ((rc = launch_k(pdl && (S->pdl_mask & 4), sh_v32_to_f16_kernel, dim3(cgrid), dim3(256), 0, st,
-                           (const float4*)(ws + L->o.v32), (uint2*)(ws + L->o.v), n4)))
-          return rc;
-        L->launches += 1;
-      }
     }
   }
   if (overlap) SH_CUDA_CHECK(cudaStreamWaitEvent(st, S->ev_join, 0));
@@ -565,27 +571,15 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   } else {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
-    if (S->attn_single_tile && d.causal) {
-      const int nq = (d.T + 127) / 128;
-      const unsigned grid = (unsigned)(nq * d.B * d.H);
-      if (d.D == 128) {
-        if ((rc = set_smem(sh_tc_attention_kernel<128>, AttnSmem<128>::TOTAL))) return rc;
-        sh_tc_attention_kernel<128><<<grid, 192, AttnSmem<128>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
-      } else {
-        if ((rc = set_smem(sh_tc_attention_kernel<64>, AttnSmem<64>::TOTAL))) return rc;
-        sh_tc_attention_kernel<64><<<grid, 192, AttnSmem<64>::TOTAL, st>>>(S->map_q, S->map_k, S->map_v, a);
-      }
+    const int nq = (d.T + 255) / 256;
+    const unsigned grid = (unsigned)(nq * d.B * d.H);
+    a.balanced = d.causal && (int)grid <= L->sm_count && S->attn_balanced;
+    if (d.D == 128) {
+      if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc;
+      if ((rc = launch_k(pdl, sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
     } else {
-      const int nq = (d.T + 255) / 256;
-      const unsigned grid = (unsigned)(nq * d.B * d.H);
-      a.balanced = d.causal && (int)grid <= L->sm_count && !getenv("SH_ATTN_ADJACENT");
-      if (d.D == 128) {
-        if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc;
-        if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
-      } else {
-        if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc;
-        if ((rc = launch_k(pdl && (S->pdl_mask & 8), sh_tc_attention2_kernel<64>, dim3(grid), dim3(320), Attn2Smem<64>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
-      }
+      if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc;
+      if ((rc = launch_k(pdl, sh_tc_attention2_kernel<64>, dim3(grid), dim3(320), Attn2Smem<64>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
     }
     L->launches += 1;
   }
@@ -593,35 +587,16 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   // ---- output experts ----------------------------------------------------------------------------
   if (simt & SH_STAGE_O) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_O, x, out, st))) return rc;
-  } else if (!L->dense && S->o_scatter) {
-    // sorted grouped GEMM with a scatter-add epilogue (needs out cleared beforehand)
-    TcGemmArgs g{};
-    g.d = d; g.K = d.D; g.ncols = d.M;
-    g.A = ws + L->o.ahat; g.lda = HD;
-    const size_t side1 = d.sides == 2 ? (size_t)d.H * d.N * d.k : 0;
-    g.lists = (const int*)(ws + L->o.lists) + side1; g.lgate = (const float*)(ws + L->o.lgate) + side1;
-    g.tiles = (const ShTile*)(ws + L->o.tiles) + (d.sides == 2 ? d.max_tiles : 0);
-    g.ntiles = (const int*)(ws + L->o.ntiles) + (d.sides == 2 ? 1 : 0);
-    g.b_rows_per_group = d.M; g.out0 = out; g.status = status;
-    dim3 grid(d.max_tiles, (d.M + 127) / 128);
-    if ((rc = launch_gemm<128, 3, GEMM_O, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
-    L->launches += 1;
   } else if (!L->dense) {
     TcOprojArgs a{};
     a.d = d;
     const size_t side1 = d.sides == 2 ? (size_t)d.N * d.H * d.k : 0;   // shared selection: the one side there is
     a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
     a.out = (float*)out; a.status = status;
-    a.nwork = d.nblk * ((d.M + 255) / 256);
-    if (L->sm_count == 0) {
-      int dev = 0;
-      SH_CUDA_CHECK(cudaGetDevice(&dev));
-      SH_CUDA_CHECK(cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, dev));
-    }
-    // The CTA-pair kernel rounds the gate-scaled token rows to fp16 once more than the single-CTA
-    // kernel; with k >= 4 the k-way fp16 sum of the value stage already uses most of the output
-    // tolerance, so those shapes keep the single-CTA kernel (as does a device that cannot hold a
-    // two-CTA cluster of this size).
+    // Up to three selections per (token, head) the CTA-pair kernel serves (its builder threads keep a
+    // token's selections in registers).  With more, the single-CTA kernel, which reads the
+    // selections from shared memory and multiplies by the gate after the UMMA; a device that cannot
+    // hold a two-CTA cluster of the pair kernel's size uses it too.
     bool pair = S->o_pair && d.k <= 3;
     if (pair) {
       const int psm = d.D == 128 ? OprojPairSmem<128>::TOTAL : OprojPairSmem<64>::TOTAL;
@@ -632,44 +607,71 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
         if (S->o_pairs_max <= 0) S->o_pairs_max = -1;
       }
       if (S->o_pairs_max < 0) pair = false;
-      else {
-        // 256 tokens x 256 features per unit, gates folded into the A operand
-        a.nwork = ((d.N + 255) / 256) * ((d.M + 255) / 256);
-        const unsigned pgrid = 2u * (unsigned)(a.nwork < S->o_pairs_max ? a.nwork : S->o_pairs_max);
-        const __half* ahat = (const __half*)(ws + L->o.ahat);
-        if (d.D == 128) rc = launch_k_pairs(pdl && (S->pdl_mask & 16), sh_tc_oproj_pair_kernel<128>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
-        else rc = launch_k_pairs(pdl && (S->pdl_mask & 16), sh_tc_oproj_pair_kernel<64>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
-        if (rc) return rc;
-        L->launches += 1;
-        sh_mark(L, 5, st);
-        SH_CUDA_CHECK(cudaGetLastError());
-        return SH_OK;
-      }
     }
-    const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
-    int as = 3, smem = 0;
-    for (; as >= 2; --as) {
-      smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.k) : OprojSmem<64>::total(as, d.H, d.k);
-      if (smem <= 227 * 1024) break;
-    }
-    if (as < 2) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
-    a.a_slots = as;
-    if (d.D == 128) {
-      if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc;
-      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<128>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
+    if (pair) {
+      // 256 tokens x 256 features per unit, gates folded into the A operand
+      const int psm = d.D == 128 ? OprojPairSmem<128>::TOTAL : OprojPairSmem<64>::TOTAL;
+      a.nwork = ((d.N + 255) / 256) * ((d.M + 255) / 256);
+      const unsigned pgrid = 2u * (unsigned)(a.nwork < S->o_pairs_max ? a.nwork : S->o_pairs_max);
+      const __half* ahat = (const __half*)(ws + L->o.ahat);
+      if (d.D == 128) rc = launch_k_pairs(pdl, sh_tc_oproj_pair_kernel<128>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
+      else rc = launch_k_pairs(pdl, sh_tc_oproj_pair_kernel<64>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
+      if (rc) return rc;
     } else {
-      if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc;
-      if ((rc = launch_k(pdl && (S->pdl_mask & 16), sh_tc_oproj_kernel<64>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
+      a.nwork = d.nblk * ((d.M + 255) / 256);
+      const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
+      int as = 3, smem = 0;
+      for (; as >= 2; --as) {
+        smem = d.D == 128 ? OprojSmem<128>::total(as, d.H, d.k) : OprojSmem<64>::total(as, d.H, d.k);
+        if (smem <= 227 * 1024) break;
+      }
+      if (as < 2) { sh_set_error("output projection: n_heads*k = %d does not fit in shared memory", d.H * d.k); return SH_ERR_UNSUPPORTED; }
+      a.a_slots = as;
+      if (d.D == 128) {
+        if ((rc = set_smem(sh_tc_oproj_kernel<128>, smem))) return rc;
+        if ((rc = launch_k(pdl, sh_tc_oproj_kernel<128>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
+      } else {
+        if ((rc = set_smem(sh_tc_oproj_kernel<64>, smem))) return rc;
+        if ((rc = launch_k(pdl, sh_tc_oproj_kernel<64>, dim3(grid), dim3(320), smem, st, S->map_ahat, S->map_wo256, a))) return rc;
+      }
     }
     L->launches += 1;
   } else {
+    // dense comparator: out = Ahat W_O, one CTA per 128 x 128 tile
     TcGemmArgs g{};
     g.d = d; g.K = HD; g.ncols = d.M; g.nrows = d.N; g.out0 = out; g.status = status;
+    g.stamp_id = SH_K_O;
     dim3 grid(d.nblk, (d.M + 127) / 128);
     if ((rc = launch_gemm<128, 4, GEMM_PLAIN, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
     L->launches += 1;
   }
   sh_mark(L, 5, st);
+  SH_CUDA_CHECK(cudaGetLastError());
+  return SH_OK;
+}
+
+// ---- self-tests of the safety net (no memory access can go wrong in either) ---------------------------
+// which = 0: one thread waits on an mbarrier nobody arrives on, with the given limit, through the
+// same bounded wait every kernel uses; it gives up, records SH_ERR_TIMEOUT and where, and returns.
+// which = 1 (debug library): one thread runs the index check on `arg` against the limit 10.
+static __global__ void sh_selftest_kernel(int* status, int which, unsigned long long arg) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); fence_barrier_init(); }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  if (which == 0) {
+    bool dead = false;
+    mbar_wait_limit(&bar, 0, status, dead, arg);
+  } else {
+    (void)SH_INDEX_OK((long long)arg, 10, status, SH_SITE_SELFTEST);
+  }
+}
+
+int sh_tc_selftest(sh_layer* L, int which, unsigned long long arg, cudaStream_t st) {
+#ifndef SH_DEBUG
+  if (which == 1) { sh_set_error("index checks exist only in the debug library (built with -DSH_DEBUG)"); return SH_ERR_UNSUPPORTED; }
+#endif
+  sh_selftest_kernel<<<1, 32, 0, st>>>((int*)(L->ws + L->o.status), which, arg);
   SH_CUDA_CHECK(cudaGetLastError());
   return SH_OK;
 }

@@ -18,9 +18,16 @@
 // TMEM columns: S0 / P0 at 0, S1 / P1 at 128, O0 at 256, O1 at 384.  Running maximum and
 // rescale: raise only by more than 8 in log2 units; O rescaled in TMEM when that happens.
 #pragma once
-#include "sh_tc_attn.cuh"
+#include "sh_tc_prims.cuh"
 
 namespace shtc {
+
+struct TcAttnArgs {
+  ShDims d;
+  __half* ahat;          // [B*T, H, D]
+  int* status;
+  int balanced;          // pair query tile p with tile ntile-1-p (causal mask, grid fits the GPU in one wave)
+};
 
 template <int D>
 struct Attn2Smem {
@@ -93,7 +100,9 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();                                         // programmatic dependent launch: the next kernel may become resident,
+  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_ATTN);
   pdl_wait();                                            // and this one starts consuming once the kernel before it has completed
+  if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_ATTN);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -265,6 +274,7 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_ATTN);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);

@@ -29,8 +29,7 @@ struct TcGateArgs {
   const float* gbias;        // [G]
   int* idx; float* gate;     // [2, N, H, k]
   int* blockcnt;             // [nblk, G] per-CTA selection histogram
-  void* zero_v;              // [B, H, T, D] fp16 (or fp32: zero_v_f32) or nullptr
-  int zero_v_f32;
+  void* zero_v;              // [B, H, T, D] fp16, or nullptr
   float* zero_out;           // [N, M] or nullptr
   int* status;
   // fused sort (cooperative launch only)
@@ -85,6 +84,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
   pdl_trigger();                                        // the sort kernel may become resident (it waits for this grid)
+  if (threadIdx.x == 0) { sh_stamp_resident(d.stamps, SH_K_GATE); sh_stamp_start(d.stamps, SH_K_GATE); }
 
   if (warp == 0 || warp == 6) {
     // (the boxes of consecutive stages arrive ~290 ns apart however many lanes issue them: with x
@@ -130,7 +130,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       for (long i = et; i < total; i += NSEL) base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (g.zero_v) {
-      const int row_bytes = d.D * (g.zero_v_f32 ? 4 : 2);  // one (token, head) row
+      const int row_bytes = d.D * 2;                       // one (token, head) row
       const int cpr = row_bytes / 16;                      // 16-byte chunks per row (a power of two: 8..32)
       const int ch = et & (cpr - 1);
       for (int tl = et / cpr; tl < nrows; tl += NSEL / cpr) {
@@ -252,6 +252,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   // ---- publish this CTA's selection histogram (the sort kernel scans them) ------------------
   if (!g.fused)
     for (int i = threadIdx.x; i < d.G; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_GATE);
 }
 
 }  // namespace shtc

@@ -1,6 +1,7 @@
-// tcgen05 GEMM kernels of the bf16 configuration: the dense Q/K projection, the grouped
-// value-expert projection and the grouped output-expert projection with its gate-weighted
-// scatter-add epilogue.  One (MT*128) x BN output tile per CTA (MT = 1 or 2 row tiles that
+// One-CTA-per-tile tcgen05 GEMM of the bf16 configuration, for the shapes the persistent kernels do
+// not take: the dense Q/K projection when 2*H*D is not a multiple of 256, the grouped value-expert
+// projection on small workloads (128-row tiles) or with d_head 64, and the dense comparator's
+// projections.  One (MT*128) x BN output tile per CTA (MT = 1 or 2 row tiles that
 // share the B operand, halving its L2 traffic), accumulators in TMEM, operands
 // staged in 128-byte-swizzled shared memory: B always by TMA, A by TMA (dense rows) or by
 // cp.async row gathers (rows addressed through a per-expert token list).
@@ -12,7 +13,7 @@
 
 namespace shtc {
 
-enum { GEMM_QKV = 0, GEMM_V = 1, GEMM_O = 2, GEMM_PLAIN = 3 };
+enum { GEMM_QKV = 0, GEMM_V = 1, GEMM_PLAIN = 3 };
 
 struct TcGemmArgs {
   ShDims d;
@@ -32,8 +33,10 @@ struct TcGemmArgs {
   const float2* rope;    // dense Q/K mode: (cos, sin) table [D/2, T] of the rotary embedding, or nullptr
   int* status;
   int* sched;            // persistent dense mode: {next tile, CTAs that made their final claim}, both 0 between launches
-  int v_f32;             // value experts: out0 is an fp32 accumulation buffer (fp32 vector reductions)
+  float* v_early;        // value experts: fp32 sums [B, H, SH_EARLY_ROWS, D] of the first rows of every sequence, or nullptr
+  int* v_early_cnt;      // ... and their arrival counters [B, H, SH_EARLY_ROWS]
   int claimers;          // claiming CTAs (or CTA pairs) over all grids that share sched; 0: this grid's own
+  int stamp_id;          // SH_K_* slot of this launch in the stamp block (sh_forward_stamped)
 };
 
 // Rotary embedding of the 16 adjacent feature pairs held in v[0..31] (fp32 bit patterns): pair i of
@@ -46,6 +49,41 @@ __device__ __forceinline__ void rope_pairs16(uint32_t* v, const float2* cs, int 
     v[2 * i] = __float_as_uint(a0 * c.x - a1 * c.y);
     v[2 * i + 1] = __float_as_uint(a0 * c.y + a1 * c.x);
   }
+}
+
+// Early-row value sums (see SH_EARLY_ROWS).  A thread that has added its gate-weighted contribution
+// to the fp32 row `sum` (vector reductions) calls this: the arrival that completes the row's k
+// contributions reads the sum back from L2, rounds it to fp16 once into the V row, and clears the
+// sum and the counter for the next pass.  (Reductions, fence, counter: the pattern of a last-block
+// reduction; the loads bypass L1.)
+__device__ __noinline__ void v_early_finish(float* sum, int* cnt, __half* vrow, int D, int k) {
+  __threadfence();
+  if (atomicAdd(cnt, 1) != k - 1) return;
+  __threadfence();
+  for (int i0 = 0; i0 < D; i0 += 32) {                   // eight 16-byte loads in flight per trip to L2
+    float4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = __ldcg(reinterpret_cast<const float4*>(sum + i0) + j);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const __half2 a = __floats2half2_rn(v[j].x, v[j].y), b = __floats2half2_rn(v[j].z, v[j].w);
+      *reinterpret_cast<uint2*>(vrow + i0 + 4 * j) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+      __stcg(reinterpret_cast<float4*>(sum + i0) + j, make_float4(0.f, 0.f, 0.f, 0.f));
+    }
+  }
+  *cnt = 0;
+}
+
+// A row tile of the table the sort wrote, as the grouped kernels use it.  The debug library checks
+// its fields first (head, expert, rows inside the side's lists) and turns a bad entry into an empty tile.
+__device__ __forceinline__ ShTile tile_checked(ShTile tl, const ShDims& d, int* status) {
+#ifdef SH_DEBUG
+  const bool ok = SH_INDEX_OK(tl.h, d.H, status, SH_SITE_V_TILE) && SH_INDEX_OK(tl.e, d.E, status, SH_SITE_V_TILE) &&
+                  SH_INDEX_OK(tl.nrows, 257, status, SH_SITE_V_TILE) &&
+                  SH_INDEX_OK((long long)tl.row0 + tl.nrows, (long long)d.N * d.k + 1, status, SH_SITE_V_TILE);
+  if (!ok) { tl.h = 0; tl.e = 0; tl.row0 = 0; tl.nrows = 0; }
+#endif
+  return tl;
 }
 
 constexpr int GEMM_BM = 128;
@@ -66,7 +104,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
   using SM = GemmSmem<BN, STAGES, MT>;
   static_assert(MT * BN <= 512, "accumulators must fit the 512 TMEM columns");
   constexpr int ROWS = MT * GEMM_BM;
-  constexpr bool GATHER = (MODE == GEMM_V || MODE == GEMM_O);
+  constexpr bool GATHER = MODE == GEMM_V;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -80,7 +118,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
   int th = 0, te = 0, row0, nrows;
   if (GATHER) {
     if ((int)blockIdx.x >= *g.ntiles) return;          // whole CTA leaves before any barrier
-    const ShTile tl = g.tiles[blockIdx.x];
+    const ShTile tl = tile_checked(g.tiles[blockIdx.x], d, g.status);
     th = tl.h; te = tl.e; row0 = tl.row0; nrows = tl.nrows;
   } else {
     row0 = blockIdx.x * ROWS;
@@ -108,6 +146,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
+  if (threadIdx.x == 0) { sh_stamp_resident(d.stamps, g.stamp_id); sh_stamp_start(d.stamps, g.stamp_id); }
 
   if (warp == 0) {
     if (lane == 0) {
@@ -154,15 +193,15 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
       const int c = et & 7, rb = et >> 3;
       const char* src[8 * MT];
       uint32_t ok[8 * MT];
-      const int abytes = A_BF16 ? 2 : 2;
-      const long acol = (MODE == GEMM_O) ? (long)th * d.D : 0;
+      constexpr int abytes = 2;
 #pragma unroll
       for (int i = 0; i < 8 * MT; ++i) {
         const int r = rb + 16 * i;
         int tok = 0;
         ok[i] = 0;
         if (r < nrows) { tok = g.lists[(size_t)th * d.N * d.k + row0 + r]; ok[i] = 16; }
-        src[i] = (const char*)g.A + ((long)tok * g.lda + acol + c * 8) * abytes;
+        if (!SH_INDEX_OK(tok, d.N, g.status, SH_SITE_V_LIST)) { tok = 0; ok[i] = 0; }
+        src[i] = (const char*)g.A + ((long)tok * g.lda + c * 8) * abytes;
       }
       const uint32_t dsw = (uint32_t)((c ^ (rb & 7)) << 4);
       int arrived = 0;
@@ -193,7 +232,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
 #pragma unroll 1
     for (int mt = 0; mt < MT; ++mt) {
     const int r = mt * GEMM_BM + q * 32 + lane;
-    const bool live = r < nrows;
+    bool live = r < nrows;
     int tok = 0;
     float gate = 0.f;
     if (live) {
@@ -201,13 +240,16 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         const size_t li = (size_t)th * d.N * d.k + row0 + r;
         tok = g.lists[li];
         gate = g.lgate[li];
+        if (!SH_INDEX_OK(tok, d.N, g.status, SH_SITE_V_TOKEN)) tok = -1;
       } else {
         tok = row0 + r;
       }
     }
+    if (tok < 0) { live = false; tok = 0; }
     if (tm_ok) {
       const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + mt * BN;
       const int bb = tok / d.T, tt = tok % d.T;
+      const bool early = MODE == GEMM_V && live && g.v_early && tt < d.early_rows;
 #pragma unroll 1
       for (int c00 = 0; c00 < BN; c00 += 64) {
         // two TMEM loads in flight per wait: the load latency, not its bandwidth, bounds this loop
@@ -245,8 +287,8 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
             __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * gate, __uint_as_float(v[2 * i + 1]) * gate);
             p[i] = *reinterpret_cast<uint32_t*>(&hv);
           }
-          if (g.v_f32) {
-            float* d32 = (float*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D + n0;
+          if (early) {
+            float* d32 = g.v_early + (((size_t)bb * d.H + th) * SH_EARLY_ROWS + tt) * d.D + n0;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
               red_add_v4_f32(d32 + 4 * i, __uint_as_float(v[4 * i]) * gate, __uint_as_float(v[4 * i + 1]) * gate,
@@ -255,12 +297,6 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
 #pragma unroll
           for (int i = 0; i < 4; ++i) red_add_v4_f16x2(dst + 8 * i, p[4 * i], p[4 * i + 1], p[4 * i + 2], p[4 * i + 3]);
           }
-        } else if (MODE == GEMM_O) {
-          float* dst = (float*)g.out0 + (size_t)tok * d.M + n0;
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            red_add_v4_f32(dst + 4 * i, __uint_as_float(v[4 * i]) * gate, __uint_as_float(v[4 * i + 1]) * gate,
-                           __uint_as_float(v[4 * i + 2]) * gate, __uint_as_float(v[4 * i + 3]) * gate);
         } else {
           float* dst = (float*)g.out0 + (size_t)tok * g.ncols + n0;
 #pragma unroll
@@ -271,11 +307,15 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
         }
         }
       }
+      if (early)
+        v_early_finish(g.v_early + (((size_t)bb * d.H + th) * SH_EARLY_ROWS + tt) * d.D, g.v_early_cnt + ((size_t)bb * d.H + th) * SH_EARLY_ROWS + tt,
+                       (__half*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D, d.D, d.k);
     }
     }
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, g.stamp_id);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_d, MT * BN);

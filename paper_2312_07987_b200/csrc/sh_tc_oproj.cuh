@@ -97,7 +97,9 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();                                         // programmatic dependent launch: the next kernel may become resident,
+  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_O);
   pdl_wait();                                            // and this one starts consuming once the kernel before it has completed
+  if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_O);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -245,6 +247,7 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_O);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);

@@ -37,7 +37,7 @@
 
 namespace shtc {
 
-constexpr int OPAIR_KMAX = 4;                            // selections per (token, head) a builder keeps in registers
+constexpr int OPAIR_KMAX = 3;                            // selections per (token, head) a builder keeps in registers (the kernel serves k <= 3)
 
 template <int D>
 struct OprojPairSmem {
@@ -116,7 +116,9 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
+  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_O);
   pdl_wait();
+  if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_O);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -209,6 +211,7 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
         const bool lj = live && j < d.k;
         ni[j] = lj ? __ldg(g.idx + so + j) : -1;
         ng[j] = lj ? __ldg(g.gate + so + j) : 0.f;
+        if (lj && !SH_INDEX_OK(ni[j], d.E, g.status, SH_SITE_O_EXPERT)) ni[j] = -1;
       }
       if (++fh == d.H) { fh = 0; fw += npairs; }
     };
@@ -234,7 +237,12 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
 #pragma unroll
           for (int j = 0; j < OPAIR_KMAX; ++j)
             if (ci[j] == e) gv = cg[j];
-          const __half2 g2 = __float2half2_rn(gv);
+          // The gate as the sum of two fp16 values: multiplying by fp16(gate) alone would put one relative
+          // error of up to 2^-11 on this expert's WHOLE contribution to the token (the same factor on
+          // every feature).  p = a * g_hi rounded; e = the exact rounding error of that product (one
+          // fused multiply-add); the result rounds p + (a * g_lo + e): the product a * gate, rounded once.
+          const __half gh1 = __float2half_rn(gv);
+          const __half2 g_hi = __half2half2(gh1), g_lo = __float2half2_rn(gv - __half2float(gh1));
           // one lane polls for the warp (256 threads polling one barrier word get in each other's way)
           if (lane == 0 && !mbar_wait(&p_empty[ps], ppar, g.status, dead)) ok = false;
           ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -245,7 +253,11 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
             uint4 v = cur[i];
             __half2* hv = reinterpret_cast<__half2*>(&v);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) hv[q] = __hmul2(hv[q], g2);
+            for (int q = 0; q < 4; ++q) {
+              const __half2 pq = __hmul2(hv[q], g_hi);
+              const __half2 eq = __hfma2(hv[q], g_hi, __hneg2(pq));
+              hv[q] = __hadd2(pq, __hfma2(hv[q], g_lo, eq));
+            }
             *reinterpret_cast<uint4*>(tile + toff[i]) = v;
           }
           fence_proxy_async_smem();                        // generic-proxy writes -> visible to the UMMA's reads
@@ -283,6 +295,7 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_O);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc_pair(tmem, 512);

@@ -79,7 +79,9 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
   // completed (plain loads do), so the layer launches this projection the ordinary way on a
   // second stream instead when it wants it to run beside the gate and sort kernels.
   pdl_trigger();
+  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, g.stamp_id);
   if (GATHER) pdl_wait();
+  if (threadIdx.x == 0) sh_stamp_start(d.stamps, g.stamp_id);
   const int ntiles = GATHER ? *g.ntiles : ((g.nrows + ROWS - 1) / ROWS) * ncol;
   // the qi-th tile of this CTA for every role but the claiming producer, or -1 when there is none
   auto next_tile = [&](int qi) -> int {
@@ -121,7 +123,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         if (t < 0) break;
         int row0, brow;
         if (GATHER) {
-          const ShTile tl = g.tiles[t];
+          const ShTile tl = tile_checked(g.tiles[t], d, g.status);
           row0 = 0;
           brow = (tl.h * d.E + tl.e) * g.b_rows_per_group;
         } else {
@@ -185,7 +187,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
       for (int qi = 0; !dead; ++qi) {
         const int t = next_tile(qi);
         if (t < 0) break;
-        const ShTile tl = g.tiles[t];
+        const ShTile tl = tile_checked(g.tiles[t], d, g.status);
         const char* src[8 * MT];
         uint32_t ok[8 * MT];
 #pragma unroll
@@ -194,6 +196,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
           int tok = 0;
           ok[i] = 0;
           if (r < tl.nrows) { tok = g.lists[(size_t)tl.h * d.N * d.k + tl.row0 + r]; ok[i] = 16; }
+          if (!SH_INDEX_OK(tok, d.N, g.status, SH_SITE_V_LIST)) { tok = 0; ok[i] = 0; }
           src[i] = (const char*)g.A + ((long)tok * g.lda + c * 8) * 2;
         }
         for (int kb = 0; kb < KB; ++kb) {
@@ -233,7 +236,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
       const int b = it & 1;
       int th = 0, row0, nrows, col0 = 0;
       if (GATHER) {
-        const ShTile tl = g.tiles[t];
+        const ShTile tl = tile_checked(g.tiles[t], d, g.status);
         th = tl.h; row0 = tl.row0; nrows = tl.nrows;
       } else {
         row0 = (t / ncol) * ROWS;
@@ -251,6 +254,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             const size_t li = (size_t)th * d.N * d.k + row0 + r;
             tok[mt] = g.lists[li];
             gate[mt] = g.lgate[li];
+            if (!SH_INDEX_OK(tok[mt], d.N, g.status, SH_SITE_V_TOKEN)) tok[mt] = -1;
           } else {
             tok[mt] = row0 + r;
           }
@@ -263,6 +267,7 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         const uint32_t trow = tmem + lane_off + b * ACC_COLS + mt * BN;
         const bool live = tok[mt] >= 0;
         const int bb = live ? tok[mt] / d.T : 0, tt = live ? tok[mt] % d.T : 0;
+        const bool early = MODE == PG_V && live && g.v_early && tt < d.early_rows;
 #pragma unroll 1
         for (int c00 = 0; c00 < BN; c00 += 64) {
           uint32_t vv[64];
@@ -303,8 +308,8 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                 __half2 hv = __floats2half2_rn(__uint_as_float(v[2 * i]) * gt, __uint_as_float(v[2 * i + 1]) * gt);
                 p[i] = *reinterpret_cast<uint32_t*>(&hv);
               }
-              if (g.v_f32) {
-                float* d32 = (float*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D + n0;
+              if (early) {
+                float* d32 = g.v_early + (((size_t)bb * d.H + th) * SH_EARLY_ROWS + tt) * d.D + n0;
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                   red_add_v4_f32(d32 + 4 * i, __uint_as_float(v[4 * i]) * gt, __uint_as_float(v[4 * i + 1]) * gt,
@@ -316,12 +321,16 @@ sh_tc_pgemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             }
           }
         }
+        if (early)
+          v_early_finish(g.v_early + (((size_t)bb * d.H + th) * SH_EARLY_ROWS + tt) * d.D, g.v_early_cnt + ((size_t)bb * d.H + th) * SH_EARLY_ROWS + tt,
+                         (__half*)g.out0 + (((size_t)bb * d.H + th) * d.T + tt) * d.D, d.D, d.k);
       }
     }
   }
   if (!GATHER) pdl_wait();
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, g.stamp_id);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);

@@ -45,8 +45,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  `dead` is the calling thread's give-up flag: once set, later waits return
-// at once so that the role falls through to the teardown.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, bool& dead) {
+// at once so that the role falls through to the teardown.  The first give-up of a launch records
+// where it happened in the status block (SH_ST_DIAG words).
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, int* status, bool& dead, uint64_t limit_ns) {
   if (dead) return false;
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
@@ -54,16 +55,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
-      if (global_timer_ns() - t0 > SH_WAIT_LIMIT_NS || *(volatile int*)status != 0) {
-        if (atomicCAS(status, 0, SH_ERR_TIMEOUT) == 0) {   // first give-up of the launch: say where (diagnostics)
-          status[1] = (int)blockIdx.x; status[2] = (int)threadIdx.x; status[3] = (int)smem_u32(bar);
-          status[4] = (int)parity; status[5] = (int)gridDim.x; status[6] = (int)blockDim.x;
+      if (global_timer_ns() - t0 > limit_ns || *(volatile int*)status != 0) {
+        if (atomicCAS(status, 0, SH_ERR_TIMEOUT) == 0) {
+          status[SH_ST_DIAG] = (int)blockIdx.x; status[SH_ST_DIAG + 1] = (int)threadIdx.x; status[SH_ST_DIAG + 2] = (int)smem_u32(bar);
+          status[SH_ST_DIAG + 3] = (int)parity; status[SH_ST_DIAG + 4] = (int)gridDim.x; status[SH_ST_DIAG + 5] = (int)blockDim.x;
         }
         dead = true;
         return false;
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, bool& dead) {
+  return mbar_wait_limit(bar, parity, status, dead, SH_WAIT_LIMIT_NS);
 }
 
 // ---- proxy fences / cp.async ---------------------------------------------------------------
@@ -301,6 +305,26 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// registers -> TMEM, the mirror image of tmem_ld32
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t elect_one() {
   uint32_t pred;

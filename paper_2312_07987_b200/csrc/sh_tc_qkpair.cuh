@@ -76,6 +76,7 @@ sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
+  if (threadIdx.x == 0) { sh_stamp_resident(d.stamps, g.stamp_id); sh_stamp_start(d.stamps, g.stamp_id); }
   // the qi-th tile of this pair, for every role but the claimer, or -1 when there is none
   auto next_tile = [&](int qi) -> int {
     const int j = qi & (TQ - 1);
@@ -206,6 +207,7 @@ sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();
+  if (threadIdx.x == 0) sh_stamp_end(d.stamps, g.stamp_id);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc_pair(tmem, 512);

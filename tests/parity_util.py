@@ -18,6 +18,21 @@ def oracle_for(inp, batches=None, rope_base=None, shared_selection=False, causal
                               shared_selection=shared_selection)
 
 
+def oracle_selection(inp, shared_selection=False):
+    """Selections, gates, offsets and token lists of ALL tokens of inp.x from the oracle's gate and
+    bucket-sort steps alone (no attention: cheap at any size); same keys as the full oracle's stages."""
+    from oracle.switchhead_oracle import bucket_lists, gate_and_select
+    cfg = inp.cfg
+    x2d = inp.x.reshape(-1, cfg.d_model).astype(np.float64)
+    out = {}
+    for side, W, b in (("S", inp.Ws, inp.bias_s), ("D", inp.Ws if shared_selection else inp.Wd,
+                                                   inp.bias_s if shared_selection else inp.bias_d)):
+        _, _, idx, gate = gate_and_select(x2d, W.astype(np.float64), b, cfg.k)
+        off, lists = bucket_lists(idx, cfg.n_experts)
+        out["idx" + side], out["gate" + side], out["offsets" + side], out["lists" + side] = idx, gate, off, lists
+    return out
+
+
 def rel_rms_err(got, ref):
     ref = np.asarray(ref, dtype=np.float64)
     return float(np.abs(np.asarray(got, dtype=np.float64) - ref).max() / np.sqrt((ref ** 2).mean()))

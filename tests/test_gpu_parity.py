@@ -9,6 +9,14 @@ from tests import parity_util as pu
 
 pytestmark = pytest.mark.gpu
 
+# Two passes over the same input.  k <= 2: bit for bit (a sum of two terms does not depend on their
+# order, and out is summed on chip in a fixed order).  k >= 3: the k gate-weighted contributions to a
+# value row arrive in a different order from run to run - fp32 reductions for the first 32 rows of a
+# sequence (the ones that reach the output unaveraged), fp16 reductions for the rest; measured
+# differences between passes: up to 3.8e-3 of the output RMS (k = 4, 2048-token sequences).  Each pass
+# is within 2e-2 of the oracle.
+RUN_TO_RUN_K3 = 6e-3
+
 
 def full_check(inp, check_stage_buffers=True, batches=None, shared_selection=False):
     cfg = inp.cfg
@@ -26,15 +34,17 @@ def full_check(inp, check_stage_buffers=True, batches=None, shared_selection=Fal
         pu.check_selection(idx, gate, ref, N, gtol)
         pu.check_lists(off, lists, ref)
     else:
-        H, k = cfg.n_heads, cfg.k
-        tok = np.concatenate([np.arange(b * T, (b + 1) * T) for b in batches])
-        pu.check_selection(idx[:, tok], gate[:, tok], ref, tok.size, gtol)
+        # the full oracle is run on the sampled sequences only (attention is what costs); selections,
+        # gates, offsets and token lists are checked for ALL N tokens - the lists pool every sequence
+        pu.check_selection(idx, gate, pu.oracle_selection(inp, shared_selection), N, gtol)
+        pu.check_lists(off, lists, pu.oracle_selection(inp, shared_selection))
     if check_stage_buffers:
         y2 = layer.sh_forward(x)          # refresh the intermediates after sh_gate_topk
         torch.cuda.synchronize()
         pu.check_stages(layer, ref, cfg, batches)
     err = pu.rel_rms_err(yb, ref["y"])
     assert err < pu.TOL_Y[cfg.dtype], f"output max-abs error / rms = {err:.3e}"
+    layer.sh_check_guards()               # no kernel wrote past the end of a workspace sub-buffer
     layer.close()
     return err
 
@@ -65,12 +75,12 @@ def test_c4_262m_bf16_full():
 
 def test_long_ctx_bf16_full_size_sampled_sequences():
     inp = inputs.make_inputs(inputs.CONFIGS["long_ctx_bf16"])
-    full_check(inp, batches=[1])
+    full_check(inp, batches=[0, 3])       # y on the first and the last sequence; selections on all tokens
 
 
 def test_wide_skew_bf16_full_size_sampled_sequences():
     inp = inputs.make_inputs(inputs.CONFIGS["wide_skew_bf16"])
-    full_check(inp, batches=[5])
+    full_check(inp, batches=[0, 7])
 
 
 @pytest.mark.parametrize("T,B,E,k,H,D", [(1, 2, 4, 2, 2, 64), (100, 3, 5, 3, 2, 64), (129, 1, 4, 4, 1, 128),
@@ -100,7 +110,7 @@ def test_causality_on_gpu():
     torch.cuda.synchronize()
     a, b = y0[:, :t0 + 1].cpu().numpy(), y1[:, :t0 + 1].cpu().numpy()
     rms = np.sqrt((a.astype(np.float64) ** 2).mean())
-    assert np.abs(a - b).max() / rms < 1e-2          # only summation-order noise of the fp16 V sums
+    assert np.abs(a - b).max() / rms < RUN_TO_RUN_K3   # k = 3: only the order of the value sums differs
     assert not np.allclose(y0[:, t0 + 1:].cpu().numpy(), y1[:, t0 + 1:].cpu().numpy())
     layer.close()
 
@@ -115,9 +125,7 @@ def test_forward_is_repeatable_and_selection_deterministic():
     for a, b in zip(r0, r1):
         assert torch.equal(a, b)
     rms = y0.double().pow(2).mean().sqrt().item()
-    # (k = 3: the value stage's fp16 sums come in arrival order; both passes are within the tolerance of
-    #  the oracle, their difference has been seen at 1.2e-2 * RMS)
-    assert (y0 - y1).abs().max().item() / rms < 4e-2
+    assert (y0 - y1).abs().max().item() / rms < RUN_TO_RUN_K3          # k = 3: see RUN_TO_RUN_K3
     layer.close()
 
 
@@ -157,13 +165,12 @@ def rope_check(inp, base=10000.0, batches=None):
     layer.sh_set_rope(0.0)                                   # off again: the plain layer
     y_off = layer.sh_forward(x)
     torch.cuda.synchronize()
-    # (k >= 3: not bit for bit, the k-way V sums are atomic / vector reductions in arrival order; two
-    #  passes have been seen 1.2e-2 * RMS apart at k = 3, and a rotation left on would be of order 1)
+    # (k >= 3: not bit for bit, see RUN_TO_RUN_K3; a rotation left on would be of order 1)
     diff = pu.rel_rms_err(y_off.cpu().numpy(), y_plain.cpu().numpy())
     if cfg.dtype == inputs.DTYPE_BF16 and cfg.k <= 2:
         assert torch.equal(y_off, y_plain), diff
     else:
-        assert diff < (1e-5 if cfg.dtype == inputs.DTYPE_F32 else 4e-2), diff
+        assert diff < (1e-5 if cfg.dtype == inputs.DTYPE_F32 else RUN_TO_RUN_K3), diff
     layer.close()
 
 
@@ -258,16 +265,6 @@ def test_padded_d_head_with_rope_and_shared_selection():
     rope_check(inputs.make_inputs(cfg))
 
 
-# ---- launch-structure switches (A/B aids): same numbers with ordinary launches on one stream ----
-@pytest.mark.parametrize("env", [{"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
-                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"}, {"SH_SORT_SEPARATE": "1"}])
-def test_launch_structure_switches_keep_the_result(env, monkeypatch):
-    for k, v in env.items():
-        monkeypatch.setenv(k, v)                           # read when the weights are set / at launch
-    full_check(inputs.make_inputs(inputs.CONFIGS["small_bf16"]))
-    full_check(inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=3), check_stage_buffers=False)
-
-
 def test_pair_output_projection_ragged_tokens_and_features():
     # CTA-pair output projection: N = 300 is not a multiple of the pair's 256 tokens (the second CTA of
     # the last pair owns 44 tokens, and with N = 100 none at all), d_model = 384 or 128 not of its 256 features
@@ -275,12 +272,10 @@ def test_pair_output_projection_ragged_tokens_and_features():
     full_check(inputs.make_inputs(inputs.LayerConfig("pair_half_empty", inputs.DTYPE_BF16, 1, 100, 128, 3, 128, 3, 1, seed=91)))
 
 
-@pytest.mark.parametrize("split", [False, True])
-def test_back_to_back_forward_passes_share_the_tile_counter_cleanly(split, monkeypatch):
-    if not split:
-        monkeypatch.setenv("SH_QK_ONE_GRID", "1")
-    # the CTA pairs of the Q/K projection (two grids, or one with SH_QK_ONE_GRID) claim tiles from one counter
-    # that the last claimer of a pass puts back: many passes in a row, with and without a host synchronisation between them
+def test_back_to_back_forward_passes_share_the_tile_counter_cleanly():
+    # the CTA pairs of the Q/K projection's two grids claim tiles from one counter that the last claimer
+    # of a pass puts back: many passes in a row, with and without a host synchronisation between them
+    # (the one-grid form is driven through the debug library, tests/test_gpu_debug_library.py)
     inp = inputs.make_inputs(inputs.CONFIGS["c4_262m_bf16"], batch=5)
     layer = binding.layer_from_inputs(inp)
     x = binding.to_device(inp.x, inp.cfg.dtype)
