@@ -3,18 +3,24 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
 
-Prints ONE JSON line.  `value` = tokens/s with x already resident in HBM (L2 flushed
-between timed steps); `e2e` = the same metric with x in pinned host memory and the result
-copied back inside the timed region; `roofline` = the dominant stage against the measured
-bf16 tensor peak (MEASURED_PEAKS.json); `cpu_baseline` = the fp64 oracle on the host cores.
-With N > 1 (torchrun) every rank runs the same workload on its own batch (independent
-sequences, no collective on the data path) and the slowest rank sets the time.
+Prints ONE JSON line.  `value` = tokens/s with x already resident in HBM, L2 flushed before
+every timed step; `e2e` = the same metric with x in pinned host memory and the result copied
+back inside the timed region; `roofline` = the kernel with the longest span INSIDE the real
+pass (device-clock stamps of sh_forward_stamped: same launches as sh_forward) against the
+measured bf16 tensor peak (MEASURED_PEAKS.json); `per_config` = the same figures for every
+bf16 workload; `cpu_baseline` = the fp64 oracle on the host cores.
+
+With --gpus N > 1 and no torchrun environment the script starts its own N ranks (torch.distributed.run,
+rendezvous on 127.0.0.1).  Every rank runs the same workload on its own batch (independent
+sequences, no collective on the data path); a barrier brackets the timed region and the slowest
+rank sets the time.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -26,11 +32,17 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 DEFAULT_CONFIG = "c4_262m_bf16"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's main kernel, from the ncu
-# capture summarised in profiles/c4_262m_bf16_forward_kernels.md (MB, workload c4_262m_bf16)
-DRAM_TRAFFIC_MB = {"c4_262m_bf16": {"gate_topk_sort": 16.92, "qk_proj": 18.91, "v_experts": 29.92,
-                                    "attention": 25.22, "o_experts": 13.23}}
+BF16_CONFIGS = ["small_bf16", "c4_262m_bf16", "long_ctx_bf16", "wide_skew_bf16"]
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel (MB), from the one-kernel ncu
+# captures summarised under profiles/ (the file named beside each workload)
+DRAM_TRAFFIC_MB = {
+    "c4_262m_bf16": {"gate": 16.92, "qk": 18.91, "v": 29.92, "attn": 25.22, "o": 13.23},   # profiles/c4_262m_bf16_forward_kernels.md
+}
+KERNEL_STAGE = {"gate": "gate_topk_sort", "sort": "gate_topk_sort", "qk_a": "qk_proj", "qk_b": "qk_proj", "v": "v_experts",
+                "attn": "attention", "o": "o_experts"}
 STAGES = ["gate_topk_sort", "qk_proj", "v_experts", "attention", "o_experts"]
+METRIC = "switchhead_layer_fwd_tokens_per_s"
+MIN_TIMED_SECONDS = 0.5        # the timed region is repeated until it has run this long (clock samples need load to see)
 
 
 def load_peaks():
@@ -42,6 +54,16 @@ def load_peaks():
     return dict(tflops=1590.0, tflops_sustained=1400.0, hbm_gbs=6650.0, source="fallback")
 
 
+def config_dict(cfg, world, args):
+    """The workload description both arms print (identical keys and values)."""
+    return {"workload": cfg.name, "batch_per_gpu": cfg.batch, "seq_len": cfg.seq, "d_model": cfg.d_model,
+            "n_heads": cfg.n_heads, "d_head": cfg.d_head, "n_experts": cfg.n_experts, "k": cfg.k,
+            "causal": True, "rope_base": args.rope if args.rope > 0 else None,
+            "shared_selection": bool(args.shared_selection),
+            "l2": "flushed before every timed step (256 MiB write)",
+            "parallelism": f"batch-sharded replicas x{world}, no collective"}
+
+
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -51,7 +73,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
-                                       "--format=csv,noheader,nounits", "-lms", "20"],
+                                       "--format=csv,noheader,nounits", "-lms", "5"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -70,19 +92,22 @@ class ClockSampler:
         rows = [l.strip().split(", ") for l in self.f if l.strip()]
         self.f.close()
         os.unlink(self.f.name)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
             except Exception:
                 continue
             for n, v in zip(names, r[3:7]):
                 if v.strip().lower().startswith("active"):
                     reasons.add(n)
         if sm:
-            hot = sorted(sm)[len(sm) // 2:]            # upper half = samples under load
-            out.update(sm_mhz=float(np.median(hot)), sm_max_mhz=float(max(mx)), samples=len(sm))
+            # samples under load: those drawing more than the midpoint between idle and peak power
+            thr = 0.5 * (min(pw) + max(pw))
+            hot = [s for s, p in zip(sm, pw) if p >= thr] or sm
+            out.update(sm_mhz=float(np.median(hot)), sm_max_mhz=float(max(mx)), samples=len(sm), samples_under_load=len(hot),
+                       power_w_max=float(max(pw)))
         out["reasons"] = sorted(reasons)
         return out
 
@@ -137,31 +162,179 @@ def run_reference(args, rank, world):
     cores = len(os.sched_getaffinity(0))
     sample = f"{sample_b} of {cfg.batch} sequences of {cfg.seq} tokens per step"
     print(json.dumps({
-        "impl": "reference", "metric": "switchhead_layer_fwd_tokens_per_s", "value": value, "unit": "tokens/s",
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": cfg.batch, "seq_len": cfg.seq, "d_model": cfg.d_model,
-                   "n_heads": cfg.n_heads, "d_head": cfg.d_head, "n_experts": cfg.n_experts, "k": cfg.k},
+        "config": config_dict(cfg, world, args),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-    }))
+    }), flush=True)
+
+
+def launch_ranks(n: int) -> int:
+    """--gpus N without a torchrun environment: start N ranks of this script on this node."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def timed_region(layer, x, out, flush, stream, steps, barrier, min_seconds):
+    """Runs the K-step timed region (flush, event, sh_forward, event) again and again until it has been
+    running for min_seconds; returns the per-repeat mean milliseconds per step."""
+    import torch
+    means = []
+    t_begin = time.perf_counter()
+    while True:
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for a, b in ev:
+            flush.fill_(1)
+            a.record(stream)
+            layer.sh_forward(x, out)
+            b.record(stream)
+        barrier()
+        means.append(float(np.mean([a.elapsed_time(b) for a, b in ev])))
+        if time.perf_counter() - t_begin >= min_seconds or len(means) >= 400:
+            return means
+
+
+def kernel_timeline(layer, x, out, flush, reps=12):
+    """Mean per-kernel spans inside the real pass, microseconds from the pass's first stamp:
+    {kernel: (start, end)} (start = first CTA past its dependency wait, end = last CTA done)."""
+    import torch
+    acc = {}
+    for _ in range(reps):
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        st = layer.sh_forward_stamped(x, out)
+        t0 = min(v[0] for v in st.values())
+        for k, (res, start, end) in st.items():
+            a = acc.setdefault(k, [0.0, 0.0, 0])
+            a[0] += (start - t0) * 1e-3; a[1] += (end - t0) * 1e-3; a[2] += 1
+    return {k: (a[0] / a[2], a[1] / a[2]) for k, a in acc.items()}
+
+
+def roofline_from_timeline(cfg, tl, fl, peaks):
+    """The kernel with the longest span inside the pass, against the bound that applies to it."""
+    N = cfg.n_tokens
+    span = {k: e - s for k, (s, e) in tl.items()}
+    if "qk_a" in span and "qk_b" in span:           # two grids of one projection: one span
+        s0 = min(tl["qk_a"][0], tl["qk_b"][0]); e0 = max(tl["qk_a"][1], tl["qk_b"][1])
+        span["qk_a"] = e0 - s0
+        del span["qk_b"]
+    dom = max(span, key=span.get)
+    us = span[dom]
+    flop = {"qk_a": fl["qk"], "v": fl["v"], "attn": fl["attn_half"], "o": fl["o"]}
+    traffic = DRAM_TRAFFIC_MB.get(cfg.name, {}).get(dom.replace("_a", ""))
+    if dom in ("gate", "sort"):
+        bytes_ = N * cfg.d_model * 2 + 4 * (2 * N * cfg.n_heads * cfg.k) * 4        # x read once + idx/gate/lists written
+        ach = bytes_ / (us * 1e-6) / 1e9
+        roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"])
+    else:
+        ach = flop[dom] / (us * 1e-6) / 1e12
+        roof = dict(bound="tensor", achieved=ach, peak=peaks["tflops"], unit="TFLOP/s", frac=ach / peaks["tflops"])
+    roof.update(kernel=KERNEL_STAGE[dom], ms=us * 1e-3, peak_source=peaks["source"],
+                timing="span of the kernel inside the real pass (device-clock stamps, first CTA past its dependency wait to last CTA done)",
+                traffic=None if traffic is None else traffic * 1e6, traffic_unit="bytes per launch (ncu)")
+    if dom == "o":
+        # the on-chip sum multiplies every token tile by all E experts of a head (zero rows for the
+        # tokens that did not select one): executed tensor work = E/k times the useful work counted here
+        roof["executed_over_useful_flop"] = cfg.n_experts / cfg.k
+    return roof
+
+
+def measure_config(cfg, args, rank, world, peaks, flush, barrier, steps, min_seconds, with_e2e):
+    """Everything measured for one workload on this rank; the caller takes the max over ranks."""
+    import torch
+    from paper_2312_07987_b200 import binding, inputs, sharding
+    inp = inputs.make_inputs(cfg)
+    inp.x = sharding.rank_batch(inp.x, rank)                                 # rows keep their gate margins
+    layer = binding.layer_from_inputs(inp, shared_selection=args.shared_selection)
+    if args.rope > 0:
+        layer.sh_set_rope(args.rope)
+    x = binding.to_device(inp.x, cfg.dtype)
+    out = torch.empty(inp.x.shape, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        layer.sh_forward(x, out)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0, "device status word set during warm-up"
+    res = dict(launches=layer.sh_launch_count())
+
+    res["repeat_means"] = timed_region(layer, x, out, flush, stream, steps, barrier, min_seconds)
+
+    # L2-warm variant: K back-to-back calls, one event pair
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(steps):
+        layer.sh_forward(x, out)
+    b.record(stream)
+    torch.cuda.synchronize()
+    res["warm_ms"] = a.elapsed_time(b) / steps
+
+    res["timeline"] = kernel_timeline(layer, x, out, flush)
+    # serialised stage times (ordinary launches, one stream, CUDA events at the stage boundaries): what each
+    # stage costs ALONE; they add up to more than a pass, in which the kernels overlap
+    stage = np.zeros(6)
+    for _ in range(6):
+        flush.fill_(1)
+        stage += np.array(layer.sh_forward_timed(x, out))
+    res["stage_ms_serialised"] = stage / 6
+
+    if with_e2e:
+        # end to end with host buffers: every step copies x in from pinned host memory and the result back
+        # out; the three run as a pipeline on three streams (pipeline.HostFedLayer), as a host-fed caller would
+        from paper_2312_07987_b200 import pipeline
+        xh = [x.cpu().pin_memory() for _ in range(2)]
+        outh = [torch.empty(inp.x.shape, dtype=torch.float32).pin_memory() for _ in range(2)]
+        pipe = pipeline.HostFedLayer(layer, x)
+        for i in range(4):
+            pipe.step(xh[i & 1], outh[i & 1])
+        pipe.wait()
+        ref = out.cpu()
+        assert torch.equal(outh[1], ref) or float((outh[1] - ref).abs().max()) < 1e-2 * float(ref.abs().max()), \
+            "pipelined result differs from the direct one"
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(pipe.s_in)
+        for i in range(steps):
+            pipe.step(xh[i & 1], outh[i & 1])
+        b.record(pipe.s_out)
+        pipe.wait()
+        barrier()
+        res["e2e_ms"] = a.elapsed_time(b)
+        res["h2d"] = int(x.numel() * x.element_size())
+        res["d2h"] = int(out.numel() * 4)
+    assert layer.sh_last_status() == 0, "device status word set during the timed region"
+    res["inp"], res["x"], res["out"] = inp, x, out
+    layer.close()
+    return res
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default=DEFAULT_CONFIG)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the table over the other workloads")
     ap.add_argument("--shared-selection", action="store_true",
                     help="one gate for the source and the destination side (the paper's Shared Selection variant)")
     ap.add_argument("--rope", type=float, default=0.0,
                     help="rotary position embeddings on Q, K with this base (0 = off, the headline configuration)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args.gpus))                 # this process becomes the launcher of N ranks
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -180,17 +353,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     cfg = inputs.CONFIGS[args.config]
     peaks = load_peaks()
-
-    # each rank owns its own batch of independent sequences (same weights, rank-specific x)
-    inp = inputs.make_inputs(cfg)
-    inp.x = sharding.rank_batch(inp.x, rank)                                 # rows keep their gate margins
-    layer = binding.layer_from_inputs(inp, shared_selection=args.shared_selection)
-    if args.rope > 0:
-        layer.sh_set_rope(args.rope)
-    x = binding.to_device(inp.x, cfg.dtype)
-    out = torch.empty(inp.x.shape, dtype=torch.float32, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # > 126 MB L2
-    stream = torch.cuda.current_stream()
 
     def barrier():
         torch.cuda.synchronize()
@@ -198,118 +361,50 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        layer.sh_forward(x, out)
-    torch.cuda.synchronize()
-    assert layer.sh_last_status() == 0, "device status word set during warm-up"
-    launches = layer.sh_launch_count()
-
-    # ---- timed region: K steps, L2 flushed before each, CUDA events on the launching stream ----
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    barrier()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in ev:
-        flush.fill_(1)
-        a.record(stream)
-        layer.sh_forward(x, out)
-        b.record(stream)
-    barrier()
-    times = np.array([a.elapsed_time(b) for a, b in ev])
-    t_total_ms = float(times.sum())
+    m = measure_config(cfg, args, rank, world, peaks, flush, barrier, args.steps, MIN_TIMED_SECONDS, with_e2e=True)
     clocks = sampler.stop() if sampler else None
 
-    # L2-warm variant: K back-to-back calls, one event pair
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    a.record(stream)
-    for _ in range(args.steps):
-        layer.sh_forward(x, out)
-    b.record(stream)
-    torch.cuda.synchronize()
-    warm_ms = a.elapsed_time(b) / args.steps
+    # ---- max over ranks (every repeat mean, so that the median is of the slowest rank's times) ----
+    nrep = int(sharding.max_over_ranks([-float(len(m["repeat_means"]))], device="cuda")[0] * -1)   # fewest repeats any rank made
+    reduced = sharding.max_over_ranks(m["repeat_means"][:nrep] + [m["e2e_ms"], m["warm_ms"]], device="cuda")
+    repeat_means, e2e_ms, warm_ms = reduced[:nrep], reduced[nrep], reduced[nrep + 1]
 
-    # ---- per-stage times (CUDA events at the stage boundaries, L2 flushed) ----
-    stage = np.zeros(6)
-    reps = 10
-    for _ in range(reps):
-        flush.fill_(1)
-        stage += np.array(layer.sh_forward_timed(x, out))
-    stage /= reps
-
-    # ---- end to end with host buffers: every step copies x in from pinned host memory and the
-    # result back out; the three run as a pipeline on three streams (pipeline.HostFedLayer), as a
-    # host-fed caller would run them ----
-    from paper_2312_07987_b200 import pipeline
-    xh = [x.cpu().pin_memory() for _ in range(2)]
-    outh = [torch.empty(inp.x.shape, dtype=torch.float32).pin_memory() for _ in range(2)]
-    pipe = pipeline.HostFedLayer(layer, x)
-    for i in range(4):
-        pipe.step(xh[i & 1], outh[i & 1])
-    pipe.wait()
-    assert torch.equal(outh[1], out.cpu()) or float((outh[1] - out.cpu()).abs().max()) < 1e-2 * float(out.abs().max()), \
-        "pipelined result differs from the direct one"
-    barrier()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(pipe.s_in)
-    for i in range(args.steps):
-        pipe.step(xh[i & 1], outh[i & 1])
-    b.record(pipe.s_out)
-    pipe.wait()
-    barrier()
-    e2e_ms = a.elapsed_time(b)
-    assert layer.sh_last_status() == 0, "device status word set during the timed region"
-
-    # ---- max over ranks ----
-    t_total_ms, e2e_ms, warm_ms = sharding.max_over_ranks([t_total_ms, e2e_ms, warm_ms], device="cuda")
-
+    line = None
     if rank == 0:
         N = cfg.n_tokens
         fl = inputs.useful_flop(cfg)
-        ms_step = t_total_ms / args.steps
+        ms_step = float(np.median(repeat_means))
         value = sharding.aggregate_throughput(N, world, ms_step * 1e-3)
         useful_tflops = world * fl["total"] / (ms_step * 1e-3) / 1e12
-        stage_flop = dict(gate_topk_sort=0.0, qk_proj=fl["qk"], v_experts=fl["v"], attention=fl["attn_half"], o_experts=fl["o"])
-        dom = int(np.argmax(stage[:5]))
-        dom_name = STAGES[dom]
-        if dom_name == "gate_topk_sort":
-            # HBM-bound stage: x read once + idx/gate/lists written
-            bytes_ = N * cfg.d_model * 2 + 4 * (2 * N * cfg.n_heads * cfg.k) * 4
-            ach = bytes_ / (stage[dom] * 1e-3) / 1e9
-            roof = dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"], traffic=None)
-        else:
-            ach = stage_flop[dom_name] / (stage[dom] * 1e-3) / 1e12
-            roof = dict(bound="tensor", achieved=ach, peak=peaks["tflops"], unit="TFLOP/s", frac=ach / peaks["tflops"], traffic=None)
-        traffic = DRAM_TRAFFIC_MB.get(cfg.name, {}).get(dom_name)
-        roof.update(kernel=dom_name, ms=float(stage[dom]), peak_source=peaks["source"],
-                    traffic=None if traffic is None else traffic * 1e6, traffic_unit="bytes per launch (ncu)")
-
+        tl = m["timeline"]
         line = {
-            "metric": "switchhead_layer_fwd_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == inputs.DTYPE_BF16 else "f32",
             "data": "synthetic",
-            "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "seq_len": cfg.seq, "d_model": cfg.d_model,
-                       "n_heads": cfg.n_heads, "d_head": cfg.d_head, "n_experts": cfg.n_experts, "k": cfg.k,
-                       "causal": True, "rope_base": args.rope if args.rope > 0 else None,
-                       "shared_selection": bool(args.shared_selection),
-                       "l2": "flushed before every timed step (256 MiB write)",
-                       "parallelism": f"batch-sharded replicas x{world}, no collective"},
+            "config": config_dict(cfg, world, args),
+            "timed_region": {"repeats": len(repeat_means), "steps_per_repeat": args.steps,
+                             "ms_per_step": "median over the repeats of the mean over a repeat's steps",
+                             "repeat_min_ms": float(min(repeat_means)), "repeat_max_ms": float(max(repeat_means))},
             "useful_tflops": useful_tflops,
             "frac_of_bf16_peak_measured": useful_tflops / (world * peaks["tflops"]),
             "frac_of_bf16_peak_nominal_2250": useful_tflops / (world * 2250.0),
             "ms_per_step_l2_warm": warm_ms,
             "useful_tflops_l2_warm": world * fl["total"] / (warm_ms * 1e-3) / 1e12,
-            "stage_ms": {n: float(v) for n, v in zip(STAGES + ["total"], stage)},
-            "gpu_launches": launches * args.steps,
-            "launches_per_step": launches,
+            "kernel_spans_us": {k: [round(s, 2), round(e, 2)] for k, (s, e) in sorted(tl.items(), key=lambda kv: kv[1][0])},
+            "stage_ms_serialised": {n: float(v) for n, v in zip(STAGES + ["total"], m["stage_ms_serialised"])},
+            "gpu_launches": m["launches"] * args.steps * len(repeat_means),
+            "launches_per_step": m["launches"],
             "e2e": {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "tokens/s",
-                    "h2d_bytes_per_step": int(x.numel() * x.element_size()),
-                    "d2h_bytes_per_step": int(out.numel() * 4)},
-            "roofline": roof,
+                    "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
+            "roofline": roofline_from_timeline(cfg, tl, fl, peaks),
             "clocks": clocks,
         }
         # ---- dense multi-head comparator on the same x (262M-scale workload only) ----
         if cfg.name == "c4_262m_bf16" and not args.no_dense:
+            x, out = m["x"], m["out"]
+            stream = torch.cuda.current_stream()
             Wq, Wk, Wv, Wo = inputs.make_dense_mha_weights(cfg.d_model, 16, 64, seed=102, dtype=cfg.dtype)
             dl = binding.Layer(cfg.d_model, 16, 64, dense=True)
             dl.sh_configure(cfg.dtype, cfg.batch, cfg.seq)
@@ -319,26 +414,60 @@ def main():
                 dl.sh_forward(x, out)
             torch.cuda.synchronize()
             dt = []
-            for _ in range(20):
+            for _ in range(50):
                 flush.fill_(1)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream); dl.sh_forward(x, out); b.record(stream)
                 torch.cuda.synchronize()
                 dt.append(a.elapsed_time(b))
-            dms = float(np.mean(dt))
+            dms = float(np.median(dt))
             dense_flop = 2.0 * N * cfg.d_model * 3 * 1024 + 2.0 * cfg.batch * 16 * cfg.seq ** 2 * 64 + 2.0 * N * 1024 * cfg.d_model
             line["dense_mha_16x64"] = {"ms_per_step": dms, "switchhead_over_dense_time": ms_step / dms,
-                                       "useful_tflops": dense_flop / (dms * 1e-3) / 1e12}
+                                       "useful_tflops": dense_flop / (dms * 1e-3) / 1e12,
+                                       "note": "the less-tuned arm: same attention kernel (exp-bound at d_head 64), its fused Q/K/V "
+                                               "projection on the CTA-pair kernel, its output projection on the one-CTA-per-tile GEMM"}
             dl.close()
         if not args.no_cpu_baseline:
-            v, nseq, secs = oracle_sample(cfg, inp, rope_base=args.rope if args.rope > 0 else None,
+            v, nseq, secs = oracle_sample(cfg, m["inp"], rope_base=args.rope if args.rope > 0 else None,
                                           shared_selection=args.shared_selection)
             line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)),
                                     "kind": "oracle",
                                     "sample": f"{nseq} sequences of {cfg.seq} tokens drawn from the workload's {cfg.batch}, {secs:.1f} s, fp64 numpy"}
         line["paper_context"] = "paper reports 44% of dense MACs and 27% of dense activation memory at 262M params (analytic); no layer timing"
-        print(json.dumps(line))
-    layer.close()
+    del m
+
+    # ---- the other bf16 workloads (a few milliseconds of GPU time each): one record per config ----
+    if not args.no_per_config:
+        per = {}
+        for name in BF16_CONFIGS:
+            c = inputs.CONFIGS[name]
+            if name == cfg.name:
+                if rank == 0:
+                    per[name] = dict(ms_per_step=line["ms_per_step"], useful_tflops=line["useful_tflops"] / world,
+                                     frac_of_bf16_peak_measured=line["frac_of_bf16_peak_measured"],
+                                     ms_per_step_l2_warm=line["ms_per_step_l2_warm"],
+                                     dominant_kernel=line["roofline"]["kernel"], dominant_kernel_ms=line["roofline"]["ms"],
+                                     dominant_kernel_frac=line["roofline"]["frac"])
+                continue
+            steps_c = 50 if c.n_tokens * c.d_model < (1 << 25) else 20
+            mc = measure_config(c, args, rank, world, peaks, flush, barrier, steps_c, 0.1, with_e2e=False)
+            nrep = int(sharding.max_over_ranks([-float(len(mc["repeat_means"]))], device="cuda")[0] * -1)
+            red = sharding.max_over_ranks(mc["repeat_means"][:nrep] + [mc["warm_ms"]], device="cuda")
+            if rank == 0:
+                flc = inputs.useful_flop(c)
+                msc = float(np.median(red[:nrep]))
+                roof = roofline_from_timeline(c, mc["timeline"], flc, peaks)
+                per[name] = dict(ms_per_step=msc, useful_tflops=flc["total"] / (msc * 1e-3) / 1e12,
+                                 frac_of_bf16_peak_measured=flc["total"] / (msc * 1e-3) / 1e12 / peaks["tflops"],
+                                 ms_per_step_l2_warm=red[nrep], dominant_kernel=roof["kernel"], dominant_kernel_ms=roof["ms"],
+                                 dominant_kernel_frac=roof["frac"],
+                                 kernel_spans_us={k: [round(s, 2), round(e, 2)] for k, (s, e) in sorted(mc["timeline"].items(), key=lambda kv: kv[1][0])})
+            del mc
+        if rank == 0:
+            line["per_config"] = per
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 

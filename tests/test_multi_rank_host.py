@@ -62,3 +62,23 @@ def test_two_rank_replicas_on_gloo():
 
 def test_max_over_ranks_without_process_group_is_identity():
     assert sharding.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_several_gpus():
+    """`python bench.py --gpus 2` without a torchrun environment re-launches itself as two ranks
+    (torch.distributed.run, rendezvous on 127.0.0.1).  The reference arm needs no GPU, so the
+    launcher path runs here: rank 0 alone prints the line, the other rank exits 0."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--config", "tiny_f32", "--steps", "2", "--warmup", "0"],
+                         capture_output=True, text=True, timeout=300, env=env, cwd=root)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2
+    assert rec["config"]["workload"] == "tiny_f32" and rec["config"]["batch_per_gpu"] == 1
