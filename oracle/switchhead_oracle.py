@@ -33,6 +33,13 @@ All arithmetic is fp64 on the values handed in (already rounded to their storage
 no intermediate rounding.  Every stage is returned so that a failing comparison can be
 localised.
 
+Transformer-XL context (switchhead_xl_forward; the paper's main configuration): keys, values and the
+source-side gate over [cache; chunk], queries and the destination side over the chunk, optional
+relative-position term in Transformer-XL's form.  Pins (tests/test_oracle_xl_pins.py): no cache = the
+plain layer; one 2T pass = two T passes with the cache (with and without positions); W_Q = 0 gives
+running means over cache + chunk; cache visible to every query, later chunk tokens to none; a
+scalar-loop writing; zero position weights = no position term; the appendix's MAC / memory table.
+
 Pins (tests/test_oracle_pins.py): E=1 with zero gate weights equals 0.25 x textbook MHA
 (Eq. 2 and Eq. 3 forms, and torch's scaled_dot_product_attention); gate forced to 1 equals
 MHA; k=E equals the dense gate-weighted einsum; top-k equals a brute-force stable sort;
@@ -233,3 +240,98 @@ def dense_mha_forward(x, Wq, Wk, Wv, Wo, causal: bool = True):
             cat[:, h * D:(h + 1) * D] = (P / P.sum(axis=1, keepdims=True)) @ Vh
         y[b] = cat @ WO
     return y
+
+
+def xl_relative_embedding(n_dist: int, d_model: int) -> np.ndarray:
+    """Sinusoidal embedding of the relative distances 0 .. n_dist-1, as Transformer-XL (which the
+    paper's main models use: "Transformer-XL-style relative positional encoding") defines it:
+    row d = [sin(d w_0) .. sin(d w_{M/2-1}), cos(d w_0) .. cos(d w_{M/2-1})], w_i = 10000^(-2i/M)."""
+    if d_model % 2:
+        raise ValueError("d_model must be even")
+    w = np.power(10000.0, -2.0 * np.arange(d_model // 2, dtype=np.float64) / d_model)
+    ang = np.arange(n_dist, dtype=np.float64)[:, None] * w[None, :]
+    return np.concatenate([np.sin(ang), np.cos(ang)], axis=1)
+
+
+def switchhead_xl_forward(x, cache, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=None,
+                          Wr=None, u=None, v=None, return_stages: bool = True):
+    """SwitchHead layer with a Transformer-XL context (the paper's main configuration, Sec. 3 and the
+    appendix on resource usage: keys and values span C*T tokens, "C - 1 past chunks").
+
+    x [B, T, M]: the current chunk.  cache [B, Tc, M]: the layer INPUT of the previous chunk(s)
+    (Tc = (C-1)*T; Tc = 0 gives the plain layer).  The source side - keys, values, the source
+    gate and its expert selection - is computed from the context ctx = [cache; x] (Tc + T tokens);
+    the destination side - queries, the destination gate, the output - from x alone.  Query i
+    (context position Tc + i) sees context positions j <= Tc + i.
+
+    Relative positions (optional; Wr [H, M, D], u, v [H, D]): Transformer-XL's decomposition
+        score[i, j] = ( (q_i + u) . k_j  +  (q_i + v) . r_{(Tc+i) - j} ) / sqrt(D),
+        r_d = xl_relative_embedding(d) Wr^h,
+    u and v being the two global bias vectors of each head.  With Wr None the score is the plain
+    q_i . k_j / sqrt(D).  Returns y [B, T, M] and, if return_stages, Q [B,T,H,D], K, V [B,Tc+T,H,D],
+    Ahat [B,T,H,D] and the selections of both sides."""
+    f = lambda a: None if a is None else np.asarray(a, dtype=np.float64)
+    x, cache, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d, Wr, u, v = map(
+        f, (x, cache, Wq, Wk, Wv, Wo, Ws, Wd, bias_s, bias_d, Wr, u, v))
+    B, T, M = x.shape
+    Tc = 0 if cache is None else cache.shape[1]
+    H, E, _, D = Wv.shape
+    ctx = x if Tc == 0 else np.concatenate([cache, x], axis=1)             # [B, Tc + T, M]
+    CT = Tc + T
+    c2d, x2d = ctx.reshape(B * CT, M), x.reshape(B * T, M)
+
+    _, _, idxS, gateS = gate_and_select(c2d, Ws, bias_s, k)                # source side: every context token
+    _, _, idxD, gateD = gate_and_select(x2d, Wd, bias_d, k)                # destination side: the chunk's tokens
+
+    Q = np.empty((B * T, H, D))
+    K = np.empty((B * CT, H, D))
+    V = np.zeros((B * CT, H, D))
+    for h in range(H):
+        Q[:, h, :] = x2d @ Wq[h]
+        K[:, h, :] = c2d @ Wk[h]
+        for e in range(E):
+            for j in range(k):
+                rows = np.nonzero(idxS[:, h, j] == e)[0]
+                if rows.size:
+                    V[rows, h, :] += gateS[rows, h, j][:, None] * (c2d[rows] @ Wv[h, e])
+
+    R = None
+    if Wr is not None:
+        emb = xl_relative_embedding(CT, M)                                  # distances 0 .. CT-1
+        R = np.stack([emb @ Wr[h] for h in range(H)])                       # [H, CT, D]
+        u = np.zeros((H, D)) if u is None else u
+        v = np.zeros((H, D)) if v is None else v
+
+    Ahat = np.empty((B * T, H, D))
+    scale = 1.0 / np.sqrt(D)
+    qpos = Tc + np.arange(T)                                                # context position of query i
+    jpos = np.arange(CT)
+    hidden = jpos[None, :] > qpos[:, None]                                  # [T, CT]: keys after the query
+    dist = np.clip(qpos[:, None] - jpos[None, :], 0, CT - 1)                # relative distance where visible
+    for b in range(B):
+        qs, cs = slice(b * T, (b + 1) * T), slice(b * CT, (b + 1) * CT)
+        for h in range(H):
+            if R is None:
+                L = Q[qs, h, :] @ K[cs, h, :].T
+            else:
+                L = (Q[qs, h, :] + u[h]) @ K[cs, h, :].T                   # content terms
+                BD = (Q[qs, h, :] + v[h]) @ R[h].T                          # [T, CT] over distances
+                L = L + np.take_along_axis(BD, dist, axis=1)                # position terms, by distance
+            L = np.where(hidden, -np.inf, L * scale)
+            L = L - L.max(axis=1, keepdims=True)
+            P = np.exp(L)
+            A = P / P.sum(axis=1, keepdims=True)
+            Ahat[qs, h, :] = A @ V[cs, h, :]
+
+    y = np.zeros((B * T, M))
+    for h in range(H):
+        for e in range(E):
+            for j in range(k):
+                rows = np.nonzero(idxD[:, h, j] == e)[0]
+                if rows.size:
+                    y[rows] += gateD[rows, h, j][:, None] * (Ahat[rows, h, :] @ Wo[h, e])
+    out = {"y": y.reshape(B, T, M)}
+    if return_stages:
+        out.update(idxS=idxS, idxD=idxD, gateS=gateS, gateD=gateD, Q=Q.reshape(B, T, H, D),
+                   K=K.reshape(B, CT, H, D), V=V.reshape(B, CT, H, D), Ahat=Ahat.reshape(B, T, H, D))
+    return out
