@@ -427,6 +427,36 @@ def main():
                                        "note": "the less-tuned arm: same attention kernel (exp-bound at d_head 64), its fused Q/K/V "
                                                "projection on the CTA-pair kernel, its output projection on the one-CTA-per-tile GEMM"}
             dl.close()
+        # ---- the same layer as the paper's main models run it: with a Transformer-XL cache of one chunk (C = 2) ----
+        if cfg.name == "c4_262m_bf16" and not args.no_dense:
+            import dataclasses
+            cx = dataclasses.replace(cfg, name="c4_262m_bf16+cache", seq=2 * cfg.seq)
+            ix = inputs.make_inputs(cx, enforce_gap=False)
+            lx = binding.layer_from_inputs(ix, cache_len=cfg.seq)
+            xx = binding.to_device(ix.x, cfg.dtype)
+            ox = torch.empty((cfg.batch, cfg.seq, cfg.d_model), dtype=torch.float32, device="cuda")
+            stream = torch.cuda.current_stream()
+            for _ in range(3):
+                lx.sh_forward(xx, ox)
+            torch.cuda.synchronize()
+            dt = []
+            for _ in range(50):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); lx.sh_forward(xx, ox); b.record(stream)
+                torch.cuda.synchronize()
+                dt.append(a.elapsed_time(b))
+            assert lx.sh_last_status() == 0
+            Tc = cfg.seq
+            # keys and values (k experts) over cache + chunk, Q and O over the chunk; a query sees Tc + (t + 1) keys
+            fx = (2.0 * (2 * N) * cfg.d_model * cfg.n_heads * cfg.d_head + 2.0 * N * cfg.d_model * cfg.n_heads * cfg.d_head
+                  + 2.0 * (2 * N) * cfg.n_heads * cfg.k * cfg.d_model * cfg.d_head + 2.0 * N * cfg.n_heads * cfg.k * cfg.d_head * cfg.d_model
+                  + 4.0 * cfg.batch * cfg.n_heads * cfg.d_head * (cfg.seq * Tc + cfg.seq * cfg.seq / 2))
+            xms = float(np.median(dt))
+            line["xl_context_c2"] = {"cache_len": Tc, "chunk_tokens_per_step": N, "ms_per_step": xms,
+                                     "chunk_tokens_per_s": N / (xms * 1e-3), "useful_tflops": fx / (xms * 1e-3) / 1e12,
+                                     "note": "x = [cache; chunk] per sequence, out for the chunk; scores q.k (no relative-position term)"}
+            lx.close()
         if not args.no_cpu_baseline:
             v, nseq, secs = oracle_sample(cfg, m["inp"], rope_base=args.rope if args.rope > 0 else None,
                                           shared_selection=args.shared_selection)

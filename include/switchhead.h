@@ -96,6 +96,20 @@ sh_layer* sh_create_dense(int d_model, int n_heads, int d_head);
  * batch*seq*n_heads*k must be below 2^31.  Invalidates workspace and weights. */
 int sh_configure(sh_layer* layer, int dtype, int batch, int seq);
 
+/* The same with a Transformer-XL context (the paper's main models, Sec. 3 "Experiments" and the
+ * appendix on resource usage: the attention of a chunk of T tokens spans C*T keys, the extra
+ * (C-1)*T being a cache of the previous chunk(s); the paper uses C = 2).  x passed to sh_forward is
+ * then [B, cache_len + seq, d_model]: for every sequence the cached tokens - the INPUT this layer
+ * received for the previous chunk, which the caller keeps - followed by the current chunk.  Keys,
+ * values and the source-side gate with its expert selection are computed for all cache_len + seq
+ * tokens; queries, the destination-side gate and the output for the chunk's tokens only, each of
+ * which sees the whole cache and the chunk up to itself.  out is [B, seq, d_model].
+ * bf16 storage: cache_len and seq must be multiples of 128 (else SH_ERR_UNSUPPORTED).
+ * The relative-position term of Transformer-XL is not part of this library: scores are
+ * q.k / sqrt(d_head).  sh_set_rope is refused for a layer with a cache; sh_gate_topk and the debug
+ * buffers cover all cache_len + seq tokens.  cache_len = 0 is sh_configure. */
+int sh_configure_xl(sh_layer* layer, int dtype, int batch, int seq, int cache_len);
+
 /* Bytes of workspace sh_set_workspace needs for the current configuration (0 if not
  * configured). */
 size_t sh_workspace_bytes(const sh_layer* layer);
@@ -137,7 +151,7 @@ int sh_set_rope(sh_layer* layer, double base, void* stream);
 
 /* The whole forward pass (gates + top-k + bucket sort, Q/K projections, value experts,
  * causal attention, output experts with the gate-weighted sum) of x [B, T, d_model] into
- * out [B, T, d_model] fp32.  Both are device pointers aligned to 16 bytes (else
+ * out [B, T, d_model] fp32 (with a cache, sh_configure_xl: x [B, cache_len + T, d_model]).  Both are device pointers aligned to 16 bytes (else
  * SH_ERR_INVALID_ARG).  out is fully overwritten.  Enqueues kernels only. */
 int sh_forward(sh_layer* layer, const void* x, void* out, void* stream);
 

@@ -21,7 +21,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
                -4: "SH_ERR_WORKSPACE", -5: "SH_ERR_CUDA", -6: "SH_ERR_TIMEOUT", -7: "SH_ERR_BOUNDS"}
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
-EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_workspace_bytes", "sh_set_workspace",
+EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_configure_xl", "sh_workspace_bytes", "sh_set_workspace",
            "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
            "sh_noalloc_gate_topk", "sh_debug_buffer", "sh_last_status", "sh_status_block", "sh_clear_status", "sh_check_guards",
            "sh_selftest", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
@@ -42,6 +42,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_create_dense.argtypes = [i32] * 3
     lib.sh_configure.restype = i32
     lib.sh_configure.argtypes = [vp, i32, i32, i32]
+    lib.sh_configure_xl.restype = i32
+    lib.sh_configure_xl.argtypes = [vp, i32, i32, i32, i32]
     lib.sh_workspace_bytes.restype = sz
     lib.sh_workspace_bytes.argtypes = [vp]
     lib.sh_set_workspace.restype = i32
@@ -133,9 +135,14 @@ class Layer:
         self.dtype = None
         self.batch = self.seq = 0
 
-    def sh_configure(self, dtype: int, batch: int, seq: int, device="cuda") -> None:
-        _check(lib.sh_configure(self.handle, dtype, batch, seq))
-        self.dtype, self.batch, self.seq = dtype, batch, seq
+    def sh_configure(self, dtype: int, batch: int, seq: int, device="cuda", cache_len: int = 0) -> None:
+        """cache_len > 0: Transformer-XL context (sh_configure_xl): x is [B, cache_len + seq, M], out [B, seq, M]."""
+        if cache_len:
+            _check(lib.sh_configure_xl(self.handle, dtype, batch, seq, cache_len))
+        else:
+            _check(lib.sh_configure(self.handle, dtype, batch, seq))
+        # (self.seq: tokens per sequence the layer sees, cache included; self.seq_out: rows of out per sequence)
+        self.dtype, self.batch, self.seq, self.seq_out = dtype, batch, cache_len + seq, seq
         nbytes = lib.sh_workspace_bytes(self.handle)
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
         base = self.workspace.data_ptr()
@@ -158,7 +165,7 @@ class Layer:
     def sh_forward(self, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         assert x.is_cuda and x.is_contiguous()
         if out is None:
-            out = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+            out = torch.empty((x.shape[0], self.seq_out, x.shape[2]), dtype=torch.float32, device=x.device)
         _check(lib.sh_forward(self.handle, _ptr(x), _ptr(out), _stream()))
         return out
 
@@ -260,13 +267,14 @@ def to_device(a: Optional[np.ndarray], dtype: int, device="cuda") -> Optional[to
     return t.to(device).contiguous()
 
 
-def layer_from_inputs(inp, batch=None, seq=None, device="cuda", shared_selection=False) -> "Layer":
+def layer_from_inputs(inp, batch=None, seq=None, device="cuda", shared_selection=False, cache_len=0) -> "Layer":
     """Create, configure and load a Layer from a LayerInputs record (see inputs.py).
-    shared_selection: the source gate (Ws, bias_s) serves both sides; Wd and bias_d are not used."""
+    shared_selection: the source gate (Ws, bias_s) serves both sides; Wd and bias_d are not used.
+    cache_len: the first cache_len tokens of every sequence of inp.x are a Transformer-XL cache."""
     cfg = inp.cfg
     B, T = inp.x.shape[0], inp.x.shape[1]
     L = Layer(cfg.d_model, cfg.n_heads, cfg.d_head, cfg.n_experts, cfg.k, shared_selection=shared_selection)
-    L.sh_configure(cfg.dtype, B, T, device=device)
+    L.sh_configure(cfg.dtype, B, T - cache_len, device=device, cache_len=cache_len)
     dv = lambda a: to_device(a, cfg.dtype, device)
     bias = lambda a: None if a is None else torch.from_numpy(a).to(device)
     L.sh_set_weights(dv(inp.Wq), dv(inp.Wk), dv(inp.Wv), dv(inp.Wo), dv(inp.Ws),

@@ -92,6 +92,7 @@ static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_exper
   L->d.D = d_head <= 32 ? 32 : d_head <= 64 ? 64 : 128;        // sh_configure fixes it for the storage type
   L->d.sides = sides;
   L->d.causal = 1;
+  L->d.Tc = 0;
   L->d.stamps = nullptr;
   L->d.status = nullptr;
   L->d.G = sides * n_heads * n_experts;
@@ -111,39 +112,54 @@ extern "C" sh_layer* sh_create_dense(int d_model, int n_heads, int d_head) {
   return create_common(d_model, n_heads, d_head, 1, 1, true);
 }
 
-extern "C" int sh_configure(sh_layer* L, int dtype, int batch, int seq) {
+static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cache_len) {
   g_err[0] = 0;
   if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
   if (dtype != SH_F32 && dtype != SH_BF16) { sh_set_error("dtype must be SH_F32 or SH_BF16 (got %d)", dtype); return SH_ERR_INVALID_ARG; }
   if (batch < 1 || seq < 1) { sh_set_error("batch and seq must be >= 1 (got %d, %d)", batch, seq); return SH_ERR_INVALID_ARG; }
+  if (cache_len < 0) { sh_set_error("cache_len must be >= 0 (got %d)", cache_len); return SH_ERR_INVALID_ARG; }
   const ShDims& d0 = L->d;
   if (dtype == SH_BF16 && d0.M % 128 != 0) {
     sh_set_error("bf16 path needs d_model %% 128 == 0 (got d_model=%d)", d0.M);
     return SH_ERR_UNSUPPORTED;
   }
+  if (cache_len > 0 && L->dense) { sh_set_error("the dense comparator has no cache"); return SH_ERR_UNSUPPORTED; }
+  if (cache_len > 0 && dtype == SH_BF16 && (cache_len % 128 != 0 || seq % 128 != 0)) {
+    // the tensor-core attention and output kernels work on 128-token tiles that must not straddle the
+    // boundary between cache and chunk, nor two sequences
+    sh_set_error("bf16 path with a cache needs cache_len and seq to be multiples of 128 (got %d, %d)", cache_len, seq);
+    return SH_ERR_UNSUPPORTED;
+  }
   // d_head is stored padded with zero columns: to 64 or 128 on the tensor-core path, to 32, 64 or
   // 128 on the fp32 path (zero columns of W_Q, W_K, W_V and zero rows of W_O change no result)
   L->d.D = dtype == SH_BF16 ? (d0.Dt <= 64 ? 64 : 128) : (d0.Dt <= 32 ? 32 : d0.Dt <= 64 ? 64 : 128);
-  const long long slots = (long long)batch * seq * d0.H * d0.k;
-  if (slots >= (1ll << 31) || (long long)batch * seq * d0.M >= (1ll << 40)) {
-    sh_set_error("problem too large: batch*seq*n_heads*k = %lld must be below 2^31", slots);
+  const int T = cache_len + seq;                           // tokens of a sequence the layer sees: cache, then chunk
+  const long long slots = (long long)batch * T * d0.H * d0.k;
+  if (slots >= (1ll << 31) || (long long)batch * T * d0.M >= (1ll << 40)) {
+    sh_set_error("problem too large: batch*(cache_len+seq)*n_heads*k = %lld must be below 2^31", slots);
     return SH_ERR_UNSUPPORTED;
   }
   L->dtype = dtype;
-  L->d.B = batch; L->d.T = seq; L->d.N = batch * seq;
+  L->d.B = batch; L->d.T = T; L->d.Tc = cache_len; L->d.N = batch * T;
   L->d.nblk = (L->d.N + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
   L->d.max_tiles = (int)((slots + SH_TILE_ROWS - 1) / SH_TILE_ROWS) + d0.H * d0.E;
   L->d.tile_rows_src = SH_TILE_ROWS;
   // (k >= 3: the fp16 reductions of a value row arrive in a different order from run to run - two
   //  passes have been seen 1e-2 of the output RMS apart; with the first rows, which reach the output
   //  unaveraged, summed in fp32 they stay within 4e-3)
-  L->d.early_rows = (dtype == SH_BF16 && (seq >= SH_EARLY_MIN_SEQ || d0.k >= 3)) ? SH_EARLY_ROWS : 0;
+  L->d.early_rows = (dtype == SH_BF16 && (T >= SH_EARLY_MIN_SEQ || d0.k >= 3)) ? SH_EARLY_ROWS : 0;
   L->ws = nullptr; L->ws_bytes = 0; L->rope = false;
   L->d.status = nullptr;
   L->weights_set = false;
   sh_tc_release(L);
   layout_workspace(L);
   return SH_OK;
+}
+
+extern "C" int sh_configure(sh_layer* L, int dtype, int batch, int seq) { return configure_common(L, dtype, batch, seq, 0); }
+
+extern "C" int sh_configure_xl(sh_layer* L, int dtype, int batch, int seq, int cache_len) {
+  return configure_common(L, dtype, batch, seq, cache_len);
 }
 
 extern "C" size_t sh_workspace_bytes(const sh_layer* L) {
@@ -318,7 +334,7 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   if (all) sh_mark(L, 4, st);
   if (!(stages & SH_STAGE_O)) {
   } else if (!L->dense) {
-    SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
+    SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)sh_out_rows(d) * d.M * 4, st));
     ShGemmArgs o{};
     o.d = d; o.A = ws + L->o.ahat; o.lda = HD; o.a_head_stride = d.D; o.Bt = ws + L->o.wo; o.ldb = d.D;
     o.K = d.D; o.ncols = d.M;
@@ -376,6 +392,7 @@ extern "C" int sh_set_rope(sh_layer* L, double base, void* stream) {
   if (L->dtype < 0 || !L->ws) { sh_set_error("sh_set_rope needs a configured layer with its workspace"); return SH_ERR_NOT_CONFIGURED; }
   if (!(base >= 0.0) || base != base) { sh_set_error("rotary base must be positive (0 switches it off), got %g", base); return SH_ERR_INVALID_ARG; }
   if (base == 0.0) { L->rope = false; return SH_OK; }
+  if (L->d.Tc > 0) { sh_set_error("rotary embeddings are for the cache-less layer (the paper's RoPE models have no cache)"); return SH_ERR_UNSUPPORTED; }
   if (L->d.Dt % 2) { sh_set_error("rotary embedding needs an even d_head (got %d)", L->d.Dt); return SH_ERR_UNSUPPORTED; }
   const int n = L->d.T * (L->d.D / 2);
   sh_rope_table_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>((float2*)(L->ws + L->o.rope), L->d.T, L->d.D, L->d.Dt, base);

@@ -23,11 +23,27 @@ struct ShDims {
   int nblk;                // ceil(N / SH_TILE_ROWS)
   int max_tiles;           // upper bound on row tiles per side
   int tile_rows_src;       // rows per tile of the source-side (value expert) tile table: 128 or 256
+  int Tc;                  // Transformer-XL context: the first Tc tokens of every sequence are the cache (keys and values
+                           // only); queries, destination gates and out rows exist for the last T - Tc tokens.  0: no cache.
   int causal;              // 1: key s visible to query t iff s <= t (default); 0: every key of the sequence
   int early_rows;          // first tokens of every sequence whose value rows are summed in fp32 (SH_EARLY_ROWS or 0)
   unsigned long long* stamps;   // sh_forward_stamped: the pass's ShStampBlock in the workspace; nullptr otherwise
   int* status;             // the status block at the start of the workspace (nullptr: the allocation-free gate entry point)
 };
+
+// With a cache in front of every sequence (ShDims::Tc): the row of `out` that belongs to context token
+// `tok` (-1 for a cache token), and the context token of an out row.
+__host__ __device__ __forceinline__ int sh_out_row(const ShDims& d, int tok) {
+  if (d.Tc == 0) return tok;
+  const int b = tok / d.T, t = tok % d.T;
+  return t < d.Tc ? -1 : b * (d.T - d.Tc) + t - d.Tc;
+}
+__host__ __device__ __forceinline__ int sh_ctx_tok(const ShDims& d, int row) {
+  if (d.Tc == 0) return row;
+  const int Tq = d.T - d.Tc;
+  return (row / Tq) * d.T + d.Tc + row % Tq;
+}
+__host__ __device__ __forceinline__ int sh_out_rows(const ShDims& d) { return d.B * (d.T - d.Tc); }
 
 // Per-kernel time stamps of one forward pass (sh_forward_stamped), %globaltimer nanoseconds:
 // resident = first CTA of the kernel running, start = first CTA past its wait for the kernel before

@@ -407,7 +407,8 @@ sh_simt_gemm_kernel(ShGemmArgs g) {
         const int b = gr / d.T, t = gr % d.T;
         atomicAdd((TC*)g.out0 + (((size_t)b * d.H + h) * d.T + t) * d.D + n, sh_from_float<TC>(s_gate[lr] * v));
       } else if (EPI == SH_EPI_O) {
-        atomicAdd((float*)g.out0 + (size_t)gr * d.M + n, s_gate[lr] * v);
+        const int orow = sh_out_row(d, gr);                // (cache tokens have no output row)
+        if (orow >= 0) atomicAdd((float*)g.out0 + (size_t)orow * d.M + n, s_gate[lr] * v);
       } else {
         ((float*)g.out0)[(size_t)gr * g.ncols + n] = v;
       }
@@ -430,6 +431,7 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
   const long total = (long)d.B * d.H * d.T;
   if (qi >= total) return;
   const int t = (int)(qi % d.T);
+  if (t < d.Tc) return;                                 // a cache token: it is a key, not a query
   const long bh = qi / d.T;
   const TM* q = Q + qi * d.D;
   const TM* Kb = K + bh * d.T * d.D;

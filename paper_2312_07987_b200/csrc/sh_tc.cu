@@ -294,7 +294,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_GATE, x, nullptr, st))) return rc;
     if (zero_for_forward) {
       SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.v, 0, (size_t)d.N * d.H * d.D * 2, st));
-      if (S->simt_mask & SH_STAGE_O) SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)d.N * d.M * 4, st));
+      if (S->simt_mask & SH_STAGE_O) SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)sh_out_rows(d) * d.M * 4, st));
       L->launches += 2;
     }
     return SH_OK;
@@ -306,7 +306,9 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
   g.blockcnt = (int*)(ws + L->o.blockcnt);
   g.zero_v = zero_for_forward ? (void*)(ws + L->o.v) : nullptr;
-  g.zero_out = (zero_for_forward && (S->simt_mask & SH_STAGE_O)) ? (float*)out : nullptr;
+  g.zero_out = (zero_for_forward && (S->simt_mask & SH_STAGE_O) && d.Tc == 0) ? (float*)out : nullptr;
+  if (zero_for_forward && (S->simt_mask & SH_STAGE_O) && d.Tc > 0)          // (out has fewer rows than there are tokens)
+    SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)sh_out_rows(d) * d.M * 4, st));
   g.status = (int*)(ws + L->o.status);
   const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
   const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
@@ -571,7 +573,7 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
   } else {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
-    const int nq = (d.T + 255) / 256;
+    const int nq = ((d.T + 127) / 128 - d.Tc / 128 + 1) / 2;    // pairs of 128-query tiles behind the cache
     const unsigned grid = (unsigned)(nq * d.B * d.H);
     a.balanced = d.causal && (int)grid <= L->sm_count && S->attn_balanced;
     if (d.D == 128) {
@@ -611,14 +613,14 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     if (pair) {
       // 256 tokens x 256 features per unit, gates folded into the A operand
       const int psm = d.D == 128 ? OprojPairSmem<128>::TOTAL : OprojPairSmem<64>::TOTAL;
-      a.nwork = ((d.N + 255) / 256) * ((d.M + 255) / 256);
+      a.nwork = ((sh_out_rows(d) + 255) / 256) * ((d.M + 255) / 256);
       const unsigned pgrid = 2u * (unsigned)(a.nwork < S->o_pairs_max ? a.nwork : S->o_pairs_max);
       const __half* ahat = (const __half*)(ws + L->o.ahat);
       if (d.D == 128) rc = launch_k_pairs(pdl, sh_tc_oproj_pair_kernel<128>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
       else rc = launch_k_pairs(pdl, sh_tc_oproj_pair_kernel<64>, dim3(pgrid), dim3(480), psm, st, S->map_wo, a, ahat);
       if (rc) return rc;
     } else {
-      a.nwork = d.nblk * ((d.M + 255) / 256);
+      a.nwork = ((sh_out_rows(d) + 127) / 128) * ((d.M + 255) / 256);
       const unsigned grid = (unsigned)(a.nwork < L->sm_count ? a.nwork : L->sm_count);
       int as = 3, smem = 0;
       for (; as >= 2; --as) {

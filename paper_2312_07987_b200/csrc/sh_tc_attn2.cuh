@@ -62,18 +62,20 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 
   const ShDims& d = g.d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nq = (d.T + 255) / 256;
   const int BH = d.B * d.H;
   const int bh = blockIdx.x % BH;
   // The two 128-query tiles of this CTA.  Saturated grid: adjacent tiles, heaviest pairs first (the
   // most steps in which both tiles share a K/V stage).  Grid that fits the GPU in one wave
   // (g.balanced): tile p with tile ntile-1-p, so that under the causal mask every CTA has the same
   // number of tile-steps and the kernel ends when the average CTA ends, not the heaviest.
-  const int ntile = (d.T + 127) / 128;
+  // (with a Transformer-XL cache of d.Tc tokens - a multiple of 128 - in front of the sequence, the
+  //  query tiles start behind it; the key tiles start at 0 as ever)
+  const int ntile = (d.T + 127) / 128, t_first = d.Tc / 128;
+  const int nq = (ntile - t_first + 1) / 2;
   const int pr = (int)(blockIdx.x / BH);
   int ta, tb;
-  if (g.balanced) { ta = pr; tb = ntile - 1 - pr; }
-  else { ta = 2 * (nq - 1 - pr); tb = ta + 1; }
+  if (g.balanced) { ta = t_first + pr; tb = ntile - 1 - pr; }
+  else { ta = t_first + 2 * (nq - 1 - pr); tb = ta + 1; }
   const bool has_b = tb < ntile && tb != ta;
   const int qrow[2] = {ta * 128, tb * 128};
   // key tiles each query tile attends to: up to its diagonal tile, or (d.causal == 0) all of them

@@ -106,7 +106,9 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
       int gh = 0, s = 0;                                    // running head counter, weight-ring stage
       uint32_t apar = 1;                                    // parity of a_empty[s] for the current ring pass
       for (int w = blockIdx.x; w < g.nwork && !dead; w += gridDim.x) {
-        const int row0 = (w / nfc) * 128, fc = w % nfc;
+        // (a 128-row tile of out is 128 consecutive tokens: with a cache in front of every sequence the
+        //  chunk length is a multiple of 128, so a tile never straddles two sequences)
+        const int row0 = sh_ctx_tok(d, (w / nfc) * 128), fc = w % nfc;
         for (int h = 0; h < d.H && !dead; ++h, ++gh) {
           const int bs = gh & 1;
           if (!mbar_wait(&b_empty[bs], ((gh >> 1) & 1) ^ 1, g.status, dead)) break;
@@ -170,8 +172,9 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
     uint32_t wpar = 0;                                     // parity of this work unit for sel_free / sel_ready
     bool ok = true;
     for (int w = blockIdx.x; w < g.nwork && ok; w += gridDim.x, wpar ^= 1) {
-      const int row0 = (w / nfc) * 128, fc = w % nfc;
-      const int nrows = min(128, d.N - row0);
+      const int row0 = (w / nfc) * 128, fc = w % nfc;      // rows of out
+      const int nrows = min(128, sh_out_rows(d) - row0);
+      const int tok0 = sh_ctx_tok(d, row0);                // their tokens (consecutive)
       // this tile's destination-side selections (contiguous in global memory) -> shared memory
       // (mbarriers with bounded waits rather than bar.sync, so that a thread that gave up cannot
       //  leave the others stuck)
@@ -179,8 +182,8 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
       if (!mbar_wait(sel_free, wpar, g.status, dead)) { ok = false; break; }
       {
         const int total = nrows * per_tok;
-        const int* gi_ = g.idx + (size_t)row0 * per_tok;
-        const float* gg = g.gate + (size_t)row0 * per_tok;
+        const int* gi_ = g.idx + (size_t)tok0 * per_tok;
+        const float* gg = g.gate + (size_t)tok0 * per_tok;
         for (int i = et; i < 128 * per_tok; i += 256) {
           s_idx[i] = i < total ? gi_[i] : -1;
           s_gt[i] = i < total ? gg[i] : 0.f;

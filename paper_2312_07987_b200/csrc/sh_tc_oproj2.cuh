@@ -100,6 +100,7 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   const int nfc = (d.M + 255) / 256;
   const int HD = d.H * D;
+  const int nout = sh_out_rows(d);                       // rows of out (= tokens, unless a cache sits in front of every sequence)
   bool dead = false;
 
   if (threadIdx.x == 0) {
@@ -200,8 +201,9 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
     // ~1 us); (fw, fh) walk the units and heads of this pair in step with the consuming loop
     int fw = pair, fh = 0;
     auto fetch = [&]() {
-      const int tokn = (fw / nfc) * 256 + (int)rank * 128 + row;
-      const bool live = fw < g.nwork && tokn < d.N;
+      const int orow = (fw / nfc) * 256 + (int)rank * 128 + row;    // row of out; its token sits behind the cache, if there is one
+      const bool live = fw < g.nwork && orow < nout;
+      const int tokn = live ? sh_ctx_tok(d, orow) : 0;
       const uint4* src = reinterpret_cast<const uint4*>(ahat + (size_t)tokn * HD + fh * D + kh * (D / 2));
 #pragma unroll
       for (int i = 0; i < CH; ++i) nxt[i] = live ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
@@ -276,7 +278,7 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
     for (int w = pair; w < g.nwork; w += npairs, ++un) {
       const int buf = un & 1;
       const int row0 = (w / nfc) * 256 + (int)rank * 128, fc = w % nfc;
-      const int rows_here = min(32, d.N - row0 - q * 32);  // <= 0: these tokens are past the end
+      const int rows_here = min(32, nout - row0 - q * 32); // <= 0: these rows are past the end
       if (!mbar_wait(&d_full[buf], (un >> 1) & 1, g.status, dead)) break;
       tc_fence_after();
       float* obase = g.out + (size_t)(row0 + q * 32) * d.M + fc * 256;
