@@ -105,10 +105,22 @@ int sh_configure(sh_layer* layer, int dtype, int batch, int seq);
  * tokens; queries, the destination-side gate and the output for the chunk's tokens only, each of
  * which sees the whole cache and the chunk up to itself.  out is [B, seq, d_model].
  * bf16 storage: cache_len and seq must be multiples of 128 (else SH_ERR_UNSUPPORTED).
- * The relative-position term of Transformer-XL is not part of this library: scores are
- * q.k / sqrt(d_head).  sh_set_rope is refused for a layer with a cache; sh_gate_topk and the debug
+ * Scores are q.k / sqrt(d_head) unless sh_set_xl_positions adds Transformer-XL's relative-position
+ * term (fp32 configuration).  sh_set_rope is refused for a layer with a cache; sh_gate_topk and the debug
  * buffers cover all cache_len + seq tokens.  cache_len = 0 is sh_configure. */
 int sh_configure_xl(sh_layer* layer, int dtype, int batch, int seq, int cache_len);
+
+/* The relative-position term of Transformer-XL (the positional encoding of the paper's main models;
+ * the paper cites it and does not restate it) for the fp32 configuration:
+ *   score[t, s] = ( (q_t + u^h) . k_s  +  (q_t + v^h) . r^h_{t-s} ) / sqrt(d_head),
+ *   r^h_dist = emb(dist) Wr^h,   emb(dist) = [sin(dist w_0..), cos(dist w_0..)], w_i = 10000^(-2i/d_model)
+ * where t and s are positions in [cache; chunk] and only keys s <= t are visible.
+ *   Wr [H, d_model, d_head] fp32, u, v [H, d_head] fp32 (NULL: zero).  Wr = NULL switches the term off.
+ * Builds the distance table for the configured sequence length in the workspace (asynchronously
+ * on `stream`); valid until the next sh_configure / sh_set_workspace.  Works with and without a
+ * cache.  SH_ERR_UNSUPPORTED for bf16 storage (the tensor-core attention kernel has no position
+ * term) and while rotary embeddings are on. */
+int sh_set_xl_positions(sh_layer* layer, const float* Wr, const float* u, const float* v, void* stream);
 
 /* Bytes of workspace sh_set_workspace needs for the current configuration (0 if not
  * configured). */

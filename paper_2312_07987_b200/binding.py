@@ -22,7 +22,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
 EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_configure_xl", "sh_workspace_bytes", "sh_set_workspace",
-           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_forward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
+           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_set_xl_positions", "sh_forward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
            "sh_noalloc_gate_topk", "sh_debug_buffer", "sh_last_status", "sh_status_block", "sh_clear_status", "sh_check_guards",
            "sh_selftest", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
 STAMP_KERNELS = ["gate", "sort", "qk_a", "qk_b", "v", "attn", "o"]
@@ -72,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_noalloc_gate_topk.argtypes = [i32] * 6 + [vp] * 8
     lib.sh_set_causal.restype = i32
     lib.sh_set_causal.argtypes = [vp, i32]
+    lib.sh_set_xl_positions.restype = i32
+    lib.sh_set_xl_positions.argtypes = [vp, vp, vp, vp, vp]
     lib.sh_set_rope.restype = i32
     lib.sh_set_rope.argtypes = [vp, ctypes.c_double, vp]
     lib.sh_debug_buffer.restype = i32
@@ -158,6 +160,13 @@ class Layer:
 
     def sh_set_causal(self, causal: bool) -> None:
         _check(lib.sh_set_causal(self.handle, 1 if causal else 0))
+
+    def sh_set_xl_positions(self, Wr, u=None, v=None) -> None:
+        """Transformer-XL relative-position term (fp32 layers): Wr [H, M, D], u, v [H, D] fp32 device tensors; None switches it off."""
+        for t in (Wr, u, v):
+            assert t is None or (t.is_cuda and t.is_contiguous() and t.dtype == torch.float32)
+        _check(lib.sh_set_xl_positions(self.handle, _ptr(Wr), _ptr(u), _ptr(v), _stream()))
+        torch.cuda.current_stream().synchronize()   # the source tensors may now be released
 
     def sh_set_rope(self, base: float) -> None:
         _check(lib.sh_set_rope(self.handle, float(base), _stream()))

@@ -75,6 +75,12 @@ static void layout_workspace(sh_layer* L) {
   const bool early = L->dtype == SH_BF16 && !L->dense;
   o.vearly = take(early ? (size_t)d.B * HD * SH_EARLY_ROWS * 4 : 16);
   o.vearly_cnt = take(early ? (size_t)d.B * d.H * SH_EARLY_ROWS * 4 : 16);
+  // fp32 configuration: Transformer-XL relative positions (sh_set_xl_positions): the embedding of the
+  // distances [T, M], its projection R [H, T, D] and the two bias vectors [2, H, D]
+  const bool xlp = L->dtype == SH_F32 && !L->dense;
+  o.xl_emb = take(xlp ? (size_t)d.T * d.M * 4 : 16);
+  o.xl_r = take(xlp ? (size_t)d.H * d.T * d.D * 4 : 16);
+  o.xl_uv = take(xlp ? (size_t)2 * d.H * d.D * 4 : 16);
   o.stamps = take(sizeof(ShStampBlock));
   o.total = off;
 }
@@ -148,7 +154,7 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
   //  passes have been seen 1e-2 of the output RMS apart; with the first rows, which reach the output
   //  unaveraged, summed in fp32 they stay within 4e-3)
   L->d.early_rows = (dtype == SH_BF16 && (T >= SH_EARLY_MIN_SEQ || d0.k >= 3)) ? SH_EARLY_ROWS : 0;
-  L->ws = nullptr; L->ws_bytes = 0; L->rope = false;
+  L->ws = nullptr; L->ws_bytes = 0; L->rope = false; L->xl_positions = false;
   L->d.status = nullptr;
   L->weights_set = false;
   sh_tc_release(L);
@@ -174,7 +180,7 @@ extern "C" int sh_set_workspace(sh_layer* L, void* workspace, size_t bytes) {
   if (!workspace) { sh_set_error("workspace is NULL"); return SH_ERR_WORKSPACE; }
   if ((uintptr_t)workspace % 256 != 0) { sh_set_error("workspace must be 256-byte aligned"); return SH_ERR_WORKSPACE; }
   if (bytes < L->o.total) { sh_set_error("workspace too small: %zu bytes given, %zu needed", bytes, L->o.total); return SH_ERR_WORKSPACE; }
-  L->ws = (char*)workspace; L->ws_bytes = bytes; L->weights_set = false; L->rope = false;
+  L->ws = (char*)workspace; L->ws_bytes = bytes; L->weights_set = false; L->rope = false; L->xl_positions = false;
   L->d.status = (int*)(L->ws + L->o.status);
   sh_tc_release(L);
   return SH_OK;
@@ -198,7 +204,7 @@ static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void
   char* ws = L->ws;
   const long HD = (long)d.H * d.D;
   SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.status, 0, 256, st));
-  SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.vearly, 0, L->o.stamps - L->o.vearly, st));   // early-row sums and counters
+  SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.vearly, 0, L->o.xl_emb - L->o.vearly, st));   // early-row sums and counters
   for (int i = 0; i < L->n_guards; ++i) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->guard_off[i], SH_GUARD_BYTE, SH_GUARD_BYTES, st));
   // Wq, Wk [H, M, Dt] -> Wqk[(which*H + h)*D + dd][m]   (rows dd >= Dt stay zero)
   TI* wqk = (TI*)(ws + L->o.wqk);
@@ -327,8 +333,14 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   if (all) sh_mark(L, 3, st);
   if (stages & SH_STAGE_ATTN) {
     const long nq = (long)d.B * d.H * d.T;
+    ShXlPos xl{};
+    if (L->xl_positions) {
+      xl.R = (const float*)(ws + L->o.xl_r);
+      xl.u = (const float*)(ws + L->o.xl_uv); xl.v = xl.u + (size_t)d.H * d.D;
+      xl.qscale = qscale;
+    }
     sh_simt_attention_kernel<TM><<<(unsigned)((nq + 3) / 4), 128, 0, st>>>((const TM*)(ws + L->o.q),
-        (const TM*)(ws + L->o.k), (const TM*)(ws + L->o.v), (TM*)(ws + L->o.ahat), d);
+        (const TM*)(ws + L->o.k), (const TM*)(ws + L->o.v), (TM*)(ws + L->o.ahat), d, xl);
     L->launches += 1;
   }
   if (all) sh_mark(L, 4, st);
@@ -386,12 +398,42 @@ extern "C" int sh_set_causal(sh_layer* L, int causal) {
   return SH_OK;
 }
 
+extern "C" int sh_set_xl_positions(sh_layer* L, const float* Wr, const float* u, const float* v, void* stream) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0 || !L->ws) { sh_set_error("sh_set_xl_positions needs a configured layer with its workspace"); return SH_ERR_NOT_CONFIGURED; }
+  if (!Wr) { L->xl_positions = false; return SH_OK; }
+  if (L->dtype != SH_F32 || L->dense) {
+    sh_set_error("the relative-position term is built for the fp32 configuration of a SwitchHead layer only");
+    return SH_ERR_UNSUPPORTED;
+  }
+  if (L->rope) { sh_set_error("rotary embeddings are switched on: one positional encoding at a time"); return SH_ERR_UNSUPPORTED; }
+  const ShDims& d = L->d;
+  if (d.M % 2) { sh_set_error("the sinusoidal embedding needs an even d_model"); return SH_ERR_UNSUPPORTED; }
+  cudaStream_t st = (cudaStream_t)stream;
+  float* emb = (float*)(L->ws + L->o.xl_emb);
+  float* R = (float*)(L->ws + L->o.xl_r);
+  float* uv = (float*)(L->ws + L->o.xl_uv);
+  const int ne = d.T * (d.M / 2);
+  sh_xl_embedding_kernel<<<(ne + 255) / 256, 256, 0, st>>>(emb, d.T, d.M);
+  const long nr = (long)d.H * d.T * d.D;
+  sh_xl_project_kernel<<<(unsigned)((nr + 255) / 256), 256, 0, st>>>(emb, Wr, R, d.H, d.T, d.M, d.D, d.Dt);
+  // u, v [H, Dt] -> [H, D] (zero padding: the padded columns of K and R are zero anyway)
+  SH_CUDA_CHECK(cudaMemsetAsync(uv, 0, (size_t)2 * d.H * d.D * 4, st));
+  if (u) SH_CUDA_CHECK(cudaMemcpy2DAsync(uv, (size_t)d.D * 4, u, (size_t)d.Dt * 4, (size_t)d.Dt * 4, d.H, cudaMemcpyDeviceToDevice, st));
+  if (v) SH_CUDA_CHECK(cudaMemcpy2DAsync(uv + (size_t)d.H * d.D, (size_t)d.D * 4, v, (size_t)d.Dt * 4, (size_t)d.Dt * 4, d.H, cudaMemcpyDeviceToDevice, st));
+  SH_CUDA_CHECK(cudaGetLastError());
+  L->xl_positions = true;
+  return SH_OK;
+}
+
 extern "C" int sh_set_rope(sh_layer* L, double base, void* stream) {
   g_err[0] = 0;
   if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
   if (L->dtype < 0 || !L->ws) { sh_set_error("sh_set_rope needs a configured layer with its workspace"); return SH_ERR_NOT_CONFIGURED; }
   if (!(base >= 0.0) || base != base) { sh_set_error("rotary base must be positive (0 switches it off), got %g", base); return SH_ERR_INVALID_ARG; }
   if (base == 0.0) { L->rope = false; return SH_OK; }
+  if (L->xl_positions) { sh_set_error("relative positions are switched on: one positional encoding at a time"); return SH_ERR_UNSUPPORTED; }
   if (L->d.Tc > 0) { sh_set_error("rotary embeddings are for the cache-less layer (the paper's RoPE models have no cache)"); return SH_ERR_UNSUPPORTED; }
   if (L->d.Dt % 2) { sh_set_error("rotary embedding needs an even d_head (got %d)", L->d.Dt); return SH_ERR_UNSUPPORTED; }
   const int n = L->d.T * (L->d.D / 2);
@@ -500,9 +542,9 @@ extern "C" int sh_clear_status(sh_layer* L, void* stream) {
   SH_CUDA_CHECK(cudaMemsetAsync(L->ws + L->o.status, 0, 256, (cudaStream_t)stream));
   // (and the early-row value sums with their arrival counters, which the last arrival of a row clears;
   //  the guards between and behind the two are rewritten)
-  SH_CUDA_CHECK(cudaMemsetAsync(L->ws + L->o.vearly, 0, L->o.stamps - L->o.vearly, (cudaStream_t)stream));
+  SH_CUDA_CHECK(cudaMemsetAsync(L->ws + L->o.vearly, 0, L->o.xl_emb - L->o.vearly, (cudaStream_t)stream));
   for (int i = 0; i < L->n_guards; ++i)
-    if (L->guard_off[i] >= L->o.vearly && L->guard_off[i] < L->o.stamps)
+    if (L->guard_off[i] >= L->o.vearly && L->guard_off[i] < L->o.xl_emb)
       SH_CUDA_CHECK(cudaMemsetAsync(L->ws + L->guard_off[i], SH_GUARD_BYTE, SH_GUARD_BYTES, (cudaStream_t)stream));
   return SH_OK;
 }

@@ -421,11 +421,22 @@ sh_simt_gemm_kernel(ShGemmArgs g) {
 // keys in chunks of 32 (lane = key), online softmax in base 2 (Q carries log2(e)/sqrt(D)).
 // Q, K, V [B, H, T, D]; Ahat [B*T, H, D].
 // ---------------------------------------------------------------------------------------
+// Optional relative-position term of Transformer-XL (fp32 configuration, sh_set_xl_positions):
+//   score[t, s] = ((q_t + u) . k_s + (q_t + v) . r_{t-s}) / sqrt(D),   r_dist = xl.R[h, dist, :]
+// Q is stored pre-multiplied by c = log2(e)/sqrt(D), so the kernel keeps q + c*u and q + c*v.
+struct ShXlPos {
+  const float* R;        // [H, T, D] projected embeddings of the distances 0..T-1, or nullptr: plain q.k scores
+  const float* u;        // [H, D] content bias
+  const float* v;        // [H, D] position bias
+  float qscale;          // c
+};
+
 template <typename TM>
 __global__ void __launch_bounds__(128)
 sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, const TM* __restrict__ V,
-                         TM* __restrict__ Ahat, ShDims d) {
+                         TM* __restrict__ Ahat, ShDims d, ShXlPos xl) {
   __shared__ float s_q[4][128];
+  __shared__ float s_qv[4][128];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long qi = (long)blockIdx.x * 4 + warp;          // index over (b, h, t)
   const long total = (long)d.B * d.H * d.T;
@@ -436,7 +447,13 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
   const TM* q = Q + qi * d.D;
   const TM* Kb = K + bh * d.T * d.D;
   const TM* Vb = V + bh * d.T * d.D;
-  for (int i = lane; i < d.D; i += 32) s_q[warp][i] = sh_to_float<TM>(q[i]);
+  const int hq = (int)(bh % d.H);
+  const float* Rh = xl.R ? xl.R + (size_t)hq * d.T * d.D : nullptr;
+  for (int i = lane; i < d.D; i += 32) {
+    const float qv = sh_to_float<TM>(q[i]);
+    s_q[warp][i] = Rh ? qv + xl.qscale * xl.u[hq * d.D + i] : qv;
+    s_qv[warp][i] = Rh ? qv + xl.qscale * xl.v[hq * d.D + i] : 0.f;
+  }
   __syncwarp();
   float o[4] = {0.f, 0.f, 0.f, 0.f};                    // lane owns d = lane + 32*i
   float m = -INFINITY, l = 0.f;
@@ -448,6 +465,12 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
       const TM* kr = Kb + (long)s * d.D;
       float a = 0.f;
       for (int i = 0; i < d.D; ++i) a = fmaf(s_q[warp][i], sh_to_float<TM>(kr[i]), a);
+      if (Rh) {                                         // position term: the embedding of the distance t - s (keys behind the query only)
+        const float* rr = Rh + (long)max(t - s, 0) * d.D;
+        float p2 = 0.f;
+        for (int i = 0; i < d.D; ++i) p2 = fmaf(s_qv[warp][i], rr[i], p2);
+        a += p2;
+      }
       sc = a;
     }
     float cm = sc;
@@ -478,4 +501,32 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
 #pragma unroll
   for (int i = 0; i < 4; ++i)
     if (lane + 32 * i < d.D) dst[lane + 32 * i] = sh_from_float<TM>(o[i] * inv);
+}
+
+// ---------------------------------------------------------------------------------------
+// Transformer-XL relative positions, one-time set-up: the sinusoidal embedding of the distances
+// 0..T-1 (row dist = [sin(dist w_0) .. sin(dist w_{M/2-1}), cos(dist w_0) .. cos(dist w_{M/2-1})],
+// w_i = 10000^(-2i/M), angles in double precision), and its projection R[h, dist, :] = emb[dist] Wr^h.
+// ---------------------------------------------------------------------------------------
+static __global__ void sh_xl_embedding_kernel(float* emb, int T, int M) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T * (M / 2)) return;
+  const int dist = i / (M / 2), f = i % (M / 2);
+  const double w = pow(10000.0, -2.0 * (double)f / (double)M);
+  double s, c;
+  sincos((double)dist * w, &s, &c);
+  emb[(size_t)dist * M + f] = (float)s;
+  emb[(size_t)dist * M + M / 2 + f] = (float)c;
+}
+
+// R[h, dist, dd] = sum_m emb[dist, m] * Wr[h, m, dd]   (Wr row-major [H, M, Dt]; columns dd >= Dt of the padded D are zero)
+static __global__ void sh_xl_project_kernel(const float* __restrict__ emb, const float* __restrict__ Wr, float* __restrict__ R,
+                                            int H, int T, int M, int D, int Dt) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long)H * T * D) return;
+  const int dd = (int)(i % D), dist = (int)((i / D) % T), h = (int)(i / ((long)D * T));
+  double acc = 0.0;
+  if (dd < Dt)
+    for (int m = 0; m < M; ++m) acc += (double)emb[(size_t)dist * M + m] * (double)Wr[((size_t)h * M + m) * Dt + dd];
+  R[i] = (float)acc;
 }

@@ -99,3 +99,42 @@ def test_xl_argument_checks():
     with pytest.raises(binding.SwitchHeadError):
         Ld.sh_configure(binding.SH_F32, 1, 16, cache_len=16)
     Ld.close()
+
+
+@pytest.mark.parametrize("T,Tc,B,E,k,H,D,M", [(64, 64, 1, 4, 2, 2, 32, 128), (33, 0, 2, 4, 2, 2, 32, 64), (17, 45, 2, 5, 3, 3, 22, 128),
+                                                (130, 70, 1, 3, 1, 2, 64, 64)])
+def test_xl_relative_positions_f32(T, Tc, B, E, k, H, D, M):
+    """The full Transformer-XL layer of the paper's main models in the fp32 configuration: cache plus the
+    relative-position term (q + u).k + (q + v).r_dist, against the oracle."""
+    cfg = inputs.LayerConfig("xl_pos", inputs.DTYPE_F32, B, Tc + T, M, H, D, E, k, seed=600 + T)
+    inp = inputs.make_inputs(cfg)
+    rng = np.random.default_rng(601)
+    Wr = (rng.standard_normal((H, M, D)) / np.sqrt(M)).astype(np.float32)
+    u = (0.5 * rng.standard_normal((H, D))).astype(np.float32)
+    v = (0.5 * rng.standard_normal((H, D))).astype(np.float32)
+    layer = binding.layer_from_inputs(inp, cache_len=Tc)
+    x = binding.to_device(inp.x, cfg.dtype)
+    y_plain = layer.sh_forward(x).clone()
+    layer.sh_set_xl_positions(*(torch.from_numpy(a).cuda() for a in (Wr, u, v)))
+    y = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0
+    ref = switchhead_xl_forward(inp.x[:, Tc:], inp.x[:, :Tc] if Tc else None, inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd,
+                                cfg.k, inp.bias_s, inp.bias_d, Wr=Wr, u=u, v=v)
+    err = pu.rel_rms_err(y.cpu().numpy(), ref["y"])
+    assert err < 1e-4, f"output max-abs error / rms = {err:.3e}"
+    assert not torch.allclose(y, y_plain, rtol=1e-3, atol=1e-3), "the position term changed nothing"
+    layer.sh_set_xl_positions(None)                       # off again: the plain scores
+    y_off = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert pu.rel_rms_err(y_off.cpu().numpy(), y_plain.cpu().numpy()) < 1e-5
+    layer.close()
+
+
+def test_xl_relative_positions_are_refused_for_bf16():
+    L = binding.Layer(256, 2, 64, 4, 2)
+    L.sh_configure(binding.SH_BF16, 1, 128)
+    with pytest.raises(binding.SwitchHeadError) as e:
+        L.sh_set_xl_positions(torch.zeros((2, 256, 64), device="cuda"))
+    assert "fp32" in str(e.value)
+    L.close()
