@@ -89,13 +89,13 @@ static sh_layer* create_common(int d_model, int n_heads, int d_head, int n_exper
   g_err[0] = 0;
   if (d_model <= 0 || d_model % 64 != 0) { sh_set_error("d_model must be a positive multiple of 64 (got %d)", d_model); return nullptr; }
   if (n_heads < 1) { sh_set_error("n_heads must be >= 1 (got %d)", n_heads); return nullptr; }
-  if (d_head < 1 || d_head > 128) { sh_set_error("d_head must be in 1..128 (got %d)", d_head); return nullptr; }
+  if (d_head < 1 || d_head > 256) { sh_set_error("d_head must be in 1..256 (got %d)", d_head); return nullptr; }
   if (n_experts < 1 || n_experts > 32) { sh_set_error("n_experts must be in 1..32 (got %d)", n_experts); return nullptr; }
   if (k < 1 || k > n_experts) { sh_set_error("k must be in 1..n_experts (got k=%d, n_experts=%d)", k, n_experts); return nullptr; }
   sh_layer* L = new (std::nothrow) sh_layer();
   if (!L) { sh_set_error("out of host memory"); return nullptr; }
   L->d.M = d_model; L->d.H = n_heads; L->d.Dt = d_head; L->d.E = n_experts; L->d.k = k;
-  L->d.D = d_head <= 32 ? 32 : d_head <= 64 ? 64 : 128;        // sh_configure fixes it for the storage type
+  L->d.D = d_head <= 32 ? 32 : d_head <= 64 ? 64 : d_head <= 128 ? 128 : 256;   // sh_configure fixes it for the storage type
   L->d.sides = sides;
   L->d.causal = 1;
   L->d.Tc = 0;
@@ -129,6 +129,11 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
     sh_set_error("bf16 path needs d_model %% 128 == 0 (got d_model=%d)", d0.M);
     return SH_ERR_UNSUPPORTED;
   }
+  if (dtype == SH_BF16 && d0.Dt > 128) {
+    // (the tensor-core attention kernel keeps S and O of two query tiles in the 512 TMEM columns: d_head <= 128)
+    sh_set_error("bf16 path supports d_head up to 128 (got %d); the fp32 configuration takes up to 256", d0.Dt);
+    return SH_ERR_UNSUPPORTED;
+  }
   if (cache_len > 0 && L->dense) { sh_set_error("the dense comparator has no cache"); return SH_ERR_UNSUPPORTED; }
   if (cache_len > 0 && dtype == SH_BF16 && (cache_len % 128 != 0 || seq % 128 != 0)) {
     // the tensor-core attention and output kernels work on 128-token tiles that must not straddle the
@@ -138,7 +143,7 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
   }
   // d_head is stored padded with zero columns: to 64 or 128 on the tensor-core path, to 32, 64 or
   // 128 on the fp32 path (zero columns of W_Q, W_K, W_V and zero rows of W_O change no result)
-  L->d.D = dtype == SH_BF16 ? (d0.Dt <= 64 ? 64 : 128) : (d0.Dt <= 32 ? 32 : d0.Dt <= 64 ? 64 : 128);
+  L->d.D = dtype == SH_BF16 ? (d0.Dt <= 64 ? 64 : 128) : (d0.Dt <= 32 ? 32 : d0.Dt <= 64 ? 64 : d0.Dt <= 128 ? 128 : 256);
   const int T = cache_len + seq;                           // tokens of a sequence the layer sees: cache, then chunk
   const long long slots = (long long)batch * T * d0.H * d0.k;
   if (slots >= (1ll << 31) || (long long)batch * T * d0.M >= (1ll << 40)) {

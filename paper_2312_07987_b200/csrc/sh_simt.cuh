@@ -435,8 +435,8 @@ template <typename TM>
 __global__ void __launch_bounds__(128)
 sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, const TM* __restrict__ V,
                          TM* __restrict__ Ahat, ShDims d, ShXlPos xl) {
-  __shared__ float s_q[4][128];
-  __shared__ float s_qv[4][128];
+  __shared__ float s_q[4][256];
+  __shared__ float s_qv[4][256];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long qi = (long)blockIdx.x * 4 + warp;          // index over (b, h, t)
   const long total = (long)d.B * d.H * d.T;
@@ -455,7 +455,7 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
     s_qv[warp][i] = Rh ? qv + xl.qscale * xl.v[hq * d.D + i] : 0.f;
   }
   __syncwarp();
-  float o[4] = {0.f, 0.f, 0.f, 0.f};                    // lane owns d = lane + 32*i
+  float o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // lane owns d = lane + 32*i (d_head up to 256)
   float m = -INFINITY, l = 0.f;
   const int last = d.causal ? t : d.T - 1;              // last visible key
   for (int s0 = 0; s0 <= last; s0 += 32) {
@@ -485,13 +485,13 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
     l = l * alpha + ps;
     m = mn;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) o[i] *= alpha;
+    for (int i = 0; i < 8; ++i) o[i] *= alpha;
     const int cnt = min(32, last - s0 + 1);
     for (int j = 0; j < cnt; ++j) {
       const float pj = __shfl_sync(0xffffffffu, p, j);
       const TM* vr = Vb + (long)(s0 + j) * d.D;
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 8; ++i)
         if (lane + 32 * i < d.D) o[i] = fmaf(pj, sh_to_float<TM>(vr[lane + 32 * i]), o[i]);
     }
   }
@@ -499,7 +499,7 @@ sh_simt_attention_kernel(const TM* __restrict__ Q, const TM* __restrict__ K, con
   TM* dst = Ahat + (((long)b * d.T + t) * d.H + h) * d.D;
   const float inv = 1.f / l;
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 8; ++i)
     if (lane + 32 * i < d.D) dst[lane + 32 * i] = sh_from_float<TM>(o[i] * inv);
 }
 

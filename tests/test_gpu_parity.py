@@ -257,6 +257,18 @@ def test_padded_d_head(dtype, D, T):
     full_check(inputs.make_inputs(cfg))
 
 
+@pytest.mark.parametrize("D,T", [(132, 70), (168, 40), (256, 33)])
+def test_d_head_above_128_in_the_fp32_configuration(D, T):
+    # the paper's 262M Wikitext-103 model (d_head 132) and its MAC-matched models (168); bf16 storage stops at 128
+    cfg = inputs.LayerConfig("dbig", inputs.DTYPE_F32, 2, T, 128, 2, D, 4, 2, seed=80 + D)
+    full_check(inputs.make_inputs(cfg))
+    L = binding.Layer(256, 2, D, 4, 2)
+    with pytest.raises(binding.SwitchHeadError) as e:
+        L.sh_configure(binding.SH_BF16, 1, 64)
+    assert "up to 128" in str(e.value)
+    L.close()
+
+
 def test_padded_d_head_with_rope_and_shared_selection():
     cfg = inputs.LayerConfig("dpad_rope", inputs.DTYPE_BF16, 2, 300, 256, 2, 100, 5, 3, seed=88)
     rope_check(inputs.make_inputs(cfg))
