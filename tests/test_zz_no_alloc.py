@@ -46,6 +46,13 @@ def test_noalloc_gate_topk_matches_regular_entry_point_twice(name, batch, gate_t
         assert (rg - gg).abs().max().item() <= gate_tol, "gate values differ"
         assert torch.equal(ref[2], got[2]), "offsets differ"
         assert torch.equal(ref[3], got[3]), "token lists differ"
+    # and against the fp64 oracle directly (selections, gates, offsets, lists of the unpermuted tokens)
+    from tests import parity_util as pu
+    got = binding.sh_noalloc_gate_topk(cfg.dtype, x0.reshape(-1, M), wg, None, H, E, k)
+    torch.cuda.synchronize()
+    want = pu.oracle_selection(inp)
+    pu.check_selection(got[0].cpu().numpy(), got[1].cpu().numpy(), want, x0.shape[0] * x0.shape[1], max(gate_tol, 1e-6))
+    pu.check_lists(got[2].cpu().numpy(), got[3].cpu().numpy(), want)
     layer.close()
 
 
