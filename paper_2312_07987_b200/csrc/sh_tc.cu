@@ -9,6 +9,7 @@
 #include "sh_tc_gemm.cuh"
 #include "sh_tc_pgemm.cuh"
 #include "sh_tc_attn2.cuh"
+#include "sh_tc_attn3.cuh"
 #include "sh_tc_gate.cuh"
 #include "sh_tc_oproj2.cuh"
 #include "sh_tc_qkpair.cuh"
@@ -576,12 +577,20 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     const int nq = ((d.T + 127) / 128 - d.Tc / 128 + 1) / 2;    // pairs of 128-query tiles behind the cache
     const unsigned grid = (unsigned)(nq * d.B * d.H);
     a.balanced = d.causal && (int)grid <= L->sm_count && S->attn_balanced;
+    // up to 1024 keys per query tile: the kernel that pipelines the 128 keys of a step as two halves (its
+    // finer hand-overs shorten the few-step chain of a short sequence); beyond: the whole-S kernel
+    // (with halves the issuing thread, eight N = 64 UMMAs per half, bounds a long loop)
+    const bool halves = d.T <= 1024;
     if (d.D == 128) {
-      if ((rc = set_smem(sh_tc_attention2_kernel<128>, Attn2Smem<128>::TOTAL))) return rc;
-      if ((rc = launch_k(pdl, sh_tc_attention2_kernel<128>, dim3(grid), dim3(320), Attn2Smem<128>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
+      auto kern = halves ? sh_tc_attention3_kernel<128> : sh_tc_attention2_kernel<128>;
+      const int smem = halves ? Attn3Smem<128>::TOTAL : Attn2Smem<128>::TOTAL;
+      if ((rc = set_smem(kern, smem))) return rc;
+      if ((rc = launch_k(pdl, kern, dim3(grid), dim3(320), smem, st, S->map_q, S->map_k, S->map_v, a))) return rc;
     } else {
-      if ((rc = set_smem(sh_tc_attention2_kernel<64>, Attn2Smem<64>::TOTAL))) return rc;
-      if ((rc = launch_k(pdl, sh_tc_attention2_kernel<64>, dim3(grid), dim3(320), Attn2Smem<64>::TOTAL, st, S->map_q, S->map_k, S->map_v, a))) return rc;
+      auto kern = halves ? sh_tc_attention3_kernel<64> : sh_tc_attention2_kernel<64>;
+      const int smem = halves ? Attn3Smem<64>::TOTAL : Attn2Smem<64>::TOTAL;
+      if ((rc = set_smem(kern, smem))) return rc;
+      if ((rc = launch_k(pdl, kern, dim3(grid), dim3(320), smem, st, S->map_q, S->map_k, S->map_v, a))) return rc;
     }
     L->launches += 1;
   }
