@@ -436,6 +436,11 @@ def main():
             cx = dataclasses.replace(cfg, name="c4_262m_bf16+cache", seq=2 * cfg.seq)
             ix = inputs.make_inputs(cx, enforce_gap=False)
             lx = binding.layer_from_inputs(ix, cache_len=cfg.seq)
+            # relative positions as in Transformer-XL: random projection and bias vectors of the trained model's shapes
+            rg = np.random.Generator(np.random.PCG64(103))
+            Wr = torch.from_numpy((rg.standard_normal((cfg.n_heads, cfg.d_model, cfg.d_head)) / np.sqrt(cfg.d_model)).astype(np.float32)).cuda()
+            uu = torch.from_numpy((0.5 * rg.standard_normal((cfg.n_heads, cfg.d_head))).astype(np.float32)).cuda()
+            vv = torch.from_numpy((0.5 * rg.standard_normal((cfg.n_heads, cfg.d_head))).astype(np.float32)).cuda()
             xx = binding.to_device(ix.x, cfg.dtype)
             ox = torch.empty((cfg.batch, cfg.seq, cfg.d_model), dtype=torch.float32, device="cuda")
             stream = torch.cuda.current_stream()
@@ -456,9 +461,27 @@ def main():
                   + 2.0 * (2 * N) * cfg.n_heads * cfg.k * cfg.d_model * cfg.d_head + 2.0 * N * cfg.n_heads * cfg.k * cfg.d_head * cfg.d_model
                   + 4.0 * cfg.batch * cfg.n_heads * cfg.d_head * (cfg.seq * Tc + cfg.seq * cfg.seq / 2))
             xms = float(np.median(dt))
+            lx.sh_set_xl_positions(Wr, uu, vv)
+            for _ in range(3):
+                lx.sh_forward(xx, ox)
+            torch.cuda.synchronize()
+            dtp = []
+            for _ in range(50):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); lx.sh_forward(xx, ox); b.record(stream)
+                torch.cuda.synchronize()
+                dtp.append(a.elapsed_time(b))
+            assert lx.sh_last_status() == 0
+            pms = float(np.median(dtp))
+            # position term: the score-bias GEMM Q R^T over the visible distances (causal part counted as for attention)
+            fpos = 2.0 * cfg.batch * cfg.n_heads * cfg.d_head * (cfg.seq * Tc + cfg.seq * cfg.seq / 2)
             line["xl_context_c2"] = {"cache_len": Tc, "chunk_tokens_per_step": N, "ms_per_step": xms,
                                      "chunk_tokens_per_s": N / (xms * 1e-3), "useful_tflops": fx / (xms * 1e-3) / 1e12,
-                                     "note": "x = [cache; chunk] per sequence, out for the chunk; scores q.k (no relative-position term)"}
+                                     "with_relative_positions": {"ms_per_step": pms, "chunk_tokens_per_s": N / (pms * 1e-3),
+                                                                 "useful_tflops": (fx + fpos) / (pms * 1e-3) / 1e12},
+                                     "note": "x = [cache; chunk] per sequence, out for the chunk; first figure: scores q.k; "
+                                             "second: with Transformer-XL's relative-position term (the paper's main configuration)"}
             lx.close()
         if not args.no_cpu_baseline:
             v, nseq, secs = oracle_sample(cfg, m["inp"], rope_base=args.rope if args.rope > 0 else None,

@@ -106,7 +106,7 @@ int sh_configure(sh_layer* layer, int dtype, int batch, int seq);
  * which sees the whole cache and the chunk up to itself.  out is [B, seq, d_model].
  * bf16 storage: cache_len and seq must be multiples of 128 (else SH_ERR_UNSUPPORTED).
  * Scores are q.k / sqrt(d_head) unless sh_set_xl_positions adds Transformer-XL's relative-position
- * term (fp32 configuration).  sh_set_rope is refused for a layer with a cache; sh_gate_topk and the debug
+ * term.  sh_set_rope is refused for a layer with a cache; sh_gate_topk and the debug
  * buffers cover all cache_len + seq tokens.  cache_len = 0 is sh_configure. */
 int sh_configure_xl(sh_layer* layer, int dtype, int batch, int seq, int cache_len);
 
@@ -116,10 +116,14 @@ int sh_configure_xl(sh_layer* layer, int dtype, int batch, int seq, int cache_le
  *   r^h_dist = emb(dist) Wr^h,   emb(dist) = [sin(dist w_0..), cos(dist w_0..)], w_i = 10000^(-2i/d_model)
  * where t and s are positions in [cache; chunk] and only keys s <= t are visible.
  *   Wr [H, d_model, d_head] fp32, u, v [H, d_head] fp32 (NULL: zero).  Wr = NULL switches the term off.
- * Builds the distance table for the configured sequence length in the workspace (asynchronously
- * on `stream`); valid until the next sh_configure / sh_set_workspace.  Works with and without a
- * cache.  SH_ERR_UNSUPPORTED for bf16 storage (the tensor-core attention kernel has no position
- * term) and while rotary embeddings are on. */
+ * Builds the distance tables for the configured sequence length in the workspace (asynchronously
+ * on `stream`); valid until the next sh_configure / sh_set_workspace.  Wr, u, v are fp32 for both
+ * storage types.  fp32 configuration: with and without a cache; the CUDA-core attention kernel
+ * evaluates both terms.  bf16 storage: for a layer with a cache (sh_configure_xl, the setting of the
+ * paper's XL models; else SH_ERR_UNSUPPORTED): every pass computes u.k per key and a score bias
+ * [B, H, seq, cache_len + seq] fp16 = Q R^T (shifted from distance order to key order) + v.r + u.k
+ * with a tensor-core GEMM, and the attention kernel adds it to its score tiles.
+ * SH_ERR_UNSUPPORTED while rotary embeddings are on. */
 int sh_set_xl_positions(sh_layer* layer, const float* Wr, const float* u, const float* v, void* stream);
 
 /* Bytes of workspace sh_set_workspace needs for the current configuration (0 if not

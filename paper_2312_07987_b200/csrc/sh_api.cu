@@ -77,10 +77,18 @@ static void layout_workspace(sh_layer* L) {
   o.vearly_cnt = take(early ? (size_t)d.B * d.H * SH_EARLY_ROWS * 4 : 16);
   // fp32 configuration: Transformer-XL relative positions (sh_set_xl_positions): the embedding of the
   // distances [T, M], its projection R [H, T, D] and the two bias vectors [2, H, D]
-  const bool xlp = L->dtype == SH_F32 && !L->dense;
+  // (bf16 storage: only for a layer with a cache, the setting the paper's XL models run in; besides the
+  //  fp32 tables an fp16 copy of R, the per-distance bias v.r [H, T], the per-key bias u.k [B, H, T] and
+  //  the score bias [B, H, Tq, T] fp16 that the attention kernel adds to its S tiles)
+  const bool xlp = !L->dense && (L->dtype == SH_F32 || d.Tc > 0);
+  const bool xlb = xlp && L->dtype == SH_BF16;
   o.xl_emb = take(xlp ? (size_t)d.T * d.M * 4 : 16);
   o.xl_r = take(xlp ? (size_t)d.H * d.T * d.D * 4 : 16);
   o.xl_uv = take(xlp ? (size_t)2 * d.H * d.D * 4 : 16);
+  o.xl_r16 = take(xlb ? (size_t)d.H * d.T * d.D * 2 : 16);
+  o.xl_vr = take(xlb ? (size_t)d.H * d.T * 4 : 16);
+  o.xl_uk = take(xlb ? (size_t)d.B * d.H * d.T * 4 : 16);
+  o.xl_bias = take(xlb ? (size_t)d.B * d.H * (d.T - d.Tc) * d.T * 2 : 16);
   o.stamps = take(sizeof(ShStampBlock));
   o.total = off;
 }
@@ -408,8 +416,9 @@ extern "C" int sh_set_xl_positions(sh_layer* L, const float* Wr, const float* u,
   if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
   if (L->dtype < 0 || !L->ws) { sh_set_error("sh_set_xl_positions needs a configured layer with its workspace"); return SH_ERR_NOT_CONFIGURED; }
   if (!Wr) { L->xl_positions = false; return SH_OK; }
-  if (L->dtype != SH_F32 || L->dense) {
-    sh_set_error("the relative-position term is built for the fp32 configuration of a SwitchHead layer only");
+  if (L->dense) { sh_set_error("the dense comparator has no relative positions"); return SH_ERR_UNSUPPORTED; }
+  if (L->dtype == SH_BF16 && L->d.Tc == 0) {
+    sh_set_error("bf16 storage: the relative-position term needs a layer configured with a cache (sh_configure_xl, cache_len >= 128)");
     return SH_ERR_UNSUPPORTED;
   }
   if (L->rope) { sh_set_error("rotary embeddings are switched on: one positional encoding at a time"); return SH_ERR_UNSUPPORTED; }
@@ -427,6 +436,12 @@ extern "C" int sh_set_xl_positions(sh_layer* L, const float* Wr, const float* u,
   SH_CUDA_CHECK(cudaMemsetAsync(uv, 0, (size_t)2 * d.H * d.D * 4, st));
   if (u) SH_CUDA_CHECK(cudaMemcpy2DAsync(uv, (size_t)d.D * 4, u, (size_t)d.Dt * 4, (size_t)d.Dt * 4, d.H, cudaMemcpyDeviceToDevice, st));
   if (v) SH_CUDA_CHECK(cudaMemcpy2DAsync(uv + (size_t)d.H * d.D, (size_t)d.D * 4, v, (size_t)d.Dt * 4, (size_t)d.Dt * 4, d.H, cudaMemcpyDeviceToDevice, st));
+  if (L->dtype == SH_BF16) {
+    // tensor-core path: R as fp16 (the B operand of the score-bias GEMM) and the per-distance term c * v . r
+    const float qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+    sh_xl_tables16_kernel<<<(unsigned)((nr + 255) / 256), 256, 0, st>>>(R, uv + (size_t)d.H * d.D, (__half*)(L->ws + L->o.xl_r16),
+                                                                       (float*)(L->ws + L->o.xl_vr), d.H, d.T, d.D, qscale);
+  }
   SH_CUDA_CHECK(cudaGetLastError());
   L->xl_positions = true;
   return SH_OK;

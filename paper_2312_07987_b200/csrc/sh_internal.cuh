@@ -79,7 +79,7 @@ __device__ __forceinline__ void sh_stamp_end(unsigned long long* s, int k) { if 
 
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, stamps, total;
+         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, stamps, total;
 };
 
 // Words of the 256-byte status block at the start of the workspace.
@@ -94,7 +94,7 @@ enum {
 
 #define SH_GUARD_BYTES 256
 #define SH_GUARD_BYTE 0xC5u
-#define SH_MAX_GUARDS 32
+#define SH_MAX_GUARDS 40
 
 struct sh_layer {
   ShDims d{};

@@ -530,3 +530,35 @@ static __global__ void sh_xl_project_kernel(const float* __restrict__ emb, const
     for (int m = 0; m < M; ++m) acc += (double)emb[(size_t)dist * M + m] * (double)Wr[((size_t)h * M + m) * Dt + dd];
   R[i] = (float)acc;
 }
+
+// Tensor-core path: R16[h, dist, :] = fp16(R[h, dist, :]) and vr[h, dist] = c * v^h . R[h, dist, :]
+// (one thread per element of R; the dot product by the thread of element dd == 0).
+static __global__ void sh_xl_tables16_kernel(const float* __restrict__ R, const float* __restrict__ v, __half* __restrict__ R16,
+                                             float* __restrict__ vr, int H, int T, int D, float c) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long)H * T * D) return;
+  R16[i] = __float2half_rn(R[i]);
+  if (i % D == 0) {
+    const int h = (int)(i / ((long)D * T));
+    double acc = 0.0;
+    for (int dd = 0; dd < D; ++dd) acc += (double)v[h * D + dd] * (double)R[i + dd];
+    vr[i / D] = c * (float)acc;
+  }
+}
+
+// Per-key content bias of the Transformer-XL score: uk[b, h, s] = c * u^h . K[b, h, s, :]  (K fp16 [B, H, T, D]); one warp per key.
+static __global__ void __launch_bounds__(256)
+sh_xl_uk_kernel(const __half* __restrict__ K, const float* __restrict__ u, float* __restrict__ uk, int H, int T, int D, long nkeys, float c) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const long w = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= nkeys) return;
+  const int h = (int)((w / T) % H);
+  const __half* kr = K + w * D;
+  float acc = 0.f;
+  for (int i = lane; i < D; i += 32) acc = fmaf(u[h * D + i], __half2float(kr[i]), acc);
+#pragma unroll
+  for (int x = 16; x > 0; x >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, x);
+  if (lane == 0) uk[w] = c * acc;
+}

@@ -13,6 +13,7 @@
 #include "sh_tc_gate.cuh"
 #include "sh_tc_oproj2.cuh"
 #include "sh_tc_qkpair.cuh"
+#include "sh_tc_xlbias.cuh"
 
 using namespace shtc;
 
@@ -77,6 +78,7 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
   CUtensorMap map_wqk, map_wqk128, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
+  CUtensorMap map_q2d, map_r16;  // score-bias GEMM of the Transformer-XL position term: Q as [B*H*T, D], R16 as [H*T, D]
   CUtensorMap map_x;             // tensor map of the last x pointer seen (x_cached)
   const void* x_cached = nullptr;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel (more than 256 gate columns)
@@ -259,6 +261,10 @@ int sh_tc_prepare(sh_layer* L) {
   if ((rc = encode_3d_f16(&S->map_k, ws + L->o.k, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = encode_3d_f16(&S->map_v, ws + L->o.v, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = sh_tc_encode_2d(&S->map_ahat, 1, ws + L->o.ahat, HD, d.N, (uint64_t)HD * 2, 64, 128))) return rc;
+  if (!L->dense && d.Tc > 0) {
+    if ((rc = sh_tc_encode_2d(&S->map_q2d, 1, ws + L->o.q, d.D, (uint64_t)d.B * d.H * d.T, (uint64_t)d.D * 2, 64, 128))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_r16, 1, ws + L->o.xl_r16, d.D, (uint64_t)d.H * d.T, (uint64_t)d.D * 2, 64, 128))) return rc;
+  }
   return SH_OK;
 }
 
@@ -574,6 +580,29 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
   } else {
     TcAttnArgs a{};
     a.d = d; a.ahat = (__half*)(ws + L->o.ahat); a.status = status;
+    if (L->xl_positions) {
+      // Transformer-XL position term: the per-key content bias c u.k, then the score bias
+      // [B, H, Tq, T] = Q R^T (skewed to key order) + c v.r + c u.k by a tensor-core GEMM; the attention
+      // kernel adds it to its S tiles
+      const float qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+      const long nkeys = (long)d.B * d.H * d.T;
+      if ((rc = launch_k(false, sh_xl_uk_kernel, dim3((unsigned)((nkeys * 32 + 255) / 256)), dim3(256), 0, st, (const __half*)(ws + L->o.k),
+                         (const float*)(ws + L->o.xl_uv), (float*)(ws + L->o.xl_uk), d.H, d.T, d.D, nkeys, qscale)))
+        return rc;
+      TcXlBiasArgs bg{};
+      bg.d = d; bg.vr = (const float*)(ws + L->o.xl_vr); bg.uk = (const float*)(ws + L->o.xl_uk);
+      bg.bias = (__half*)(ws + L->o.xl_bias); bg.status = status;
+      const unsigned bgrid = (unsigned)(d.B * d.H * ((d.T - d.Tc) / 128));
+      if (d.D == 128) {
+        if ((rc = set_smem(sh_tc_xlbias_kernel<128>, XlBiasSmem<128>::TOTAL))) return rc;
+        if ((rc = launch_k(pdl, sh_tc_xlbias_kernel<128>, dim3(bgrid), dim3(320), XlBiasSmem<128>::TOTAL, st, S->map_q2d, S->map_r16, bg))) return rc;
+      } else {
+        if ((rc = set_smem(sh_tc_xlbias_kernel<64>, XlBiasSmem<64>::TOTAL))) return rc;
+        if ((rc = launch_k(pdl, sh_tc_xlbias_kernel<64>, dim3(bgrid), dim3(320), XlBiasSmem<64>::TOTAL, st, S->map_q2d, S->map_r16, bg))) return rc;
+      }
+      L->launches += 2;
+      a.bias = (const __half*)(ws + L->o.xl_bias);
+    }
     const int nq = ((d.T + 127) / 128 - d.Tc / 128 + 1) / 2;    // pairs of 128-query tiles behind the cache
     const unsigned grid = (unsigned)(nq * d.B * d.H);
     a.balanced = d.causal && (int)grid <= L->sm_count && S->attn_balanced;

@@ -27,7 +27,24 @@ struct TcAttnArgs {
   __half* ahat;          // [B*T, H, D]
   int* status;
   int balanced;          // pair query tile p with tile ntile-1-p (causal mask, grid fits the GPU in one wave)
+  const __half* bias;    // [B, H, T - Tc, T] added to the scores (Transformer-XL position and content-bias terms, log2 units), or nullptr
 };
+
+// Adds 64 or 128 consecutive bias values (fp16, 16-byte aligned run of this query row) to the scores in sv.
+template <int N>
+__device__ __forceinline__ void add_score_bias(uint32_t* sv, const __half* run) {
+#pragma unroll
+  for (int i = 0; i < N / 8; ++i) {
+    const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(run) + i);
+    const __half2* h2 = reinterpret_cast<const __half2*>(&b4);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float2 f = __half22float2(h2[u]);
+      sv[8 * i + 2 * u] = __float_as_uint(__uint_as_float(sv[8 * i + 2 * u]) + f.x);
+      sv[8 * i + 2 * u + 1] = __float_as_uint(__uint_as_float(sv[8 * i + 2 * u + 1]) + f.y);
+    }
+  }
+}
 
 template <int D>
 struct Attn2Smem {
@@ -190,6 +207,8 @@ sh_tc_attention2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s + lane_off + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
       tmem_ld_wait();
+      if (g.bias && qrow[t] + r < d.T)
+        add_score_bias<128>(sv, g.bias + ((size_t)bh * (d.T - d.Tc) + (qrow[t] - d.Tc + r)) * d.T + j * 128);
       if (j == n - 1) {
         // last tile: the diagonal one (key c visible iff c <= r), or without the causal mask the
         // tile that holds the end of the sequence (keys past it were zero-filled by the loads)

@@ -201,6 +201,8 @@ sh_tc_attention3_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         tmem_ld32(tmem_s + lane_off, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
         tmem_ld32(tmem_s + lane_off + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
         tmem_ld_wait();
+        if (g.bias && qrow[t] + r < d.T)
+          add_score_bias<64>(sv, g.bias + ((size_t)bh * (d.T - d.Tc) + (qrow[t] - d.Tc + r)) * d.T + j * 128 + 64 * x);
         if (j == n - 1) {
           // last tile: the diagonal one (key c visible iff c <= r), or without the causal mask the
           // tile that holds the end of the sequence (keys past it were zero-filled by the loads)

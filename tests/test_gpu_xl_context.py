@@ -131,10 +131,46 @@ def test_xl_relative_positions_f32(T, Tc, B, E, k, H, D, M):
     layer.close()
 
 
-def test_xl_relative_positions_are_refused_for_bf16():
+@pytest.mark.parametrize("T,Tc,B,E,k,H,D,M", [(128, 128, 2, 4, 2, 2, 64, 256), (256, 256, 2, 5, 3, 2, 64, 512),
+                                                (384, 128, 1, 4, 2, 3, 128, 384), (128, 512, 1, 16, 4, 2, 128, 256),
+                                                (1024, 1024, 1, 4, 2, 1, 128, 256)])   # the last: 2048 keys, the whole-S attention kernel
+def test_xl_relative_positions_bf16(T, Tc, B, E, k, H, D, M):
+    """The paper's main configuration on the tensor-core path: cache + Transformer-XL position term (score bias
+    = Q R^T skewed to key order + v.r + u.k, added to the S tiles by the attention kernel)."""
+    cfg = inputs.LayerConfig("xl_pos16", inputs.DTYPE_BF16, B, Tc + T, M, H, D, E, k, seed=700 + T)
+    inp = inputs.make_inputs(cfg)
+    rng = np.random.default_rng(701)
+    Wr = (rng.standard_normal((H, M, D)) / np.sqrt(M)).astype(np.float32)
+    u = (0.5 * rng.standard_normal((H, D))).astype(np.float32)
+    v = (0.5 * rng.standard_normal((H, D))).astype(np.float32)
+    layer = binding.layer_from_inputs(inp, cache_len=Tc)
+    x = binding.to_device(inp.x, cfg.dtype)
+    y_plain = layer.sh_forward(x).clone()
+    layer.sh_set_xl_positions(*(torch.from_numpy(a).cuda() for a in (Wr, u, v)))
+    y = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0
+    ref = switchhead_xl_forward(inp.x[:, Tc:], inp.x[:, :Tc], inp.Wq, inp.Wk, inp.Wv, inp.Wo, inp.Ws, inp.Wd,
+                                cfg.k, inp.bias_s, inp.bias_d, Wr=Wr, u=u, v=v)
+    err = pu.rel_rms_err(y.cpu().numpy(), ref["y"])
+    assert err < pu.TOL_Y[cfg.dtype], f"output max-abs error / rms = {err:.3e}"
+    A = layer.sh_debug_buffer("AHAT").float().cpu().numpy().astype(np.float64).reshape(B, cfg.seq, H, D)[:, Tc:]
+    tola = 1e-2 * (np.abs(ref["Ahat"]) + 2 * np.sqrt((ref["Ahat"] ** 2).mean()))
+    assert not (np.abs(A - ref["Ahat"]) > tola).any(), "Ahat differs"
+    assert not torch.allclose(y, y_plain, rtol=1e-2, atol=1e-2), "the position term changed nothing"
+    layer.sh_set_xl_positions(None)
+    y_off = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    if cfg.k <= 2:
+        assert torch.equal(y_off, y_plain)
+    layer.sh_check_guards()
+    layer.close()
+
+
+def test_xl_relative_positions_bf16_need_a_cache():
     L = binding.Layer(256, 2, 64, 4, 2)
     L.sh_configure(binding.SH_BF16, 1, 128)
     with pytest.raises(binding.SwitchHeadError) as e:
         L.sh_set_xl_positions(torch.zeros((2, 256, 64), device="cuda"))
-    assert "fp32" in str(e.value)
+    assert "cache" in str(e.value)
     L.close()
