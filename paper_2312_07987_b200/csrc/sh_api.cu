@@ -89,6 +89,8 @@ static void layout_workspace(sh_layer* L) {
   o.xl_vr = take(xlb ? (size_t)d.H * d.T * 4 : 16);
   o.xl_uk = take(xlb ? (size_t)d.B * d.H * d.T * 4 : 16);
   o.xl_bias = take(xlb ? (size_t)d.B * d.H * (d.T - d.Tc) * d.T * 2 : 16);
+  // W_O once more with the experts innermost on the contraction axis: [H, M, D*E] (sparse output projection)
+  o.wos = take(sh_o_sparse_ok(L) ? HD * d.E * d.M * mid : 16);
   o.stamps = take(sizeof(ShStampBlock));
   o.total = off;
 }
@@ -248,6 +250,12 @@ static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void
     // Wv [H, E, M, D] -> [H, E, D, M];  Wo [H, E, D, M] -> [H, E, M, D]
     repack<TI, TI>(Wv, ws + L->o.wv, d.H * d.E, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
     repack<TI, TM>(Wo, ws + L->o.wo, d.H * d.E, d.Dt, d.M, (long)d.D * d.M, d.D, 1, st);
+    if (sh_o_sparse_ok(L)) {
+      // Wo [H, E, D, M] -> [H, M, D*E]: element (h, e, dd, m) at (h*M + m)*(D*E) + dd*E + e
+      if (d.D != d.Dt) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wos, 0, (size_t)HD * d.E * d.M * sizeof(TM), st));
+      for (int h = 0; h < d.H; ++h)
+        repack<TI, TM>((const TI*)Wo + (size_t)h * d.E * d.Dt * d.M, (TM*)(ws + L->o.wos) + (size_t)h * d.M * d.D * d.E, d.E, d.Dt, d.M, 1, (long)d.D * d.E, d.E, st);
+    }
   }
   SH_CUDA_CHECK(cudaGetLastError());
   return SH_OK;

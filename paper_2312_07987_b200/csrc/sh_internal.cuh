@@ -79,7 +79,7 @@ __device__ __forceinline__ void sh_stamp_end(unsigned long long* s, int k) { if 
 
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, stamps, total;
+         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, stamps, total;
 };
 
 // Words of the 256-byte status block at the start of the workspace.
@@ -113,6 +113,14 @@ struct sh_layer {
   size_t guard_off[SH_MAX_GUARDS] = {};   // byte offsets of the guards behind the workspace sub-buffers
   int n_guards = 0;
 };
+
+// Shapes the sparse output projection (sh_tc_oproj_sp_kernel) serves: with at most two selections out of
+// every four neighbouring experts a token's gate-scaled rows are 2:4 sparse along an expert-innermost
+// contraction axis.  The layer then keeps a second, expert-interleaved copy of W_O in the workspace.
+inline bool sh_o_sparse_ok(const sh_layer* L) {
+  const ShDims& d = L->d;
+  return L->dtype == SH_BF16 && !L->dense && d.k <= 2 && (d.E == 4 || d.E == 8) && d.D == 128 && d.H <= 4;
+}
 
 template <typename T> __device__ __forceinline__ float sh_to_float(T v);
 template <> __device__ __forceinline__ float sh_to_float<float>(float v) { return v; }

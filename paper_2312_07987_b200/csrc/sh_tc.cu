@@ -14,6 +14,7 @@
 #include "sh_tc_oproj2.cuh"
 #include "sh_tc_qkpair.cuh"
 #include "sh_tc_xlbias.cuh"
+#include "sh_tc_oproj_sp.cuh"
 
 using namespace shtc;
 
@@ -77,7 +78,7 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
-  CUtensorMap map_wqk, map_wqk128, map_wv, map_wo, map_wo256, map_ahat, map_wgate;
+  CUtensorMap map_wqk, map_wqk128, map_wv, map_wo, map_wo256, map_wos, map_ahat, map_wgate;
   CUtensorMap map_q2d, map_r16;  // score-bias GEMM of the Transformer-XL position term: Q as [B*H*T, D], R16 as [H*T, D]
   CUtensorMap map_x;             // tensor map of the last x pointer seen (x_cached)
   const void* x_cached = nullptr;
@@ -94,6 +95,7 @@ struct TcState {
   bool qk_two_grids = true; // ... as two grids around the gate kernel
   bool qk_pair = true;      // CTA-pair Q/K kernel (else single-CTA persistent)
   bool o_pair = true;       // CTA-pair output projection for k <= 3 (else single-CTA)
+  bool o_sparse = true;     // sparse-A CTA-pair output projection where the shape allows (sh_o_sparse_ok)
   bool persistent = true;   // persistent Q/K and value-expert GEMMs (else one CTA per tile)
   bool fused_sort = true;   // sort fused into the gate kernel when it needs at most half of the SMs
   bool attn_balanced = true;
@@ -207,6 +209,7 @@ int sh_tc_prepare(sh_layer* L) {
   S->qk_two_grids = !getenv("SH_QK_ONE_GRID");
   S->qk_pair = !getenv("SH_QK_SINGLE");
   S->o_pair = !getenv("SH_O_SINGLE");
+  S->o_sparse = !getenv("SH_O_MASKED");
   S->persistent = !getenv("SH_NO_PERSISTENT");
   S->fused_sort = !getenv("SH_SORT_SEPARATE");
   S->attn_balanced = !getenv("SH_ATTN_ADJACENT");
@@ -249,6 +252,7 @@ int sh_tc_prepare(sh_layer* L) {
     if ((rc = sh_tc_encode_2d(&S->map_wv, 0, ws + L->o.wv, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 128))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo256, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 256))) return rc;
+    if (sh_o_sparse_ok(L) && (rc = sh_tc_encode_2d(&S->map_wos, 1, ws + L->o.wos, (uint64_t)d.D * d.E, (uint64_t)d.H * d.M, (uint64_t)d.D * d.E * 2, 64, 128))) return rc;
   } else {
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, HD, d.M, (uint64_t)HD * 2, 64, 128))) return rc;
   }
@@ -638,7 +642,17 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     // selections from shared memory and multiplies by the gate after the UMMA; a device that cannot
     // hold a two-CTA cluster of the pair kernel's size uses it too.
     bool pair = S->o_pair && d.k <= 3;
-    if (pair) {
+    const bool sparse = pair && S->o_sparse && sh_o_sparse_ok(L);
+    if (sparse) {
+      constexpr int psm = OprojSpSmem<128>::TOTAL;
+      if (d.E == 4) { if ((rc = set_smem(sh_tc_oproj_sp_kernel<128, 1>, psm))) return rc; }
+      else if ((rc = set_smem(sh_tc_oproj_sp_kernel<128, 2>, psm))) return rc;
+      if (S->o_pairs_max == 0) {
+        S->o_pairs_max = d.E == 4 ? max_pairs(sh_tc_oproj_sp_kernel<128, 1>, 480, psm) : max_pairs(sh_tc_oproj_sp_kernel<128, 2>, 480, psm);
+        if (S->o_pairs_max <= 0) S->o_pairs_max = -1;
+      }
+      if (S->o_pairs_max < 0) pair = false;
+    } else if (pair) {
       const int psm = d.D == 128 ? OprojPairSmem<128>::TOTAL : OprojPairSmem<64>::TOTAL;
       if (d.D == 128) { if ((rc = set_smem(sh_tc_oproj_pair_kernel<128>, psm))) return rc; }
       else if ((rc = set_smem(sh_tc_oproj_pair_kernel<64>, psm))) return rc;
@@ -648,7 +662,16 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
       }
       if (S->o_pairs_max < 0) pair = false;
     }
-    if (pair) {
+    if (pair && sparse) {
+      // 256 tokens x 256 features per unit, the selection as 2:4 sparsity of the gate-scaled A operand
+      constexpr int psm = OprojSpSmem<128>::TOTAL;
+      a.nwork = ((sh_out_rows(d) + 255) / 256) * ((d.M + 255) / 256);
+      const unsigned pgrid = 2u * (unsigned)(a.nwork < S->o_pairs_max ? a.nwork : S->o_pairs_max);
+      const __half* ahat = (const __half*)(ws + L->o.ahat);
+      if (d.E == 4) rc = launch_k_pairs(pdl, sh_tc_oproj_sp_kernel<128, 1>, dim3(pgrid), dim3(480), psm, st, S->map_wos, a, ahat);
+      else rc = launch_k_pairs(pdl, sh_tc_oproj_sp_kernel<128, 2>, dim3(pgrid), dim3(480), psm, st, S->map_wos, a, ahat);
+      if (rc) return rc;
+    } else if (pair) {
       // 256 tokens x 256 features per unit, gates folded into the A operand
       const int psm = d.D == 128 ? OprojPairSmem<128>::TOTAL : OprojPairSmem<64>::TOTAL;
       a.nwork = ((sh_out_rows(d) + 255) / 256) * ((d.M + 255) / 256);
