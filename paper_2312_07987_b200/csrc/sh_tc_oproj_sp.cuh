@@ -95,6 +95,10 @@ sh_tc_oproj_sp_kernel(const __grid_constant__ CUtensorMap mapWos, TcOprojArgs g,
   constexpr int SPH = 2 * SPT;                           // ring stages per head
   constexpr int WPH = 8 * SPT;                           // weight blocks per head (E * D / 64)
   static_assert(WST <= 8 && PST <= 4 && WST > 4, "barrier slots / ring step");
+  // A builder group skips the other group's SPT stages of every head: from its last stage of one head to
+  // its first of the next it moves SPT + 1 stages on.  With fewer ring slots than that it could arrive two
+  // phases ahead of a slot's empty barrier, and a parity wait cannot tell phase p from phase p - 2.
+  static_assert(PST >= SPT + 1, "ring depth against the builders' stride");
   constexpr uint32_t TBLK = 128 * 128;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;

@@ -33,6 +33,10 @@ def main(case: str) -> None:
             tp.full_check(inputs.make_inputs(inputs.LayerConfig("edge_bf16_wide", inputs.DTYPE_BF16, B, T, M, H, D, E, k, seed=300 + T)))
         for cfg in tp._random_bf16_configs(4, 11):
             tp.full_check(inputs.make_inputs(cfg), check_stage_buffers=False)
+    elif case == "sparse_o":
+        # the shapes the 2:4-sparse output projection serves (or, with SH_O_MASKED, the masked kernel on them)
+        for cfg in tp.SPARSE_O_CONFIGS:
+            tp.full_check(inputs.make_inputs(cfg), check_stage_buffers=False)
     elif case == "index_selftest":
         inp = inputs.make_inputs(inputs.CONFIGS["small_bf16"], batch=1)
         layer = binding.layer_from_inputs(inp)

@@ -277,6 +277,25 @@ def test_padded_d_head_with_rope_and_shared_selection():
     rope_check(inputs.make_inputs(cfg))
 
 
+# Shapes of the 2:4-sparse output projection (k <= 2, E = 4 or 8, stored d_head 128, at most 4 heads): one
+# selection only (the second kept position of a group is padding), two selections in one group of four
+# or one in each (E = 8), padded d_head, token counts and d_model that leave CTA pairs and feature
+# chunks ragged, several work units per CTA pair (the position codes move between the two accumulators)
+SPARSE_O_CONFIGS = [
+    inputs.LayerConfig("sp_e4k1", inputs.DTYPE_BF16, 2, 150, 384, 2, 128, 4, 1, seed=401),
+    inputs.LayerConfig("sp_e8k1", inputs.DTYPE_BF16, 1, 300, 256, 3, 128, 8, 1, seed=402),
+    inputs.LayerConfig("sp_e8k2_pad", inputs.DTYPE_BF16, 3, 200, 640, 3, 100, 8, 2, seed=403, zipf_bias=1.2),
+    inputs.LayerConfig("sp_e4k2_h1", inputs.DTYPE_BF16, 1, 100, 128, 1, 128, 4, 2, seed=404),
+    inputs.LayerConfig("sp_e4k2_units", inputs.DTYPE_BF16, 40, 512, 2048, 4, 128, 4, 2, seed=405),
+    inputs.LayerConfig("sp_e8k2_units", inputs.DTYPE_BF16, 24, 1000, 1536, 2, 128, 8, 2, seed=406, zipf_bias=1.2),
+]
+
+
+@pytest.mark.parametrize("cfg", SPARSE_O_CONFIGS, ids=lambda c: c.name)
+def test_sparse_output_projection_shapes(cfg):
+    full_check(inputs.make_inputs(cfg), check_stage_buffers=False, batches=[0, cfg.batch - 1] if cfg.batch > 3 else None)
+
+
 def test_pair_output_projection_ragged_tokens_and_features():
     # CTA-pair output projection: N = 300 is not a multiple of the pair's 256 tokens (the second CTA of
     # the last pair owns 44 tokens, and with N = 100 none at all), d_model = 384 or 128 not of its 256 features
