@@ -245,8 +245,13 @@ def roofline_from_timeline(cfg, tl, fl, peaks):
                 traffic=None if traffic is None else traffic * 1e6, traffic_unit="bytes per launch (ncu)")
     if dom == "o":
         # the on-chip sum multiplies every token tile by all E experts of a head (zero rows for the
-        # tokens that did not select one): executed tensor work = E/k times the useful work counted here
+        # tokens that did not select one): logical tensor work = E/k times the useful work counted here;
+        # where the selection is 2:4 sparse along the expert-innermost contraction axis (k <= 2, E = 4
+        # or 8, d_head 128, <= 4 heads) the sparse instruction does that product in half the cycles
+        sparse = cfg.k <= 2 and cfg.n_experts in (4, 8) and 64 < cfg.d_head <= 128 and cfg.n_heads <= 4
         roof["executed_over_useful_flop"] = cfg.n_experts / cfg.k
+        roof["tensor_cycles_over_useful"] = cfg.n_experts / cfg.k / (2 if sparse else 1)
+        roof["o_kernel"] = "2:4-sparse CTA-pair kernel" if sparse else "masked kernel"
     return roof
 
 

@@ -62,9 +62,12 @@ static void layout_workspace(sh_layer* L) {
   const size_t slots = (size_t)2 * d.N * d.H * d.k;
   o.idx = take(slots * 4);
   o.gate = take(slots * 4);
-  o.blockcnt = take((size_t)d.nblk * d.G * 4);
-  o.blockoff = take((size_t)d.nblk * d.G * 4);
-  o.offsets = take((size_t)2 * d.H * (d.E + 1) * 4);
+  // (a layer whose value projection is tiled by expert pairs sorts H * E(E-1)/2 buckets in a forward pass)
+  const bool vp = sh_v_pairs_ok(L);
+  const size_t hist = vp && d.H * sh_pair_count(d.E) > d.G ? (size_t)d.H * sh_pair_count(d.E) : (size_t)d.G;
+  o.blockcnt = take((size_t)d.nblk * hist * 4);
+  o.blockoff = take((size_t)d.nblk * hist * 4);
+  o.offsets = take(((size_t)2 * d.H * (d.E + 1) + (vp ? (size_t)d.H * (sh_pair_count(d.E) + 1) : 0)) * 4);
   o.lists = take(slots * 4);
   o.lgate = take(slots * 4);
   o.tiles = take((size_t)2 * d.max_tiles * sizeof(ShTile));
@@ -91,6 +94,7 @@ static void layout_workspace(sh_layer* L) {
   o.xl_bias = take(xlb ? (size_t)d.B * d.H * (d.T - d.Tc) * d.T * 2 : 16);
   // W_O once more with the experts innermost on the contraction axis: [H, M, D*E] (sparse output projection)
   o.wos = take(sh_o_sparse_ok(L) ? HD * d.E * d.M * mid : 16);
+  o.gid = take(vp ? (size_t)d.N * d.H * 4 : 16);      // pair number of every (token, head), source side
   o.stamps = take(sizeof(ShStampBlock));
   o.total = off;
 }
@@ -163,7 +167,7 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
   L->dtype = dtype;
   L->d.B = batch; L->d.T = T; L->d.Tc = cache_len; L->d.N = batch * T;
   L->d.nblk = (L->d.N + SH_TILE_ROWS - 1) / SH_TILE_ROWS;
-  L->d.max_tiles = (int)((slots + SH_TILE_ROWS - 1) / SH_TILE_ROWS) + d0.H * d0.E;
+  L->d.max_tiles = (int)((slots + SH_TILE_ROWS - 1) / SH_TILE_ROWS) + d0.H * d0.E + d0.H * sh_pair_count(d0.E > 8 ? 2 : d0.E);
   L->d.tile_rows_src = SH_TILE_ROWS;
   // (k >= 3: the fp16 reductions of a value row arrive in a different order from run to run - two
   //  passes have been seen 1e-2 of the output RMS apart; with the first rows, which reach the output

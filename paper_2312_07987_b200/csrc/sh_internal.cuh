@@ -31,6 +31,16 @@ struct ShDims {
   int* status;             // the status block at the start of the workspace (nullptr: the allocation-free gate entry point)
 };
 
+// Unordered pairs {a < b} of E experts, numbered row by row: (0,1), (0,2), ..., (0,E-1), (1,2), ...
+// (the value projection of a k = 2 layer is tiled by (head, pair): sh_tc_vpair_kernel).
+__host__ __device__ __forceinline__ int sh_pair_count(int E) { return E * (E - 1) / 2; }
+__host__ __device__ __forceinline__ int sh_pair_id(int a, int b, int E) { return a * (2 * E - a - 1) / 2 + (b - a - 1); }
+__host__ __device__ __forceinline__ void sh_pair_decode(int id, int E, int& a, int& b) {
+  a = 0;
+  while (a < E - 2 && id >= E - 1 - a) { id -= E - 1 - a; ++a; }
+  b = a + 1 + id;
+}
+
 // With a cache in front of every sequence (ShDims::Tc): the row of `out` that belongs to context token
 // `tok` (-1 for a cache token), and the context token of an out row.
 __host__ __device__ __forceinline__ int sh_out_row(const ShDims& d, int tok) {
@@ -79,7 +89,7 @@ __device__ __forceinline__ void sh_stamp_end(unsigned long long* s, int k) { if 
 
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, stamps, total;
+         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, gid, stamps, total;
 };
 
 // Words of the 256-byte status block at the start of the workspace.
@@ -120,6 +130,13 @@ struct sh_layer {
 inline bool sh_o_sparse_ok(const sh_layer* L) {
   const ShDims& d = L->d;
   return L->dtype == SH_BF16 && !L->dense && d.k <= 2 && (d.E == 4 || d.E == 8) && d.D == 128 && d.H <= 4;
+}
+
+// Shapes whose value projection is tiled by (head, pair of selected experts) instead of (head, expert):
+// k = 2, so every (token, head) belongs to exactly one pair; few enough pairs for the sort's 32-bit masks.
+inline bool sh_v_pairs_ok(const sh_layer* L) {
+  const ShDims& d = L->d;
+  return L->dtype == SH_BF16 && !L->dense && d.k == 2 && d.E >= 2 && d.E <= 8 && d.D == 128;
 }
 
 template <typename T> __device__ __forceinline__ float sh_to_float(T v);

@@ -120,6 +120,7 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
   const int tok0 = blk * SH_TILE_ROWS;
   const int nrows = min(SH_TILE_ROWS, d.N - tok0);
   for (int i = tid; i < 2 * nb; i += nthreads) s_pre[i] = 0;   // s_pre and s_tot
+  for (int i = tid; i < 4 * nb; i += nthreads) s_wcnt[i] = 0;  // (k = 1: only the buckets a warp meets are written)
   // bucket b = tid % nb; the thread sums the blocks part, part + parts, ... in registers.  These
   // loads do not depend on the selections copy below, so both are in flight together.
   int my_b = -1, my_tot = 0, my_pre = 0;
@@ -129,7 +130,7 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
       if (tid / nb < parts) {
         my_b = tid % nb;
         const int part = tid / nb;
-#pragma unroll 4
+#pragma unroll 8
         for (int bk = part; bk < d.nblk; bk += parts) {
           const int c = blockcnt[(size_t)bk * nb + my_b];
           my_tot += c;
@@ -169,7 +170,18 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
       run += s_tot[g * d.E + e];
     }
   }
-  for (int grp = gs; grp < d.sides * d.H; grp += GS) {            // per-warp counts of this block's tokens
+  // One entry per (token, group) (k = 1: also the (head, expert pair) buckets of the pair-tiled value
+  // projection, which can be many): the lanes of a warp that share a bucket find each other with
+  // match.any instead of one ballot per bucket.
+  const bool one_sel = d.k == 1;
+  for (int grp = gs; one_sel && grp < d.sides * d.H; grp += GS) {
+    const int side = grp / d.H, h = grp % d.H;
+    int ev = tl < nrows ? s_idx[side * 128 * per_tok + tl * d.H + h] : -1;
+    if (ev >= 0 && !SH_INDEX_OK(ev, d.E, d.status, SH_SITE_SORT_EXPERT)) ev = -1;
+    const unsigned m = __match_any_sync(0xffffffffu, ev >= 0 ? ev : 0x10000 + lane);
+    if (ev >= 0 && lane == __ffs(m) - 1) s_wcnt[(grp * d.E + ev) * 4 + twarp] = __popc(m);
+  }
+  for (int grp = gs; !one_sel && grp < d.sides * d.H; grp += GS) {            // per-warp counts of this block's tokens
     const int side = grp / d.H, h = grp % d.H;
     unsigned mask = 0;
     if (tl < nrows)
@@ -185,7 +197,24 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
   sync();
   {
     const int t = tok0 + tl;
-    for (int grp = gs; grp < d.sides * d.H; grp += GS) {
+    for (int grp = gs; one_sel && grp < d.sides * d.H; grp += GS) {
+      const int side = grp / d.H, h = grp % d.H;
+      const int sel = side * 128 * per_tok + tl * d.H + h;
+      int ev = tl < nrows ? s_idx[sel] : -1;
+      if ((unsigned)ev >= (unsigned)d.E) ev = -1;
+      const unsigned m = __match_any_sync(0xffffffffu, ev >= 0 ? ev : 0x10000 + lane);
+      if (ev >= 0) {
+        const int b = grp * d.E + ev;
+        int pos = __popc(m & ((1u << lane) - 1u));
+        for (int w = 0; w < twarp; ++w) pos += s_wcnt[b * 4 + w];
+        const size_t dst = (size_t)grp * d.N + s_off[b] + s_pre[b] + pos;
+        if (SH_INDEX_OK(s_off[b] + s_pre[b] + pos, (long long)d.N, d.status, SH_SITE_SORT_SLOT)) {
+          lists[dst] = t;
+          lgate[dst] = s_gt[sel];
+        }
+      }
+    }
+    for (int grp = gs; !one_sel && grp < d.sides * d.H; grp += GS) {
       const int side = grp / d.H, h = grp % d.H;
       const int sel = side * 128 * per_tok + (tl * d.H + h) * d.k;
       unsigned mask = 0;
@@ -269,6 +298,9 @@ static inline int sh_sort_threads(const ShDims& d) {
   // at most 512 threads (16 K registers), so that a block fits beside a 320-thread GEMM CTA on an SM
   int gs = d.sides * d.H;
   if (gs > 4) gs = 4;
+  // (the histogram prefix is shared out over all threads - bucket by bucket, block range by block range -
+  //  and is a chain of L2 round trips: with many buckets or blocks, more threads than token slices pay)
+  if ((long)d.G * d.nblk > 2048 && gs < 4) gs = 4;
   return 128 * gs;
 }
 

@@ -15,6 +15,7 @@
 #include "sh_tc_qkpair.cuh"
 #include "sh_tc_xlbias.cuh"
 #include "sh_tc_oproj_sp.cuh"
+#include "sh_tc_vpair.cuh"
 
 using namespace shtc;
 
@@ -95,6 +96,8 @@ struct TcState {
   bool qk_two_grids = true; // ... as two grids around the gate kernel
   bool qk_pair = true;      // CTA-pair Q/K kernel (else single-CTA persistent)
   bool o_pair = true;       // CTA-pair output projection for k <= 3 (else single-CTA)
+  bool v_pairs = true;      // value projection tiled by (head, expert pair) on CTA pairs where the shape allows (sh_v_pairs_ok)
+  int v_pairs_max = 0;      // clusters of that kernel the device holds at once (0: not asked yet, -1: none)
   bool o_sparse = true;     // sparse-A CTA-pair output projection where the shape allows (sh_o_sparse_ok)
   bool persistent = true;   // persistent Q/K and value-expert GEMMs (else one CTA per tile)
   bool fused_sort = true;   // sort fused into the gate kernel when it needs at most half of the SMs
@@ -210,6 +213,7 @@ int sh_tc_prepare(sh_layer* L) {
   S->qk_pair = !getenv("SH_QK_SINGLE");
   S->o_pair = !getenv("SH_O_SINGLE");
   S->o_sparse = !getenv("SH_O_MASKED");
+  S->v_pairs = !getenv("SH_V_BY_EXPERT");
   S->persistent = !getenv("SH_NO_PERSISTENT");
   S->fused_sort = !getenv("SH_SORT_SEPARATE");
   S->attn_balanced = !getenv("SH_ATTN_ADJACENT");
@@ -287,11 +291,27 @@ static int x_map(sh_layer* L, const void* x, const CUtensorMap** out) {
 
 // The gate kernel's x stream comes cold from HBM (~1.2 us per box round trip), so what bounds its
 // main loop is the bytes in flight per CTA: 8 stages when they fit, else 4.
-static int gate_smem_bytes(int Gp, int G, int stages) {
+static int gate_smem_bytes(int Gp, int G, int stages) {   // G: histogram width (gate columns, or (head, pair) buckets if more)
   const int stage = 128 * 64 * 2 + ((Gp * 128 + 1023) & ~1023);
   const int pipe = stages * stage, stag = 128 * (Gp + 1) * 4;
   const int bar_off = ((pipe > stag ? pipe : stag) + 1023) & ~1023;
   return bar_off + 256 + 3 * G * 4 + 1024;
+}
+
+using VPS = VPairSmem<6>;
+// Forward passes of a k = 2 layer tile the value projection by (head, pair of selected experts): the gate
+// kernel then buckets the source side by pair, and sh_tc_vpair_kernel replaces the expert-tiled kernel.
+static bool use_v_pairs(sh_layer* L) {
+  TcState* S = (TcState*)L->tc;
+  if (!S->v_pairs || !sh_v_pairs_ok(L) || !S->gate_gp || (S->simt_mask & (SH_STAGE_GATE | SH_STAGE_V))) return false;
+  if (S->v_pairs_max == 0) {
+    if (set_smem(sh_tc_vpair_kernel<6>, VPS::TOTAL) != SH_OK) S->v_pairs_max = -1;
+    else {
+      S->v_pairs_max = max_pairs(sh_tc_vpair_kernel<6>, 320, VPS::TOTAL);
+      if (S->v_pairs_max <= 0) S->v_pairs_max = -1;
+    }
+  }
+  return S->v_pairs_max > 0;
 }
 
 // Gate + top-k + bucket sort.  With zero_for_forward the gate kernel also clears the value buffer.
@@ -316,13 +336,16 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.d = d; g.Gp = S->gate_gp; g.gbias = (const float*)(ws + L->o.gbias);
   g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
   g.blockcnt = (int*)(ws + L->o.blockcnt);
-  g.zero_v = zero_for_forward ? (void*)(ws + L->o.v) : nullptr;
+  const bool vp = zero_for_forward && use_v_pairs(L);
+  g.vpairs = vp; g.NP = sh_pair_count(d.E); g.GH = vp ? d.H * g.NP : d.G; g.gid = (int*)(ws + L->o.gid);
+  const int GHmax = g.GH > d.G ? g.GH : d.G;
+  g.zero_v = (zero_for_forward && !vp) ? (void*)(ws + L->o.v) : nullptr;    // (the pair-tiled kernel stores every value row once)
   g.zero_out = (zero_for_forward && (S->simt_mask & SH_STAGE_O) && d.Tc == 0) ? (float*)out : nullptr;
   if (zero_for_forward && (S->simt_mask & SH_STAGE_O) && d.Tc > 0)          // (out has fewer rows than there are tokens)
     SH_CUDA_CHECK(cudaMemsetAsync(out, 0, (size_t)sh_out_rows(d) * d.M * 4, st));
   g.status = (int*)(ws + L->o.status);
-  const bool deep = gate_smem_bytes(S->gate_gp, d.G, 8) <= 200 * 1024;
-  const int smem = gate_smem_bytes(S->gate_gp, d.G, deep ? 8 : 4);
+  const bool deep = gate_smem_bytes(S->gate_gp, GHmax, 8) <= 200 * 1024;
+  const int smem = gate_smem_bytes(S->gate_gp, GHmax, deep ? 8 : 4);
   if ((rc = deep ? set_smem(sh_tc_gate_kernel<8>, smem) : set_smem(sh_tc_gate_kernel<4>, smem))) return rc;
   // In a forward pass only the value experts read sorted lists (the output projection works from
   // idx / gate, token tile by token tile), so only the source side is sorted there -- unless the
@@ -330,6 +353,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   // sort's loops run over sides * H groups.
   ShDims ds = d;
   if (zero_for_forward && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
+  if (vp) { ds.sides = 1; ds.E = g.NP; ds.k = 1; ds.G = g.GH; ds.tile_rows_src = 256; }   // buckets (head, pair), one entry per (token, head)
   // Fused sort: when every CTA of the gate kernel can be resident at once (cooperative launch) and the
   // sort's scratch fits behind the logits tile in the idle operand ring, the gate kernel places the
   // tokens itself and there is no sort kernel.  Used when the gate kernel needs at most half of the SMs:
@@ -338,7 +362,8 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   {
     const int stage = 128 * 64 * 2 + ((S->gate_gp * 128 + 1023) & ~1023);
     const int pipe = (deep ? 8 : 4) * stage, stag = 128 * (S->gate_gp + 1) * 4;
-    g.fused = S->fused_sort && 2 * d.nblk <= L->sm_count && ((stag + 15) & ~15) + (int)sh_sort_smem_bytes(d) <= pipe;
+    const int sort_bytes = (int)(sh_sort_smem_bytes(d) > sh_sort_smem_bytes(ds) ? sh_sort_smem_bytes(d) : sh_sort_smem_bytes(ds));
+    g.fused = S->fused_sort && 2 * d.nblk <= L->sm_count && ((stag + 15) & ~15) + sort_bytes <= pipe;
     if (g.fused && S->gate_coop == 0) {
       int dev = 0, coop = 0, per_sm = 0;
       SH_CUDA_CHECK(cudaGetDevice(&dev));
@@ -349,7 +374,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
     }
     if (S->gate_coop < 0) g.fused = 0;
   }
-  g.sort_sides = ds.sides; g.tile_rows_src = d.tile_rows_src; g.max_tiles = d.max_tiles;
+  g.sort_sides = ds.sides; g.tile_rows_src = ds.tile_rows_src; g.max_tiles = d.max_tiles;
   g.offsets = (int*)(ws + L->o.offsets); g.lists = (int*)(ws + L->o.lists); g.lgate = (float*)(ws + L->o.lgate);
   g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
   g.gridbar = (int*)(ws + L->o.status) + SH_ST_GRIDBAR;
@@ -367,14 +392,14 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   }
   if (deep) sh_tc_gate_kernel<8><<<d.nblk, GATE_THREADS, smem, st>>>(*map_x, S->map_wgate, g);
   else sh_tc_gate_kernel<4><<<d.nblk, GATE_THREADS, smem, st>>>(*map_x, S->map_wgate, g);
-  size_t ssm = sh_sort_smem_bytes(d);
+  size_t ssm = sh_sort_smem_bytes(ds);
   // sort_apart: ask for enough shared memory that a sort block fits beside a gate CTA but not beside a
   // ~198 KB GEMM CTA: next to the Q/K projection's CTAs (whose waiting warps poll) a block takes
   // 11 us instead of 4.7
   if (sort_apart && ssm < 40 * 1024) ssm = 40 * 1024;
   if ((rc = set_smem(sh_sort_kernel, (int)ssm))) return rc;
   if ((rc = launch_k(S->pdl && !L->ev, sh_sort_kernel, dim3(d.nblk), dim3(sh_sort_threads(ds)), ssm, st,
-                     (const int*)(ws + L->o.idx), (const float*)(ws + L->o.gate), (const int*)(ws + L->o.blockcnt),
+                     (const int*)(ws + (vp ? L->o.gid : L->o.idx)), (const float*)(ws + L->o.gate), (const int*)(ws + L->o.blockcnt),
                      (int*)(ws + L->o.offsets), (int*)(ws + L->o.lists), (float*)(ws + L->o.lgate),
                      (ShTile*)(ws + L->o.tiles), (int*)(ws + L->o.ntiles), ds)))
     return rc;
@@ -552,6 +577,16 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
   if (!L->dense) {
     if (simt & SH_STAGE_V) {
       if ((rc = sh_simt_run_bf16(L, SH_STAGE_V, x, out, st))) return rc;
+    } else if (use_v_pairs(L)) {
+      TcVPairArgs g{};
+      g.d = d; g.x = x; g.lists = (const int*)(ws + L->o.lists);
+      g.tiles = (const ShTile*)(ws + L->o.tiles); g.ntiles = (const int*)(ws + L->o.ntiles);
+      g.idx = (const int*)(ws + L->o.idx); g.gate = (const float*)(ws + L->o.gate);
+      g.v = (__half*)(ws + L->o.v); g.status = status;
+      const int bound = (d.N * d.H + 255) / 256 + d.H * sh_pair_count(d.E);       // tiles: at most this many
+      const unsigned pgrid = 2u * (unsigned)(bound < S->v_pairs_max ? bound : S->v_pairs_max);
+      if ((rc = launch_k_pairs(pdl, sh_tc_vpair_kernel<6>, dim3(pgrid), dim3(320), VPS::TOTAL, st, S->map_wv, g))) return rc;
+      L->launches += 1;
     } else {
       TcGemmArgs g{};
       g.d = d; g.K = d.M; g.ncols = d.D;

@@ -59,6 +59,7 @@ sh_tc_attention3_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   uint64_t* p_full = bars + 13;   // [2][2]: P_x of the step is in TMEM (one arrival per softmax warp)
   uint64_t* pv_done = bars + 17;  // [2] per query tile: one more P V product has completed (two per step)
   uint32_t* tmem_slot = (uint32_t*)(bars + 19);
+  uint64_t* o_done = bars + 20;   // [2] per query tile: its last product has completed (one phase per launch)
 
   const ShDims& d = g.d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -91,6 +92,7 @@ sh_tc_attention3_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
       mbar_init(&pv_done[i], 1);
+      mbar_init(&o_done[i], 1);
     }
     for (int i = 0; i < 4; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); }
     fence_barrier_init();
@@ -170,6 +172,7 @@ sh_tc_attention3_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
               umma_f16_tmem_a(tmem + 256 + t * 128, tmem + t * 128 + x * 64 + 8 * k, desc_pack(v_lo + (4 * x + k) * (2048 >> 4)), idesc_pv,
                               (j | x | k) != 0);
             umma_commit(&pv_done[t]);
+            if (x == 1 && j == nt[t] - 1) umma_commit(&o_done[t]);   // the tile's O is final when this completes
             // the half's next S goes right behind: executed in issue order, it overwrites P_x only after
             // the product above has read it
             if (j + 1 < nt[t]) issue_s(t, x, j + 1);
@@ -264,9 +267,11 @@ sh_tc_attention3_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         if (lane == 0) mbar_arrive(&p_full[t * 2 + x]);
       }
     }
-    // the last two products of the tile, one after the other: a parity wait cannot tell a phase from the
-    // one two before it, and only the product before these two is known to be complete here
-    if (ok && n > 0 && mbar_wait(&pv_done[t], (2 * n - 2) & 1, g.status, dead) && mbar_wait(&pv_done[t], (2 * n - 1) & 1, g.status, dead)) {
+    // The tile's last product.  (Not a parity wait on pv_done: after its last arrival on p_full a warp
+    // can be late - the tail below is cold code - and find BOTH of the last two products complete; a
+    // parity wait for the first of them would then wait for a phase that never comes.  Seen as a 1 s
+    // time-out once in ~500 passes at T = 512 with 160 (batch, head) pairs.)
+    if (ok && n > 0 && mbar_wait(&o_done[t], 0, g.status, dead)) {
       tc_fence_after();
       const int tq = qrow[t] + r;
       const float inv = 1.f / l;

@@ -39,6 +39,13 @@ struct TcGateArgs {
   int max_tiles;
   int* offsets; int* lists; float* lgate; ShTile* tiles; int* ntiles;
   int* gridbar;              // {arrived, departed}, both 0 between launches
+  // value projection tiled by expert PAIRS (k = 2, forward pass only): the source side is bucketed by
+  // (head, pair number) - histogram, sort and tile table run over H * NP buckets with one entry per
+  // (token, head) - and the destination side is not bucketed at all
+  int vpairs;                // 0 / 1
+  int NP;                    // pairs per head: E (E - 1) / 2
+  int GH;                    // histogram width: vpairs ? H * NP : G
+  int* gid;                  // [N, H] pair number of every (token, head)
 };
 
 constexpr int GATE_THREADS = 608;
@@ -77,7 +84,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     fence_barrier_init();
     tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapW);
   }
-  for (int i = threadIdx.x; i < d.G; i += blockDim.x) s_hist[i] = 0;
+  for (int i = threadIdx.x; i < g.GH; i += blockDim.x) s_hist[i] = 0;
   if (warp == 1) { tmem_alloc(tmem_slot, tmem_cols); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
@@ -178,8 +185,8 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     // fused sort: its scratch sits behind the logits rows; the selections go there as well
     int* s_sort = reinterpret_cast<int*>(sgen + ((stag_bytes + 15) & ~15));
     const int per_tok = d.H * d.k;
-    int* s_idx = s_sort + 8 * d.G;                        // [2][128 * per_tok], as sh_sort_block lays it out
-    float* s_gt = reinterpret_cast<float*>(s_idx + 2 * 128 * per_tok);
+    int* s_idx = s_sort + 8 * g.GH;                       // [2][128 * per_tok], as sh_sort_block lays it out
+    float* s_gt = reinterpret_cast<float*>(s_idx + 2 * 128 * per_tok);     // (pair mode: [128 * H] pair numbers; gates unused)
     const bool sel_ok = mbar_wait(logits_ready, 0, g.status, dead);
     if (sel_ok) {
       const int r = et & 127, sub = et >> 7;
@@ -191,6 +198,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
           const int side = grp / d.H, h = grp % d.H;
           const size_t o = (((size_t)side * d.N + t) * d.H + h) * d.k;
           unsigned taken = 0;
+          int first = 0;
           for (int j = 0; j < d.k; ++j) {
             int best = -1;
             float bz = 0.f;
@@ -203,6 +211,16 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const float gv = 1.f / (1.f + expf(-bz));
             g.idx[o + j] = best;
             g.gate[o + j] = gv;
+            if (g.vpairs) {
+              if (j == 0) first = best;
+              else if (side == 0) {
+                const int pid = sh_pair_id(min(first, best), max(first, best), d.E);
+                g.gid[(size_t)t * d.H + h] = pid;
+                if (g.fused) s_idx[r * d.H + h] = pid;
+                atomicAdd(&s_hist[h * g.NP + pid], 1);
+              }
+              continue;
+            }
             if (g.fused) {
               s_idx[side * 128 * per_tok + (r * d.H + h) * d.k + j] = best;
               s_gt[side * 128 * per_tok + (r * d.H + h) * d.k + j] = gv;
@@ -216,10 +234,10 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       // ---- publish the histogram, meet the other CTAs, place this CTA's tokens ----------------------
       auto sel_sync = [] { asm volatile("bar.sync 1, 512;" ::: "memory"); };
       sel_sync();                                           // s_hist, s_idx, s_gt complete
-      for (int i = et; i < d.G; i += NSEL) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
+      for (int i = et; i < g.GH; i += NSEL) g.blockcnt[(size_t)blockIdx.x * g.GH + i] = s_hist[i];
       __threadfence();
       sel_sync();
-      int* s_flag = s_hist + d.G;                           // (the histogram area is 3 G words)
+      int* s_flag = s_hist + g.GH;                          // (the histogram area is 3 GH words)
       if (et == 0) {
         bool ok = sel_ok;
         atomicAdd(g.gridbar, 1);
@@ -239,6 +257,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       if (*(volatile int*)s_flag) {
         ShDims ds = d;
         ds.sides = g.sort_sides;
+        if (g.vpairs) { ds.sides = 1; ds.E = g.NP; ds.k = 1; ds.G = g.GH; }   // buckets (head, pair), one entry per (token, head)
         sh_sort_block(g.idx, g.gate, g.blockcnt, g.offsets, g.lists, g.lgate, g.tiles, g.ntiles, ds, s_sort, et, NSEL, (int)blockIdx.x, true, sel_sync);
       }
     }
@@ -251,7 +270,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
   }
   // ---- publish this CTA's selection histogram (the sort kernel scans them) ------------------
   if (!g.fused)
-    for (int i = threadIdx.x; i < d.G; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * d.G + i] = s_hist[i];
+    for (int i = threadIdx.x; i < g.GH; i += blockDim.x) g.blockcnt[(size_t)blockIdx.x * g.GH + i] = s_hist[i];
   if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_GATE);
 }
 

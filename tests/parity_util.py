@@ -67,7 +67,7 @@ def run_layer(inp, device="cuda", shared_selection=False):
     x = binding.to_device(inp.x, cfg.dtype, device)
     y = layer.sh_forward(x)
     torch.cuda.synchronize()
-    assert layer.sh_last_status() == 0, "device status word reports a failed kernel"
+    assert layer.sh_last_status() == 0, f"device status word reports a failed kernel: status block {layer.sh_status_block()}"
     return layer, x, y
 
 

@@ -23,7 +23,7 @@ def run_case(case, extra_env=None):
 
 
 @pytest.mark.parametrize("env", [{}, {"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
-                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_O_MASKED": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"},
+                                 {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_O_MASKED": "1"}, {"SH_V_BY_EXPERT": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"},
                                  {"SH_SORT_SEPARATE": "1"}, {"SH_SIMT_STAGES": "31"}],
                          ids=lambda e: "+".join(sorted(e)) or "default")
 def test_launch_structure_switches_keep_the_result(env):
@@ -33,6 +33,7 @@ def test_launch_structure_switches_keep_the_result(env):
 def test_sparse_output_projection_shapes_with_index_checks_and_against_the_masked_kernel():
     run_case("sparse_o")
     run_case("sparse_o", {"SH_O_MASKED": "1"})
+    run_case("sparse_o", {"SH_V_BY_EXPERT": "1"})
 
 
 def test_index_checks_stay_silent_on_edge_shapes():

@@ -323,6 +323,28 @@ def test_back_to_back_forward_passes_share_the_tile_counter_cleanly():
     layer.close()
 
 
+def test_many_passes_of_a_multi_wave_shape_stay_clean_and_identical():
+    # 160 (batch, head) pairs at T = 512: the attention grid takes more than two waves, the gate kernel two,
+    # the sort runs as a kernel of its own.  A late softmax warp once found both of its tile's last two
+    # products complete and waited for a barrier phase that never came (one pass in ~500): every pass
+    # must leave the status word clear and, k = 2, give the same bits.
+    cfg = inputs.LayerConfig("multi_wave", inputs.DTYPE_BF16, 40, 512, 2048, 4, 128, 4, 2, seed=405)
+    inp = inputs.make_inputs(cfg, enforce_gap=False)
+    layer = binding.layer_from_inputs(inp)
+    x = binding.to_device(inp.x, cfg.dtype)
+    out = torch.empty(inp.x.shape, dtype=torch.float32, device="cuda")
+    first = None
+    for i in range(600):
+        layer.sh_forward(x, out)
+        torch.cuda.synchronize()
+        assert layer.sh_last_status() == 0, f"pass {i}: status block {layer.sh_status_block()}"
+        if first is None:
+            first = out.clone()
+        else:
+            assert torch.equal(out, first), f"pass {i}: output differs by {float((out - first).abs().max())}"
+    layer.close()
+
+
 def _random_bf16_configs(n, seed):
     # seeded draws over the shape space the bf16 path accepts: ragged token counts (tile tails, a CTA
     # pair whose second half is empty), d_model any multiple of 128, both stored head widths and
