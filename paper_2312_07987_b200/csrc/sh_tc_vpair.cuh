@@ -25,6 +25,10 @@
 
 namespace shtc {
 
+#ifndef VPAIR_LAG
+#define VPAIR_LAG 2                                        // gather rounds in flight per thread before it waits for the oldest
+#endif
+
 struct TcVPairArgs {
   ShDims d;
   const void* x;             // [N, M] bf16
@@ -175,8 +179,8 @@ sh_tc_vpair_kernel(const __grid_constant__ CUtensorMap mapW, TcVPairArgs g) {
           cp_async_16(sa + (rb + 16 * i) * 128 + dsw, src[i] + (long)kb * 128, ok[i]);
         cp_async_commit();
         ++issued;
-        if (issued - n_arr > 2) {                          // the copies of the stage issued two rounds ago have landed
-          cp_async_wait<2>();
+        if (issued - n_arr > VPAIR_LAG) {                  // the copies of the stage issued VPAIR_LAG rounds ago have landed
+          cp_async_wait<VPAIR_LAG>();
           landed();
         }
         if (++s == STAGES) { s = 0; par ^= 1; }
