@@ -595,19 +595,31 @@ static __global__ void sh_xl_tables16_kernel(const float* __restrict__ R, const 
   }
 }
 
-// Per-key content bias of the Transformer-XL score: uk[b, h, s] = c * u^h . K[b, h, s, :]  (K fp16 [B, H, T, D]); one warp per key.
+// Per-key content bias of the Transformer-XL score: uk[b, h, s] = c * u^h . K[b, h, s, :]  (K fp16 [B, H, T, D],
+// D a multiple of 64); eight lanes per key, 16-byte loads (a warp reads four keys' rows at a time).
 static __global__ void __launch_bounds__(256)
 sh_xl_uk_kernel(const __half* __restrict__ K, const float* __restrict__ u, float* __restrict__ uk, int H, int T, int D, long nkeys, float c) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const long w = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (w >= nkeys) return;
-  const int h = (int)((w / T) % H);
-  const __half* kr = K + w * D;
+  const long key = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
+  const int sub = threadIdx.x & 7;
   float acc = 0.f;
-  for (int i = lane; i < D; i += 32) acc = fmaf(u[h * D + i], __half2float(kr[i]), acc);
+  if (key < nkeys) {
+    const int h = (int)((key / T) % H);
+    const uint4* kr = reinterpret_cast<const uint4*>(K + key * D);
+    const float* uh = u + h * D;
+    for (int i = sub; i < D / 8; i += 8) {                 // 16-byte chunk i of the row: 8 values
+      const uint4 v = __ldg(kr + i);
+      const __half2* hv = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
-  for (int x = 16; x > 0; x >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, x);
-  if (lane == 0) uk[w] = c * acc;
+      for (int q = 0; q < 4; ++q) {
+        const float2 f = __half22float2(hv[q]);
+        acc = fmaf(uh[8 * i + 2 * q], f.x, acc);
+        acc = fmaf(uh[8 * i + 2 * q + 1], f.y, acc);
+      }
+    }
+  }
+#pragma unroll
+  for (int x = 4; x > 0; x >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, x);
+  if (sub == 0 && key < nkeys) uk[key] = c * acc;
 }

@@ -271,7 +271,7 @@ int sh_tc_prepare(sh_layer* L) {
   if ((rc = sh_tc_encode_2d(&S->map_ahat, 1, ws + L->o.ahat, HD, d.N, (uint64_t)HD * 2, 64, 128))) return rc;
   if (!L->dense && d.Tc > 0) {
     if ((rc = sh_tc_encode_2d(&S->map_q2d, 1, ws + L->o.q, d.D, (uint64_t)d.B * d.H * d.T, (uint64_t)d.D * 2, 64, 128))) return rc;
-    if ((rc = sh_tc_encode_2d(&S->map_r16, 1, ws + L->o.xl_r16, d.D, (uint64_t)d.H * d.T, (uint64_t)d.D * 2, 64, 128))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_r16, 1, ws + L->o.xl_r16, d.D, (uint64_t)d.H * d.T, (uint64_t)d.D * 2, 64, 64))) return rc;
   }
   return SH_OK;
 }
@@ -625,7 +625,7 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
       // kernel adds it to its S tiles
       const float qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
       const long nkeys = (long)d.B * d.H * d.T;
-      if ((rc = launch_k(false, sh_xl_uk_kernel, dim3((unsigned)((nkeys * 32 + 255) / 256)), dim3(256), 0, st, (const __half*)(ws + L->o.k),
+      if ((rc = launch_k(false, sh_xl_uk_kernel, dim3((unsigned)((nkeys * 8 + 255) / 256)), dim3(256), 0, st, (const __half*)(ws + L->o.k),
                          (const float*)(ws + L->o.xl_uv), (float*)(ws + L->o.xl_uk), d.H, d.T, d.D, nkeys, qscale)))
         return rc;
       TcXlBiasArgs bg{};

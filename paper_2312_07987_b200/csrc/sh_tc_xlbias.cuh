@@ -8,10 +8,11 @@
 // happens in the store: the 32 x 32 chunk of a warp goes through shared memory and every store
 // instruction writes 32 consecutive keys of one query row (2-byte elements, coalesced).
 //
-// CTA = (batch*head, 128-query tile of the chunk): Q tile loaded once, the distance tiles of R16[h]
-// streamed through a ring of 3 (only distances up to the tile's largest query position exist), UMMA
-// N = 128 into two alternating TMEM buffers, eight epilogue warps (two per TMEM lane quarter, two of the
-// four 32-column chunks each).
+// CTA = (batch*head, 128-query tile of the chunk): Q tile loaded once, 64-distance tiles of R16[h]
+// streamed through a ring of 2 (only distances up to the tile's largest query position exist), UMMA
+// N = 64 into two alternating TMEM buffers, eight epilogue warps (two per TMEM lane quarter, one
+// 32-column chunk each).  The epilogue is a chain of short latencies, so what helps is warps: the
+// CTA is sized (100 KB of shared memory) for two per SM.
 // Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + UMMA issuer, warps 2..9 = epilogue.
 #pragma once
 #include "sh_tc_prims.cuh"
@@ -28,22 +29,24 @@ struct TcXlBiasArgs {
 
 template <int D>
 struct XlBiasSmem {
-  static constexpr int T_BYTES = 128 * D * 2;
-  static constexpr int RST = 3;
+  static constexpr int T_BYTES = 128 * D * 2;            // the query tile
+  static constexpr int R_BYTES = 64 * D * 2;             // one tile of 64 distances
+  static constexpr int RST = 2;
   static constexpr int Q_OFF = 0;
   static constexpr int R_OFF = T_BYTES;
-  static constexpr int STG_OFF = R_OFF + RST * T_BYTES;
+  static constexpr int STG_OFF = R_OFF + RST * R_BYTES;
   static constexpr int STG_WARP = (32 * 33 + 64) * 4;   // the 32 x 32 chunk (padded rows) + the 63 u.k values it meets
   static constexpr int BAR_OFF = STG_OFF + 8 * STG_WARP;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;
 };
 
 template <int D>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(320, 2)
 sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapR, TcXlBiasArgs g) {
   using SM = XlBiasSmem<D>;
   constexpr int DB = D / 64, RST = SM::RST;
-  constexpr uint32_t BLK = 128 * 128;
+  constexpr uint32_t BLK = 128 * 128;                    // a 64-column block of the query tile
+  constexpr uint32_t RBLK = 64 * 128;                    // a 64-column block of a distance tile
   extern __shared__ unsigned char smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -60,7 +63,7 @@ sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
   const int Tq = d.T - d.Tc, tiles_q = Tq / 128;
   const int nbh = d.B * d.H;
   const int bh = blockIdx.x % nbh, it = tiles_q - 1 - blockIdx.x / nbh, h = bh % d.H;   // longest tiles (most distances) first
-  const int ncol = d.Tc / 128 + it + 1;                  // distance tiles that hold a visible distance for some row of this tile
+  const int ncol = 2 * (d.Tc / 128 + it + 1);            // 64-distance tiles that hold a visible distance for some row of this tile
   bool dead = false;
 
   if (threadIdx.x == 0) {
@@ -70,7 +73,7 @@ sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     fence_barrier_init();
     tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapR);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 256); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_slot, 128); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -86,14 +89,14 @@ sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       for (int ct = 0; ct < ncol; ++ct) {
         const int s = ct % RST;
         if (!mbar_wait(&r_empty[s], ((ct / RST) & 1) ^ 1, g.status, dead)) break;
-        mbar_expect_tx(&r_full[s], SM::T_BYTES);
+        mbar_expect_tx(&r_full[s], SM::R_BYTES);
 #pragma unroll
-        for (int c = 0; c < DB; ++c) tma_load_2d(sbase + SM::R_OFF + s * SM::T_BYTES + c * BLK, &mapR, &r_full[s], c * 64, h * d.T + ct * 128);
+        for (int c = 0; c < DB; ++c) tma_load_2d(sbase + SM::R_OFF + s * SM::R_BYTES + c * RBLK, &mapR, &r_full[s], c * 64, h * d.T + ct * 64);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_f16(128, 128, 0, 0, 0);
+      constexpr uint32_t idesc = make_idesc_f16(128, 64, 0, 0, 0);
       const uint32_t q_lo = desc_lo_k(sbase + SM::Q_OFF), r_lo0 = desc_lo_k(sbase + SM::R_OFF);
       if (mbar_wait(q_full, 0, g.status, dead)) {
         for (int ct = 0; ct < ncol; ++ct) {
@@ -101,12 +104,10 @@ sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
           if (!mbar_wait(&r_full[s], (ct / RST) & 1, g.status, dead)) break;
           if (!mbar_wait(&acc_empty[b], ((ct >> 1) & 1) ^ 1, g.status, dead)) break;
           tc_fence_after();
-          const uint32_t r_lo = r_lo0 + s * (SM::T_BYTES >> 4);
+          const uint32_t r_lo = r_lo0 + s * (SM::R_BYTES >> 4);
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t koff = (k / 4) * (BLK >> 4) + 2 * (k % 4);
-            umma_f16(tmem + b * 128, desc_pack(q_lo + koff), desc_pack(r_lo + koff), idesc, k != 0);
-          }
+          for (int k = 0; k < D / 16; ++k)
+            umma_f16(tmem + b * 64, desc_pack(q_lo + (k / 4) * (BLK >> 4) + 2 * (k % 4)), desc_pack(r_lo + (k / 4) * (RBLK >> 4) + 2 * (k % 4)), idesc, k != 0);
           umma_commit(&r_empty[s]);
           umma_commit(&acc_full[b]);
         }
@@ -126,33 +127,30 @@ sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
       const int b = ct & 1;
       if (!mbar_wait(&acc_full[b], (ct >> 1) & 1, g.status, dead)) break;
       tc_fence_after();
-#pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        const int c = half * 2 + cc;
-        const int dist0 = ct * 128 + c * 32;
+      {
+        const int dist0 = ct * 64 + half * 32;             // this warp's 32 distances of the tile
         const int s_lo = d.Tc + qi0 - dist0 - 31;          // keys this chunk meets: s_lo .. s_lo + 62
         const float vrd = vr[dist0 + lane];
         const float uk0 = (s_lo + lane >= 0) ? ukr[s_lo + lane] : 0.f;
         const float uk1 = (s_lo + 32 + lane >= 0 && s_lo + 32 + lane < d.T) ? ukr[s_lo + 32 + lane] : 0.f;
         uint32_t v[32];
-        tmem_ld32(tmem + lane_off + b * 128 + c * 32, v);
+        tmem_ld32(tmem + lane_off + b * 64 + half * 32, v);
         tmem_ld_wait();
-        if (cc == 1) {                                     // this warp's share of the accumulator is in registers
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&acc_empty[b]);
-        }
+        tc_fence_before();                                 // this warp's share of the accumulator is in registers
         __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[b]);
 #pragma unroll
         for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = __uint_as_float(v[i]);
         suk[lane] = uk0;
         suk[32 + lane] = uk1;
         __syncwarp();
+        __half* op = out_bh + ((long)qi0 * d.T + (s_lo + 31 - lane));   // row qi0 + rr, key s_lo + 31 + rr - lane: += T + 1 per row
+        const int s0 = s_lo + 31 - lane;
 #pragma unroll 8
         for (int rr = 0; rr < 32; ++rr) {
-          const int s = s_lo + 31 + rr - lane;             // the key at distance dist0 + lane from query row qi0 + rr
-          if (s >= 0) out_bh[(size_t)(qi0 + rr) * d.T + s] = __float2half_rn(stg[rr * 33 + lane] + vrd + suk[31 + rr - lane]);
+          if (s0 + rr >= 0) op[(long)rr * (d.T + 1)] = __float2half_rn(stg[rr * 33 + lane] + vrd + suk[31 + rr - lane]);
         }
+        __syncwarp();
       }
     }
   }
@@ -160,7 +158,7 @@ sh_tc_xlbias_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, 256);
+    tmem_dealloc(tmem, 128);
   }
 }
 
