@@ -247,32 +247,46 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
     for (int e = 0; e < d.E; ++e) offsets[g * (d.E + 1) + e] = s_off[g * d.E + e];
     offsets[g * (d.E + 1) + d.E] = s_off[g * d.E + d.E - 1] + s_tot[g * d.E + d.E - 1];
   }
-  // Tile table of a side: the full tiles of all buckets first, then the partial ones (one per bucket at
-  // most), so that a persistent kernel whose CTAs take tiles t, t + grid, t + 2 grid, ... gets an even
-  // share of both kinds (bucket by bucket, full and partial tiles alternate with a period that can divide
-  // the grid size).
+  // Tile table of a side.  Kernel of its own (the larger problems): the full tiles of all buckets first,
+  // then the partial ones (one per bucket at most), so that a persistent kernel whose CTAs take tiles
+  // t, t + grid, t + 2 grid, ... gets an even share of both kinds (bucket by bucket, full and partial
+  // tiles alternate with a period that can divide the grid size).  Fused into the gate kernel (small
+  // problems, where this block's tail is on the layer's critical path and every cold instruction line
+  // costs an L2 round trip): bucket by bucket, by one thread per side.
   int* s_pbase = s_wcnt;                 // [nb] index of the bucket's partial tile (the per-warp counts are done with)
-  sync();
-  if (tid < 32 * d.sides) {              // one warp per side: prefix sums over its buckets, 32 at a time
-    const int side = tid >> 5;
-    const int tr = side == 0 ? d.tile_rows_src : SH_TILE_ROWS;    // 128 or 256
-    const int sh = 31 - __clz(tr);
-    const int b_lo = side * d.H * d.E, b_hi = b_lo + d.H * d.E;
-    int run = 0;
-    for (int pass = 0; pass < 2; ++pass)                          // full tiles, then partial ones
-      for (int b0 = b_lo; b0 < b_hi; b0 += 32) {
-        const int b = b0 + lane;
-        const int v = b < b_hi ? (pass == 0 ? s_tot[b] >> sh : (int)((s_tot[b] & (tr - 1)) != 0)) : 0;
-        int inc = v;
+  if (!have_sel) {
+    sync();
+    if (tid < 32 * d.sides) {            // one warp per side: prefix sums over its buckets, 32 at a time
+      const int side = tid >> 5;
+      const int tr = side == 0 ? d.tile_rows_src : SH_TILE_ROWS;    // 128 or 256
+      const int sh = 31 - __clz(tr);
+      const int b_lo = side * d.H * d.E, b_hi = b_lo + d.H * d.E;
+      int run = 0;
+      for (int pass = 0; pass < 2; ++pass)                          // full tiles, then partial ones
+        for (int b0 = b_lo; b0 < b_hi; b0 += 32) {
+          const int b = b0 + lane;
+          const int v = b < b_hi ? (pass == 0 ? s_tot[b] >> sh : (int)((s_tot[b] & (tr - 1)) != 0)) : 0;
+          int inc = v;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int u = __shfl_up_sync(0xffffffffu, inc, o);
-          if (lane >= o) inc += u;
+          for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += u;
+          }
+          if (b < b_hi) (pass == 0 ? s_tbase : s_pbase)[b] = run + inc - v;
+          run += __shfl_sync(0xffffffffu, inc, 31);
         }
-        if (b < b_hi) (pass == 0 ? s_tbase : s_pbase)[b] = run + inc - v;
-        run += __shfl_sync(0xffffffffu, inc, 31);
-      }
-    if (lane == 0) ntiles[side] = run;
+      if (lane == 0) ntiles[side] = run;
+    }
+  } else if (tid < d.sides) {
+    const int side = tid;
+    const int tr = side == 0 ? d.tile_rows_src : SH_TILE_ROWS;
+    const int sh = 31 - __clz(tr);
+    int run = 0;
+    for (int b = side * d.H * d.E; b < (side + 1) * d.H * d.E; ++b) {
+      s_tbase[b] = run;
+      run += (s_tot[b] + tr - 1) >> sh;
+    }
+    ntiles[side] = run;
   }
   sync();
   for (int i = tid; i < d.sides * d.H * d.E * 32; i += nthreads) {   // 32 threads share a bucket's tiles
@@ -285,7 +299,7 @@ static __device__ __forceinline__ void sh_sort_block(const int* __restrict__ idx
       ShTile tl2;
       tl2.h = h; tl2.e = e; tl2.row0 = s_off[b] + ti * tr;
       tl2.nrows = min(tr, cnt - ti * tr);
-      tp[tl2.nrows == tr ? s_tbase[b] + ti : s_pbase[b]] = tl2;
+      tp[(have_sel || tl2.nrows == tr) ? s_tbase[b] + ti : s_pbase[b]] = tl2;
     }
   }
 }
