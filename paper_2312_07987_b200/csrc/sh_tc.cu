@@ -735,12 +735,21 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     }
     L->launches += 1;
   } else {
-    // dense comparator: out = Ahat W_O, one CTA per 128 x 128 tile
+    // dense comparator: out = Ahat W_O on the CTA-pair GEMM (256 x 256 tiles) when the device holds such
+    // clusters and d_model allows, else one CTA per 128 x 128 tile
     TcGemmArgs g{};
     g.d = d; g.K = HD; g.ncols = d.M; g.nrows = d.N; g.out0 = out; g.status = status;
     g.stamp_id = SH_K_O;
-    dim3 grid(d.nblk, (d.M + 127) / 128);
-    if ((rc = launch_gemm<128, 4, GEMM_PLAIN, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
+    if (S->persistent && S->qk_pair && d.M % 256 == 0 && HD % 64 == 0 && qk_pairs_max(S) > 0) {
+      g.sched = status + SH_ST_SCHED;                        // (the Q/K projection's claims of this pass are over: its last claimer put the counters back)
+      if ((rc = set_smem(sh_tc_qk_pair_kernel<6, 1>, QkPS::TOTAL))) return rc;
+      const int ptiles = ((d.N + 255) / 256) * (d.M / 256);
+      const unsigned pgrid = 2u * (unsigned)(ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max);
+      if ((rc = launch_k_pairs(pdl, sh_tc_qk_pair_kernel<6, 1>, dim3(pgrid), dim3(320), QkPS::TOTAL, st, S->map_ahat, S->map_wo, g))) return rc;
+    } else {
+      dim3 grid(d.nblk, (d.M + 127) / 128);
+      if ((rc = launch_gemm<128, 4, GEMM_PLAIN, 0, 0>(S->map_ahat, S->map_wo, g, grid, st))) return rc;
+    }
     L->launches += 1;
   }
   sh_mark(L, 5, st);

@@ -36,7 +36,9 @@ struct QkPairSmem {
   static constexpr int TOTAL = BAR_OFF + 512 + 1024;
 };
 
-template <int STAGES>
+// MODE 0: the Q/K(/V) projection (bf16 operands, epilogue above).  MODE 1: a plain product of fp16 operands
+// with an fp32 row-major result, out0[row, col] (the dense comparator's output projection).
+template <int STAGES, int MODE = 0>
 __global__ void __launch_bounds__(320, 1)
 sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, TcGemmArgs g) {
   using SM = QkPairSmem<STAGES>;
@@ -76,7 +78,9 @@ sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
-  if (threadIdx.x == 0) { sh_stamp_resident(d.stamps, g.stamp_id); sh_stamp_start(d.stamps, g.stamp_id); }
+  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, g.stamp_id);
+  if (MODE == 1) pdl_wait();                             // its A operand is the attention kernel's result
+  if (threadIdx.x == 0) sh_stamp_start(d.stamps, g.stamp_id);
   // the qi-th tile of this pair, for every role but the claimer, or -1 when there is none
   auto next_tile = [&](int qi) -> int {
     const int j = qi & (TQ - 1);
@@ -129,7 +133,7 @@ sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     }
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = make_idesc_f16(256, BN, 1, 1, 0);
+      constexpr uint32_t idesc = MODE == 0 ? make_idesc_f16(256, BN, 1, 1, 0) : make_idesc_f16(256, BN, 0, 0, 0);
       const uint32_t a_lo0 = desc_lo_k(sbase), b_lo0 = desc_lo_k(sbase + SM::A_BYTES);
       int s = 0, it = 0;
       uint32_t par = 0;
@@ -185,6 +189,13 @@ sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
           uint32_t* v = &vv[hh2 * 32];
           const int n0 = col0 + c0;
           if (!live || n0 >= g.ncols) continue;
+          if (MODE == 1) {
+            float* dstf = (float*)g.out0 + (size_t)tokn * g.ncols + n0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<uint4*>(dstf + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            continue;
+          }
           const int which = n0 / HD, hd = (n0 % HD) / d.D, dd = n0 % d.D;
           __half* dst = (__half*)(which == 0 ? g.out0 : which == 1 ? g.out1 : g.out2) +
                         (((size_t)bb * d.H + hd) * d.T + tt) * d.D + dd;
