@@ -103,9 +103,10 @@ sh_tc_attention3_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  pdl_trigger();                                         // programmatic dependent launch: the next kernel may become resident,
   if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_ATTN);
-  pdl_wait();                                            // and this one starts consuming once the kernel before it has completed
+  pdl_wait();                                            // programmatic dependent launch: consume once the kernel before this one has completed;
+  pdl_trigger();                                         // only then may the next kernel become resident: what it does ahead of ITS wait (the
+                                                         // output projection reads the selections there) sees every earlier kernel of the pass complete
   if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_ATTN);
 
   if (warp == 0) {

@@ -139,8 +139,11 @@ sh_tc_oproj_sp_kernel(const __grid_constant__ CUtensorMap mapWos, TcOprojArgs g,
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
   if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_O);
-  pdl_wait();
-  if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_O);
+  // Ahead of the wait for the attention kernel's result (this kernel is launched to become resident while
+  // that one drains) everything that does not need Ahat gets under way: the weight stream (weights are
+  // constant) and the first unit's position codes (the selections come from the gate kernel, which the
+  // attention kernel saw complete before it let this one start).  The roles that read Ahat or write out
+  // wait where they need to.
 
   if (warp == 0) {
     if (lane == 0) {
@@ -237,6 +240,8 @@ sh_tc_oproj_sp_kernel(const __grid_constant__ CUtensorMap mapWos, TcOprojArgs g,
       }
       if (++fh == d.H) { fh = 0; fw += npairs; }
     };
+    pdl_wait();                                            // Ahat is complete
+    if (bt == 0) sh_stamp_start(d.stamps, SH_K_O);
     fetch();
     const uint32_t trow = row * 128, tx = row & 7;         // 16-byte chunk j of a stage row: block j / 8, chunk (j % 8) ^ tx (128-byte swizzle)
     int gs = 0;                                            // running stage number of this pair
@@ -328,6 +333,7 @@ sh_tc_oproj_sp_kernel(const __grid_constant__ CUtensorMap mapWos, TcOprojArgs g,
       if (lane == 0) mbar_arrive_leader(&m_full[unit_no & 1]);
     };
     if (pair < g.nwork) { codes_of(pair); put_codes(1, 0); }
+    pdl_wait();                                            // (out is not written before the kernels ahead are done)
     int un = 0;
     for (int w = pair; w < g.nwork; w += npairs, ++un) {
       const int buf = un & 1;
