@@ -75,11 +75,9 @@ def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=N
             Q, K, V, selD = [], [], [], []
             for t in range(T):
                 xt = x[b][t]
-                q_t, k_t = _vecmat(xt, Wq[h]), _vecmat(xt, Wk[h])
-                if rope_base is not None:
-                    q_t, k_t = _rope_complex(q_t, t, rope_base), _rope_complex(k_t, t, rope_base)
-                Q.append(q_t)
-                K.append(k_t)
+                moe_q, moe_k = isinstance(Wq[h][0][0], list), isinstance(Wk[h][0][0], list)   # [E][M][D] instead of [M][D]
+                q_t = None if moe_q else _vecmat(xt, Wq[h])
+                k_t = None if moe_k else _vecmat(xt, Wk[h])
                 zs = _vecmat(xt, Ws[h])
                 zd = _vecmat(xt, Ws[h] if shared_selection else Wd[h])
                 if bias_s is not None:
@@ -95,6 +93,22 @@ def switchhead_forward_loops(x, Wq, Wk, Wv, Wo, Ws, Wd, k, bias_s=None, bias_d=N
                         v[d] += g * pe[d]
                 V.append(v)
                 selD.append([(e, _sigmoid(zd[e])) for e in _select(zd, k)])
+                if moe_k:                                   # key experts: the source side's selection and scores
+                    k_t = [0.0] * D
+                    for e in _select(zs, k):
+                        pe = _vecmat(xt, Wk[h][e])
+                        for d in range(D):
+                            k_t[d] += _sigmoid(zs[e]) * pe[d]
+                if moe_q:                                   # query experts: the destination side's
+                    q_t = [0.0] * D
+                    for e, g in selD[-1]:
+                        pe = _vecmat(xt, Wq[h][e])
+                        for d in range(D):
+                            q_t[d] += g * pe[d]
+                if rope_base is not None:
+                    q_t, k_t = _rope_complex(q_t, t, rope_base), _rope_complex(k_t, t, rope_base)
+                Q.append(q_t)
+                K.append(k_t)
             for t in range(T):
                 last = t if causal else T - 1
                 logits = [sum(Q[t][d] * K[s][d] for d in range(D)) / math.sqrt(D)

@@ -40,6 +40,13 @@ plain layer; one 2T pass = two T passes with the cache (with and without positio
 running means over cache + chunk; cache visible to every query, later chunk tokens to none; a
 scalar-loop writing; zero position weights = no position term; the appendix's MAC / memory table.
 
+MoE key / query projections (expert_projection; Wk or Wq given as [H, E, M, D]): the K^h and Q^h expert
+sums of Sec. 2.2, keys with the source side's selection and scores, queries with the destination
+side's.  Pins (tests/test_oracle_moe_qk_pins.py): a scalar-loop writing; identical experts = the dense
+projection times the sum of the selected gates; every expert selected with a constant gate = a dense
+projection with the summed weights; experts nobody selected do not matter, selected ones do, and the
+keys follow the SOURCE side; renumbering a side's experts; the context form against the plain layer.
+
 Pins (tests/test_oracle_pins.py): E=1 with zero gate weights equals 0.25 x textbook MHA
 (Eq. 2 and Eq. 3 forms, and torch's scaled_dot_product_attention); gate forced to 1 equals
 MHA; k=E equals the dense gate-weighted einsum; top-k equals a brute-force stable sort;
@@ -133,6 +140,20 @@ def rope_rotate(a: np.ndarray, positions: np.ndarray, base: float) -> np.ndarray
     return out
 
 
+def expert_projection(x2d, W_he, idx_h, gate_h):
+    """Gate-weighted sum of the selected experts' projections of every row (Sec. 2.2, the K^h / Q^h /
+    V^h expert sums): out[t] = sum_j gate_h[t, j] * x2d[t] @ W_he[idx_h[t, j]].
+    x2d [N, M]; W_he [E, M, D]: the experts of one head; idx_h, gate_h [N, k]."""
+    N, k = idx_h.shape
+    out = np.zeros((N, W_he.shape[2]))
+    for e in range(W_he.shape[0]):
+        for j in range(k):
+            rows = np.nonzero(idx_h[:, j] == e)[0]
+            if rows.size:
+                out[rows] += gate_h[rows, j][:, None] * (x2d[rows] @ W_he[e])
+    return out
+
+
 def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=None,
                        causal: bool = True, gate_override: Optional[float] = None,
                        return_stages: bool = True, rope_base: Optional[float] = None,
@@ -140,6 +161,11 @@ def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=No
     """Forward pass of one SwitchHead layer in fp64.
 
     x [B, T, M]; Wq, Wk [H, M, D]; Wv [H, E, M, D]; Wo [H, E, D, M]; Ws, Wd [H, M, E].
+    MoE key / query projections (the paper's Sec. 2.2 writes the key and query expert sums like the
+    value one; its ablation over which projections are experts): Wk [H, E, M, D] makes the keys
+    K^h[t] = sum_{e in E_S^h(t)} s_S^h[t,e] x[t] W_K^{h,e} (source-side selection, like the values);
+    Wq [H, E, M, D] makes the queries Q^h[t] = sum_{e in E_D^h(t)} s_D^h[t,e] x[t] W_Q^{h,e}
+    (destination-side selection, like the output).
     gate_override: if given, every selected expert's gate is replaced by this constant
     (used only to pin the E=1 case to plain multi-head attention).
     shared_selection: the "Shared Selection" variant of the paper's appendix: one gate serves
@@ -169,8 +195,8 @@ def switchhead_forward(x, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None, bias_d=No
     K = np.empty((N, H, D))
     V = np.zeros((N, H, D))
     for h in range(H):
-        Q[:, h, :] = x2d @ Wq[h]
-        K[:, h, :] = x2d @ Wk[h]
+        Q[:, h, :] = x2d @ Wq[h] if Wq.ndim == 3 else expert_projection(x2d, Wq[h], idxD[:, h, :], gateD[:, h, :])
+        K[:, h, :] = x2d @ Wk[h] if Wk.ndim == 3 else expert_projection(x2d, Wk[h], idxS[:, h, :], gateS[:, h, :])
         # value experts: only the rows that selected expert e are projected with it
         for e in range(E):
             for j in range(k):
@@ -287,8 +313,8 @@ def switchhead_xl_forward(x, cache, Wq, Wk, Wv, Wo, Ws, Wd, k: int, bias_s=None,
     K = np.empty((B * CT, H, D))
     V = np.zeros((B * CT, H, D))
     for h in range(H):
-        Q[:, h, :] = x2d @ Wq[h]
-        K[:, h, :] = c2d @ Wk[h]
+        Q[:, h, :] = x2d @ Wq[h] if Wq.ndim == 3 else expert_projection(x2d, Wq[h], idxD[:, h, :], gateD[:, h, :])
+        K[:, h, :] = c2d @ Wk[h] if Wk.ndim == 3 else expert_projection(c2d, Wk[h], idxS[:, h, :], gateS[:, h, :])
         for e in range(E):
             for j in range(k):
                 rows = np.nonzero(idxS[:, h, j] == e)[0]
