@@ -83,6 +83,19 @@ sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k);
  * idx / gate / offsets / lists debug buffers' first half) are then equal. */
 sh_layer* sh_create_shared(int d_model, int n_heads, int d_head, int n_experts, int k);
 
+/* SwitchHead layer whose query and / or key projections are experts too (Sec. 2.2 writes K^h and
+ * Q^h as expert sums like V^h; the paper's ablation over which projections are experts keeps them
+ * dense in the final model, which is what sh_create builds).  moe_k != 0: K^h[t] = sum over the
+ * experts the SOURCE side of token t selected, weighted by its scores, of x[t] W_K^{h,e} (the
+ * selection the value projection uses); moe_q != 0: Q^h[t] likewise with the DESTINATION side's
+ * selection (the one the output projection uses).  sh_set_weights then takes Wq as [H, E, d_model,
+ * d_head] (moe_q) and Wk as [H, E, d_model, d_head] (moe_k) instead of [H, d_model, d_head].
+ * shared_selection != 0: one gate for both sides, as sh_create_shared (keys and queries then use the
+ * same selection).  Runs in the fp32 configuration (SH_F32) only: sh_configure refuses SH_BF16 for
+ * such a layer; sh_set_rope refuses it too.  Other arguments and limits as sh_create. */
+sh_layer* sh_create_moe_qk(int d_model, int n_heads, int d_head, int n_experts, int k, int moe_q, int moe_k,
+                           int shared_selection);
+
 /* Dense multi-head attention comparator (Eq. 1-2) built from the same kernels: every head
  * has one dense W_V and W_O and there are no gates.  Used only to time a parameter-matched
  * dense layer beside SwitchHead.  Weights are passed to sh_set_weights with n_experts = 1

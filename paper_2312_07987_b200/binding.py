@@ -21,7 +21,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
                -4: "SH_ERR_WORKSPACE", -5: "SH_ERR_CUDA", -6: "SH_ERR_TIMEOUT", -7: "SH_ERR_BOUNDS"}
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
-EXPORTS = ["sh_create", "sh_create_shared", "sh_create_dense", "sh_configure", "sh_configure_xl", "sh_workspace_bytes", "sh_set_workspace",
+EXPORTS = ["sh_create", "sh_create_shared", "sh_create_moe_qk", "sh_create_dense", "sh_configure", "sh_configure_xl", "sh_workspace_bytes", "sh_set_workspace",
            "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_set_xl_positions", "sh_forward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
            "sh_noalloc_gate_topk", "sh_debug_buffer", "sh_last_status", "sh_status_block", "sh_clear_status", "sh_check_guards",
            "sh_selftest", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
@@ -38,6 +38,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_create.argtypes = [i32] * 5
     lib.sh_create_shared.restype = vp
     lib.sh_create_shared.argtypes = [i32] * 5
+    lib.sh_create_moe_qk.restype = vp
+    lib.sh_create_moe_qk.argtypes = [i32] * 8
     lib.sh_create_dense.restype = vp
     lib.sh_create_dense.argtypes = [i32] * 3
     lib.sh_configure.restype = i32
@@ -120,12 +122,14 @@ class Layer:
     """Owns one sh_layer handle plus the torch tensors that back its workspace."""
 
     def __init__(self, d_model: int, n_heads: int, d_head: int, n_experts: int = 1, k: int = 1,
-                 dense: bool = False, shared_selection: bool = False):
+                 dense: bool = False, shared_selection: bool = False, moe_q: bool = False, moe_k: bool = False):
         self.dense = dense
         self.shared_selection = shared_selection
         self.dims = (d_model, n_heads, d_head, n_experts, k)
         if dense:
             h = lib.sh_create_dense(d_model, n_heads, d_head)
+        elif moe_q or moe_k:
+            h = lib.sh_create_moe_qk(d_model, n_heads, d_head, n_experts, k, int(moe_q), int(moe_k), int(shared_selection))
         elif shared_selection:
             h = lib.sh_create_shared(d_model, n_heads, d_head, n_experts, k)
         else:
@@ -282,7 +286,9 @@ def layer_from_inputs(inp, batch=None, seq=None, device="cuda", shared_selection
     cache_len: the first cache_len tokens of every sequence of inp.x are a Transformer-XL cache."""
     cfg = inp.cfg
     B, T = inp.x.shape[0], inp.x.shape[1]
-    L = Layer(cfg.d_model, cfg.n_heads, cfg.d_head, cfg.n_experts, cfg.k, shared_selection=shared_selection)
+    # (Wq / Wk given per expert, [H, E, M, D]: a layer with query / key experts)
+    L = Layer(cfg.d_model, cfg.n_heads, cfg.d_head, cfg.n_experts, cfg.k, shared_selection=shared_selection,
+              moe_q=inp.Wq.ndim == 4, moe_k=inp.Wk.ndim == 4)
     L.sh_configure(cfg.dtype, B, T - cache_len, device=device, cache_len=cache_len)
     dv = lambda a: to_device(a, cfg.dtype, device)
     bias = lambda a: None if a is None else torch.from_numpy(a).to(device)

@@ -94,7 +94,10 @@ static void layout_workspace(sh_layer* L) {
   o.xl_bias = take(xlb ? (size_t)d.B * d.H * (d.T - d.Tc) * d.T * 2 : 16);
   // W_O once more with the experts innermost on the contraction axis: [H, M, D*E] (sparse output projection)
   o.wos = take(sh_o_sparse_ok(L) ? HD * d.E * d.M * mid : 16);
-  o.gid = take(vp ? (size_t)d.N * d.H * 4 : 16);      // pair number of every (token, head), source side
+  o.gid = take(vp ? (size_t)d.N * d.H * 4 : 16);
+  // query / key experts (sh_create_moe_qk): [H, E, D, M] like the value experts
+  o.wq_e = take(L->moe_q ? HD * d.E * d.M * in : 16);
+  o.wk_e = take(L->moe_k ? HD * d.E * d.M * in : 16);      // pair number of every (token, head), source side
   o.stamps = take(sizeof(ShStampBlock));
   o.total = off;
 }
@@ -128,6 +131,13 @@ extern "C" sh_layer* sh_create_shared(int d_model, int n_heads, int d_head, int 
   return create_common(d_model, n_heads, d_head, n_experts, k, false, 1);
 }
 
+extern "C" sh_layer* sh_create_moe_qk(int d_model, int n_heads, int d_head, int n_experts, int k, int moe_q, int moe_k,
+                                      int shared_selection) {
+  sh_layer* L = create_common(d_model, n_heads, d_head, n_experts, k, false, shared_selection ? 1 : 2);
+  if (L) { L->moe_q = moe_q != 0; L->moe_k = moe_k != 0; }
+  return L;
+}
+
 extern "C" sh_layer* sh_create_dense(int d_model, int n_heads, int d_head) {
   return create_common(d_model, n_heads, d_head, 1, 1, true);
 }
@@ -149,6 +159,10 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
     return SH_ERR_UNSUPPORTED;
   }
   if (cache_len > 0 && L->dense) { sh_set_error("the dense comparator has no cache"); return SH_ERR_UNSUPPORTED; }
+  if ((L->moe_q || L->moe_k) && dtype != SH_F32) {
+    sh_set_error("query / key experts run in the fp32 configuration only (the tensor-core path keeps the paper's dense Q/K projections)");
+    return SH_ERR_UNSUPPORTED;
+  }
   if (cache_len > 0 && dtype == SH_BF16 && (cache_len % 128 != 0 || seq % 128 != 0)) {
     // the tensor-core attention and output kernels work on 128-token tiles that must not straddle the
     // boundary between cache and chunk, nor two sequences
@@ -232,8 +246,19 @@ static int set_weights_t(sh_layer* L, const void* Wq, const void* Wk, const void
     SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wo, 0, (size_t)HD * d.E * d.M * sizeof(TM), st));
     if (!L->dense) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wv, 0, (size_t)HD * d.E * d.M * sizeof(TI), st));
   }
-  repack<TI, TI>(Wq, wqk, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
-  repack<TI, TI>(Wk, wqk + HD * d.M, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+  // (with query / key experts: Wq / Wk [H, E, M, Dt] -> [H, E, D, M], like the value experts)
+  if (L->moe_q) {
+    if (d.D != d.Dt) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wq_e, 0, (size_t)HD * d.E * d.M * sizeof(TI), st));
+    repack<TI, TI>(Wq, ws + L->o.wq_e, d.H * d.E, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+  } else {
+    repack<TI, TI>(Wq, wqk, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+  }
+  if (L->moe_k) {
+    if (d.D != d.Dt) SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.wk_e, 0, (size_t)HD * d.E * d.M * sizeof(TI), st));
+    repack<TI, TI>(Wk, ws + L->o.wk_e, d.H * d.E, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+  } else {
+    repack<TI, TI>(Wk, wqk + HD * d.M, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
+  }
   if (L->dense) {
     // Wv [H, 1, M, D] joins the fused projection; Wo [H, 1, D, M] -> Wo_t[m][h*D + dd]
     repack<TI, TI>(Wv, wqk + 2 * HD * d.M, d.H, d.M, d.Dt, (long)d.D * d.M, d.M, 1, st);
@@ -332,16 +357,55 @@ static int forward_simt(sh_layer* L, int stages, const void* x, void* out, cudaS
   }
   if (all) sh_mark(L, 1, st);
   if (stages & SH_STAGE_QK) {
-  ShGemmArgs g{};
-  g.d = d;
-  // Q, K (and V for the dense comparator)
-  g.A = x; g.lda = d.M; g.Bt = ws + L->o.wqk; g.ldb = d.M; g.K = d.M;
-  g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
-  g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v; g.qscale = qscale;
-  g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
-  dim3 grid_qk(d.nblk, (g.ncols + 63) / 64);
-  sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_qk, 256, 0, st>>>(g);
-  L->launches += 1;
+    ShGemmArgs g{};
+    g.d = d;
+    g.A = x; g.lda = d.M; g.ldb = d.M; g.K = d.M; g.nrows = d.N;
+    g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
+    if (!L->moe_q && !L->moe_k) {
+      // Q, K (and V for the dense comparator)
+      g.Bt = ws + L->o.wqk;
+      g.ncols = (L->dense ? 3 : 2) * HD;
+      g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v; g.qscale = qscale;
+      dim3 grid_qk(d.nblk, (g.ncols + 63) / 64);
+      sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_qk, 256, 0, st>>>(g);
+      L->launches += 1;
+    } else {
+      // query / key experts: whichever of the two is dense is one projection of HD columns; an expert
+      // projection is the value experts' grouped GEMM with its own weights, side and output
+      g.ncols = HD;
+      dim3 grid_1(d.nblk, (HD + 63) / 64);
+      if (!L->moe_q) {
+        g.Bt = ws + L->o.wqk; g.out0 = ws + L->o.q; g.qscale = qscale;
+        sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_1, 256, 0, st>>>(g);
+        L->launches += 1;
+      }
+      if (!L->moe_k) {
+        g.Bt = (const TI*)(ws + L->o.wqk) + (size_t)HD * d.M; g.out0 = ws + L->o.k; g.qscale = 1.f;
+        sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_QKV><<<grid_1, 256, 0, st>>>(g);
+        L->launches += 1;
+      }
+      ShGemmArgs e{};
+      e.d = d; e.A = x; e.lda = d.M; e.ldb = d.M; e.K = d.M; e.ncols = d.D; e.b_group_stride = (long)d.D * d.M;
+      dim3 grid_e(d.max_tiles, (d.D + 63) / 64);
+      if (L->moe_k) {                                      // source side, like the values
+        SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.k, 0, (size_t)d.N * HD * sizeof(TM), st));
+        e.Bt = ws + L->o.wk_e; e.out0 = ws + L->o.k; e.vscale = 0.f;
+        e.lists = (const int*)(ws + L->o.lists); e.lgate = (const float*)(ws + L->o.lgate);
+        e.tiles = (const ShTile*)(ws + L->o.tiles); e.ntiles = (const int*)(ws + L->o.ntiles);
+        sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_V><<<grid_e, 256, 0, st>>>(e);
+        L->launches += 2;
+      }
+      if (L->moe_q) {                                      // destination side, like the output (stored scaled, as the dense queries are)
+        SH_CUDA_CHECK(cudaMemsetAsync(ws + L->o.q, 0, (size_t)d.N * HD * sizeof(TM), st));
+        const size_t side1 = d.sides == 2 ? (size_t)d.H * d.N * d.k : 0;
+        e.Bt = ws + L->o.wq_e; e.out0 = ws + L->o.q; e.vscale = qscale;
+        e.lists = (const int*)(ws + L->o.lists) + side1; e.lgate = (const float*)(ws + L->o.lgate) + side1;
+        e.tiles = (const ShTile*)(ws + L->o.tiles) + (d.sides == 2 ? d.max_tiles : 0);
+        e.ntiles = (const int*)(ws + L->o.ntiles) + (d.sides == 2 ? 1 : 0);
+        sh_simt_gemm_kernel<TI, TI, TM, SH_EPI_V><<<grid_e, 256, 0, st>>>(e);
+        L->launches += 2;
+      }
+    }
   }
   if (all) sh_mark(L, 2, st);
   if (!L->dense && (stages & SH_STAGE_V)) {
@@ -468,6 +532,7 @@ extern "C" int sh_set_rope(sh_layer* L, double base, void* stream) {
   if (L->xl_positions) { sh_set_error("relative positions are switched on: one positional encoding at a time"); return SH_ERR_UNSUPPORTED; }
   if (L->d.Tc > 0) { sh_set_error("rotary embeddings are for the cache-less layer (the paper's RoPE models have no cache)"); return SH_ERR_UNSUPPORTED; }
   if (L->d.Dt % 2) { sh_set_error("rotary embedding needs an even d_head (got %d)", L->d.Dt); return SH_ERR_UNSUPPORTED; }
+  if (L->moe_q || L->moe_k) { sh_set_error("rotary embeddings are applied in the dense Q/K projection's epilogue: not with query / key experts"); return SH_ERR_UNSUPPORTED; }
   const int n = L->d.T * (L->d.D / 2);
   sh_rope_table_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>((float2*)(L->ws + L->o.rope), L->d.T, L->d.D, L->d.Dt, base);
   SH_CUDA_CHECK(cudaGetLastError());

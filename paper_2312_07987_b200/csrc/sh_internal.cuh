@@ -89,7 +89,7 @@ __device__ __forceinline__ void sh_stamp_end(unsigned long long* s, int k) { if 
 
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, gid, stamps, total;
+         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, gid, wq_e, wk_e, stamps, total;
 };
 
 // Words of the 256-byte status block at the start of the workspace.
@@ -109,6 +109,7 @@ enum {
 struct sh_layer {
   ShDims d{};
   bool dense = false;
+  bool moe_q = false, moe_k = false;   // query / key projections are experts too (destination / source side selection)
   int dtype = -1;
   char* ws = nullptr;
   size_t ws_bytes = 0;

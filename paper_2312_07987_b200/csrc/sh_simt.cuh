@@ -361,6 +361,7 @@ struct ShGemmArgs {
   int a_head_stride;                // grouped O: column offset of head h inside an A row
   void* out0; void* out1; void* out2;
   float qscale;
+  float vscale;                     // grouped V-type epilogue: extra factor on the gate-scaled result (0 = none)
   const float2* rope;               // QKV epilogue: (cos, sin) table [D/2, T] of the rotary embedding, or nullptr
   ShDims d;
 };
@@ -468,7 +469,7 @@ sh_simt_gemm_kernel(ShGemmArgs g) {
         dst[(((size_t)b * d.H + hh) * d.T + t) * d.D + dd] = sh_from_float<TC>(which == 0 ? v * g.qscale : v);
       } else if (EPI == SH_EPI_V) {
         const int b = gr / d.T, t = gr % d.T;
-        atomicAdd((TC*)g.out0 + (((size_t)b * d.H + h) * d.T + t) * d.D + n, sh_from_float<TC>(s_gate[lr] * v));
+        atomicAdd((TC*)g.out0 + (((size_t)b * d.H + h) * d.T + t) * d.D + n, sh_from_float<TC>(s_gate[lr] * v * (g.vscale != 0.f ? g.vscale : 1.f)));
       } else if (EPI == SH_EPI_O) {
         const int orow = sh_out_row(d, gr);                // (cache tokens have no output row)
         if (orow >= 0) atomicAdd((float*)g.out0 + (size_t)orow * d.M + n, s_gate[lr] * v);

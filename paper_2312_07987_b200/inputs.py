@@ -45,6 +45,8 @@ class LayerConfig:
     seed: int
     zipf_bias: float = 0.0   # exponent of the per-expert Zipf gate-bias profile (0 = no bias)
     min_gap: float = 1e-3    # required logit margin at rank k
+    moe_q: bool = False      # query / key projections as experts too (Wq / Wk drawn as [H, E, M, D])
+    moe_k: bool = False
 
     @property
     def n_tokens(self) -> int:
@@ -148,8 +150,8 @@ def make_inputs(cfg: LayerConfig, *, batch: Optional[int] = None, seq: Optional[
     def normal(shape, fan_in):
         return rng.standard_normal(shape, dtype=np.float64) / np.sqrt(fan_in)
 
-    Wq = _store(normal((H, M, D), M), cfg.dtype)
-    Wk = _store(normal((H, M, D), M), cfg.dtype)
+    Wq = _store(normal((H, E, M, D) if cfg.moe_q else (H, M, D), M), cfg.dtype)
+    Wk = _store(normal((H, E, M, D) if cfg.moe_k else (H, M, D), M), cfg.dtype)
     Wv = _store(normal((H, E, M, D), M), cfg.dtype)
     Wo = _store(normal((H, E, D, M), D), cfg.dtype)
     Ws = _store(normal((H, M, E), M), cfg.dtype)
