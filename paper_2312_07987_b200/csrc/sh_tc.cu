@@ -672,11 +672,11 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     const size_t side1 = d.sides == 2 ? (size_t)d.N * d.H * d.k : 0;   // shared selection: the one side there is
     a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
     a.out = (float*)out; a.status = status;
-    // Up to three selections per (token, head) the CTA-pair kernel serves (its builder threads keep a
-    // token's selections in registers).  With more, the single-CTA kernel, which reads the
-    // selections from shared memory and multiplies by the gate after the UMMA; a device that cannot
-    // hold a two-CTA cluster of the pair kernel's size uses it too.
-    bool pair = S->o_pair && d.k <= 3;
+    // Up to four selections per (token, head) the CTA-pair kernels serve (their builder threads keep a
+    // token's selections in registers).  With more, the single-CTA kernel, which reads the selections
+    // from shared memory and multiplies by the gate after the UMMA; a device that cannot hold a two-CTA
+    // cluster of the pair kernel's size uses it too.
+    bool pair = S->o_pair && d.k <= OPAIR_KMAX;
     const bool sparse = pair && S->o_sparse && sh_o_sparse_ok(L);
     if (sparse) {
       constexpr int psm = OprojSpSmem<128>::TOTAL;

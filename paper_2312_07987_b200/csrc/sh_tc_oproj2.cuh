@@ -37,7 +37,7 @@
 
 namespace shtc {
 
-constexpr int OPAIR_KMAX = 3;                            // selections per (token, head) a builder keeps in registers (the kernel serves k <= 3)
+constexpr int OPAIR_KMAX = 4;                            // selections per (token, head) a builder keeps in registers (the kernel serves k <= 4)
 
 template <int D>
 struct OprojPairSmem {
