@@ -91,8 +91,11 @@ sh_layer* sh_create_shared(int d_model, int n_heads, int d_head, int n_experts, 
  * selection (the one the output projection uses).  sh_set_weights then takes Wq as [H, E, d_model,
  * d_head] (moe_q) and Wk as [H, E, d_model, d_head] (moe_k) instead of [H, d_model, d_head].
  * shared_selection != 0: one gate for both sides, as sh_create_shared (keys and queries then use the
- * same selection).  Runs in the fp32 configuration (SH_F32) only: sh_configure refuses SH_BF16 for
- * such a layer; sh_set_rope refuses it too.  Other arguments and limits as sh_create. */
+ * same selection).  SH_F32 takes every shape.  SH_BF16 (tensor-core path): an expert projection of
+ * keys / queries runs on the pair-tiled value-expert kernel, so sh_configure wants k = 2, 2..8
+ * experts, d_head in 65..128 and, when only one of the two is an expert projection, an even number
+ * of heads; it refuses other shapes.  sh_set_rope refuses such a layer.  Other arguments and limits
+ * as sh_create. */
 sh_layer* sh_create_moe_qk(int d_model, int n_heads, int d_head, int n_experts, int k, int moe_q, int moe_k,
                            int shared_selection);
 

@@ -64,10 +64,10 @@ static void layout_workspace(sh_layer* L) {
   o.gate = take(slots * 4);
   // (a layer whose value projection is tiled by expert pairs sorts H * E(E-1)/2 buckets in a forward pass)
   const bool vp = sh_v_pairs_ok(L);
-  const size_t hist = vp && d.H * sh_pair_count(d.E) > d.G ? (size_t)d.H * sh_pair_count(d.E) : (size_t)d.G;
+  const size_t hist = vp && 2 * d.H * sh_pair_count(d.E) > d.G ? (size_t)2 * d.H * sh_pair_count(d.E) : (size_t)d.G;
   o.blockcnt = take((size_t)d.nblk * hist * 4);
   o.blockoff = take((size_t)d.nblk * hist * 4);
-  o.offsets = take(((size_t)2 * d.H * (d.E + 1) + (vp ? (size_t)d.H * (sh_pair_count(d.E) + 1) : 0)) * 4);
+  o.offsets = take(((size_t)2 * d.H * (d.E + 1) + (vp ? (size_t)2 * d.H * (sh_pair_count(d.E) + 1) : 0)) * 4);
   o.lists = take(slots * 4);
   o.lgate = take(slots * 4);
   o.tiles = take((size_t)2 * d.max_tiles * sizeof(ShTile));
@@ -94,7 +94,7 @@ static void layout_workspace(sh_layer* L) {
   o.xl_bias = take(xlb ? (size_t)d.B * d.H * (d.T - d.Tc) * d.T * 2 : 16);
   // W_O once more with the experts innermost on the contraction axis: [H, M, D*E] (sparse output projection)
   o.wos = take(sh_o_sparse_ok(L) ? HD * d.E * d.M * mid : 16);
-  o.gid = take(vp ? (size_t)d.N * d.H * 4 : 16);
+  o.gid = take(vp ? (size_t)2 * d.N * d.H * 4 : 16);  // (both sides: query experts are tiled by the destination side's pairs)
   // query / key experts (sh_create_moe_qk): [H, E, D, M] like the value experts
   o.wq_e = take(L->moe_q ? HD * d.E * d.M * in : 16);
   o.wk_e = take(L->moe_k ? HD * d.E * d.M * in : 16);      // pair number of every (token, head), source side
@@ -160,8 +160,15 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
   }
   if (cache_len > 0 && L->dense) { sh_set_error("the dense comparator has no cache"); return SH_ERR_UNSUPPORTED; }
   if ((L->moe_q || L->moe_k) && dtype != SH_F32) {
-    sh_set_error("query / key experts run in the fp32 configuration only (the tensor-core path keeps the paper's dense Q/K projections)");
-    return SH_ERR_UNSUPPORTED;
+    // on the tensor-core path an expert projection of keys or queries is the pair-tiled value kernel with
+    // other weights: the shapes that kernel serves, and a dense half (if any) the CTA-pair GEMM can tile
+    const bool ok = d0.k == 2 && d0.E >= 2 && d0.E <= 8 && d0.Dt > 64 && d0.Dt <= 128 &&
+                    ((L->moe_q && L->moe_k) || (d0.H * 128) % 256 == 0);
+    if (!ok) {
+      sh_set_error("query / key experts with bf16 storage need k = 2, 2..8 experts, d_head in 65..128 and, when only one of the "
+                   "two is an expert projection, an even number of heads (the fp32 configuration takes every shape)");
+      return SH_ERR_UNSUPPORTED;
+    }
   }
   if (cache_len > 0 && dtype == SH_BF16 && (cache_len % 128 != 0 || seq % 128 != 0)) {
     // the tensor-core attention and output kernels work on 128-token tiles that must not straddle the

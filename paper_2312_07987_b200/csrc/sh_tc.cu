@@ -79,7 +79,7 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
 
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
-  CUtensorMap map_wqk, map_wqk128, map_wv, map_wo, map_wo256, map_wos, map_ahat, map_wgate;
+  CUtensorMap map_wqk, map_wqk128, map_wv, map_wq_e, map_wk_e, map_wo, map_wo256, map_wos, map_ahat, map_wgate;
   CUtensorMap map_q2d, map_r16;  // score-bias GEMM of the Transformer-XL position term: Q as [B*H*T, D], R16 as [H*T, D]
   CUtensorMap map_x;             // tensor map of the last x pointer seen (x_cached)
   const void* x_cached = nullptr;
@@ -254,6 +254,8 @@ int sh_tc_prepare(sh_layer* L) {
   if ((rc = sh_tc_encode_2d(&S->map_wqk128, 0, ws + L->o.wqk, d.M, (uint64_t)nproj * HD, (uint64_t)d.M * 2, 64, 128))) return rc;
   if (!L->dense) {
     if ((rc = sh_tc_encode_2d(&S->map_wv, 0, ws + L->o.wv, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
+    if (L->moe_q && (rc = sh_tc_encode_2d(&S->map_wq_e, 0, ws + L->o.wq_e, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
+    if (L->moe_k && (rc = sh_tc_encode_2d(&S->map_wk_e, 0, ws + L->o.wk_e, d.M, (uint64_t)d.H * d.E * d.D, (uint64_t)d.M * 2, 64, d.D))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 128))) return rc;
     if ((rc = sh_tc_encode_2d(&S->map_wo256, 1, ws + L->o.wo, d.D, (uint64_t)d.H * d.E * d.M, (uint64_t)d.D * 2, 64, 256))) return rc;
     if (sh_o_sparse_ok(L) && (rc = sh_tc_encode_2d(&S->map_wos, 1, ws + L->o.wos, (uint64_t)d.D * d.E, (uint64_t)d.H * d.M, (uint64_t)d.D * d.E * 2, 64, 128))) return rc;
@@ -337,7 +339,9 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
   g.blockcnt = (int*)(ws + L->o.blockcnt);
   const bool vp = zero_for_forward && use_v_pairs(L);
-  g.vpairs = vp; g.NP = sh_pair_count(d.E); g.GH = vp ? d.H * g.NP : d.G; g.gid = (int*)(ws + L->o.gid);
+  // (query experts are tiled by the DESTINATION side's pairs: then both sides are bucketed by pair)
+  g.vpairs = vp ? ((L->moe_q && d.sides == 2) ? 2 : 1) : 0;
+  g.NP = sh_pair_count(d.E); g.GH = vp ? g.vpairs * d.H * g.NP : d.G; g.gid = (int*)(ws + L->o.gid);
   const int GHmax = g.GH > d.G ? g.GH : d.G;
   g.zero_v = (zero_for_forward && !vp) ? (void*)(ws + L->o.v) : nullptr;    // (the pair-tiled kernel stores every value row once)
   g.zero_out = (zero_for_forward && (S->simt_mask & SH_STAGE_O) && d.Tc == 0) ? (float*)out : nullptr;
@@ -353,7 +357,7 @@ static int tc_gate_sort(sh_layer* L, const void* x, void* out, bool zero_for_for
   // sort's loops run over sides * H groups.
   ShDims ds = d;
   if (zero_for_forward && !(S->simt_mask & SH_STAGE_O)) ds.sides = 1;
-  if (vp) { ds.sides = 1; ds.E = g.NP; ds.k = 1; ds.G = g.GH; ds.tile_rows_src = 256; }   // buckets (head, pair), one entry per (token, head)
+  if (vp) { ds.sides = g.vpairs; ds.E = g.NP; ds.k = 1; ds.G = g.GH; ds.tile_rows_src = 256; }   // buckets (side, head, pair), one entry per (token, head)
   // Fused sort: when every CTA of the gate kernel can be resident at once (cooperative launch) and the
   // sort's scratch fits behind the logits tile in the idle operand ring, the gate kernel places the
   // tokens itself and there is no sort kernel.  Used when the gate kernel needs at most half of the SMs:
@@ -480,9 +484,21 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   // with one grid, and 265 against 270.5 at 16384 tokens.
   int qkA = 0, qkB = 0;                                    // CTA pairs of the two grids
   TcGemmArgs qg{};
+  if (L->moe_q || L->moe_k) {
+    // expert projections of keys / queries run on the pair-tiled kernel (pair-bucketed lists), or - debug
+    // library, SH_SIMT_STAGES - on the CUDA-core kernels together with gate and value stage (expert lists)
+    const bool bad = (simt & SH_STAGE_QK) ? use_v_pairs(L)
+                                          : (!use_v_pairs(L) || !S->persistent || !S->qk_pair || qk_pairs_max(S) <= 0);
+    if (bad) {
+      sh_set_error("query / key experts need the CTA-pair projection kernels on this device and in this build");
+      return SH_ERR_UNSUPPORTED;
+    }
+  }
+  // a layer with query (key) experts projects only its keys (queries) densely; with both, nothing
+  const int qk_ncols = (L->moe_q || L->moe_k) ? HD : 2 * HD;
   if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_bn == 256 && S->persistent && S->qk_pair &&
-      S->qk_two_grids && qk_pairs_max(S) > 0) {
-    const int ptiles = ((d.N + 255) / 256) * ((2 * HD + 255) / 256);
+      S->qk_two_grids && qk_pairs_max(S) > 0 && !(L->moe_q && L->moe_k)) {
+    const int ptiles = ((d.N + 255) / 256) * ((qk_ncols + 255) / 256);
     const int pairs = ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max;
     // (one gate CTA per SM; running two per SM with half the stages, to leave grid A more SMs when
     //  there are more gate CTAs than half the SMs, made the gate kernel 2.4 us slower and the layer
@@ -492,9 +508,10 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     qkA = (L->sm_count - gate_sms) / 2;
     if (qkA > pairs) qkA = pairs;
     qkB = pairs - qkA;
-    qg.d = d; qg.K = d.M; qg.ncols = 2 * HD; qg.nrows = d.N;
-    qg.out0 = ws + L->o.q; qg.out1 = ws + L->o.k; qg.out2 = ws + L->o.v;
-    qg.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+    qg.d = d; qg.K = d.M; qg.ncols = qk_ncols; qg.nrows = d.N;
+    qg.out0 = ws + (L->moe_q ? L->o.k : L->o.q); qg.out1 = ws + L->o.k; qg.out2 = ws + L->o.v;
+    qg.qscale = L->moe_q ? 1.f : 1.4426950408889634f / sqrtf((float)d.Dt);
+    qg.b_row0 = L->moe_q ? HD : 0;
     qg.status = status; qg.sched = status + SH_ST_SCHED; qg.claimers = qkA + qkB;
     qg.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
     qg.stamp_id = SH_K_QK_A;
@@ -540,12 +557,15 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     // (launched above, as two grids)
   } else if (simt & SH_STAGE_QK) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_QK, x, out, st))) return rc;
+  } else if (L->moe_q && L->moe_k) {
+    // (queries and keys are both expert projections: they follow the value experts below)
   } else {
     cudaStream_t qst = overlap ? S->side : st;              // side stream when overlapping
     TcGemmArgs g{};
-    g.d = d; g.K = d.M; g.ncols = (L->dense ? 3 : 2) * HD; g.nrows = d.N;
-    g.out0 = ws + L->o.q; g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
-    g.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+    g.d = d; g.K = d.M; g.ncols = L->dense ? 3 * HD : (L->moe_q || L->moe_k) ? HD : 2 * HD; g.nrows = d.N;
+    g.out0 = ws + (L->moe_q ? L->o.k : L->o.q); g.out1 = ws + L->o.k; g.out2 = ws + L->o.v;
+    g.qscale = L->moe_q ? 1.f : 1.4426950408889634f / sqrtf((float)d.Dt);
+    g.b_row0 = L->moe_q ? HD : 0;
     g.status = status;
     g.sched = status + SH_ST_SCHED;
     g.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
@@ -585,8 +605,26 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
       g.v = (__half*)(ws + L->o.v); g.status = status;
       const int bound = (d.N * d.H + 255) / 256 + d.H * sh_pair_count(d.E);       // tiles: at most this many
       const unsigned pgrid = 2u * (unsigned)(bound < S->v_pairs_max ? bound : S->v_pairs_max);
+      g.scale = 0.f; g.stamp_id = SH_K_V;
       if ((rc = launch_k_pairs(pdl, sh_tc_vpair_kernel<6>, dim3(pgrid), dim3(320), VPS::TOTAL, st, S->map_wv, g))) return rc;
       L->launches += 1;
+      // key / query experts: the same kernel with the key (query) experts' weights, the source
+      // (destination) side's pair tiles and gates, into the K (Q) buffer; queries carry the score scale
+      if (L->moe_k && !(simt & SH_STAGE_QK)) {
+        g.v = (__half*)(ws + L->o.k); g.stamp_id = -1;
+        if ((rc = launch_k_pairs(pdl, sh_tc_vpair_kernel<6>, dim3(pgrid), dim3(320), VPS::TOTAL, st, S->map_wk_e, g))) return rc;
+        L->launches += 1;
+      }
+      if (L->moe_q && !(simt & SH_STAGE_QK)) {
+        const size_t s1 = d.sides == 2 ? 1 : 0;            // destination side (with a shared selection: the one side there is)
+        g.lists = (const int*)(ws + L->o.lists) + s1 * (size_t)d.H * d.N;
+        g.tiles = (const ShTile*)(ws + L->o.tiles) + s1 * (size_t)d.max_tiles;
+        g.ntiles = (const int*)(ws + L->o.ntiles) + s1;
+        g.idx = (const int*)(ws + L->o.idx) + s1 * (size_t)d.N * d.H * d.k; g.gate = (const float*)(ws + L->o.gate) + s1 * (size_t)d.N * d.H * d.k;
+        g.v = (__half*)(ws + L->o.q); g.scale = 1.4426950408889634f / sqrtf((float)d.Dt); g.stamp_id = -1;
+        if ((rc = launch_k_pairs(pdl, sh_tc_vpair_kernel<6>, dim3(pgrid), dim3(320), VPS::TOTAL, st, S->map_wq_e, g))) return rc;
+        L->launches += 1;
+      }
     } else {
       TcGemmArgs g{};
       g.d = d; g.K = d.M; g.ncols = d.D;

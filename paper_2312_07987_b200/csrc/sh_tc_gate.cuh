@@ -42,10 +42,10 @@ struct TcGateArgs {
   // value projection tiled by expert PAIRS (k = 2, forward pass only): the source side is bucketed by
   // (head, pair number) - histogram, sort and tile table run over H * NP buckets with one entry per
   // (token, head) - and the destination side is not bucketed at all
-  int vpairs;                // 0 / 1
+  int vpairs;                // 0, or the number of sides bucketed by pair: 1 = the source side, 2 = both (query experts)
   int NP;                    // pairs per head: E (E - 1) / 2
-  int GH;                    // histogram width: vpairs ? H * NP : G
-  int* gid;                  // [N, H] pair number of every (token, head)
+  int GH;                    // histogram width: vpairs ? vpairs * H * NP : G
+  int* gid;                  // [vpairs, N, H] pair number of every (token, head)
 };
 
 constexpr int GATE_THREADS = 608;
@@ -213,11 +213,11 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             g.gate[o + j] = gv;
             if (g.vpairs) {
               if (j == 0) first = best;
-              else if (side == 0) {
+              else if (side < g.vpairs) {
                 const int pid = sh_pair_id(min(first, best), max(first, best), d.E);
-                g.gid[(size_t)t * d.H + h] = pid;
-                if (g.fused) s_idx[r * d.H + h] = pid;
-                atomicAdd(&s_hist[h * g.NP + pid], 1);
+                g.gid[((size_t)side * d.N + t) * d.H + h] = pid;
+                if (g.fused) s_idx[side * 128 * d.H + r * d.H + h] = pid;
+                atomicAdd(&s_hist[(side * d.H + h) * g.NP + pid], 1);
               }
               continue;
             }
@@ -257,7 +257,7 @@ sh_tc_gate_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
       if (*(volatile int*)s_flag) {
         ShDims ds = d;
         ds.sides = g.sort_sides;
-        if (g.vpairs) { ds.sides = 1; ds.E = g.NP; ds.k = 1; ds.G = g.GH; }   // buckets (head, pair), one entry per (token, head)
+        if (g.vpairs) { ds.sides = g.vpairs; ds.E = g.NP; ds.k = 1; ds.G = g.GH; }   // buckets (side, head, pair), one entry per (token, head)
         sh_sort_block(g.idx, g.gate, g.blockcnt, g.offsets, g.lists, g.lgate, g.tiles, g.ntiles, ds, s_sort, et, NSEL, (int)blockIdx.x, true, sel_sync);
       }
     }

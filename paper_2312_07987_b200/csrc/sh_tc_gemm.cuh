@@ -36,6 +36,7 @@ struct TcGemmArgs {
   float* v_early;        // value experts: fp32 sums [B, H, SH_EARLY_ROWS, D] of the first rows of every sequence, or nullptr
   int* v_early_cnt;      // ... and their arrival counters [B, H, SH_EARLY_ROWS]
   int claimers;          // claiming CTAs (or CTA pairs) over all grids that share sched; 0: this grid's own
+  int b_row0;            // CTA-pair dense projection: first weight row (a layer with query experts projects the keys alone: row H*D)
   int stamp_id;          // SH_K_* slot of this launch in the stamp block (sh_forward_stamped)
 };
 

@@ -116,7 +116,7 @@ sh_tc_qk_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         }
         if (t < 0) break;
         const int row0 = (t / ncol) * 256 + (int)rank * 128;
-        const int brow = (t % ncol) * BN + (int)rank * 128;
+        const int brow = g.b_row0 + (t % ncol) * BN + (int)rank * 128;
         for (int kb = 0; kb < KB; ++kb) {
           if (!mbar_wait(&empty_bar[s], par, g.status, dead)) break;
           const uint32_t sa = sbase + s * SM::STAGE_BYTES, sb = sa + SM::A_BYTES;

@@ -37,7 +37,9 @@ struct TcVPairArgs {
   const int* ntiles;
   const int* idx;            // source side [N, H, 2]
   const float* gate;         // source side [N, H, 2]
-  __half* v;                 // [B, H, T, D]
+  __half* v;                 // [B, H, T, D]: the projection's result (V; K or Q of a layer with key / query experts)
+  float scale;               // extra factor on the result (the queries' log2(e)/sqrt(d_head)); 0 = none
+  int stamp_id;              // SH_K_V, or -1: no stamps (the key / query launches)
   int* status;
 };
 
@@ -84,13 +86,16 @@ sh_tc_vpair_kernel(const __grid_constant__ CUtensorMap mapW, TcVPairArgs g) {
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
-  if (threadIdx.x == 0) sh_stamp_resident(d.stamps, SH_K_V);
+  if (threadIdx.x == 0 && g.stamp_id >= 0) sh_stamp_resident(d.stamps, g.stamp_id);
   pdl_wait();                                              // the sorted lists and the tile table
-  if (threadIdx.x == 0) sh_stamp_start(d.stamps, SH_K_V);
+  if (threadIdx.x == 0 && g.stamp_id >= 0) sh_stamp_start(d.stamps, g.stamp_id);
+  // (the first tile's entry is fetched beside the tile count, not behind it: every dependent trip to L2
+  //  costs this kernel's start 2-3 us while the Q/K projection's operand traffic keeps L2 busy)
+  const ShTile tile_first = g.tiles[pair];                // (the table has room for every pair's index)
   const int ntiles = *g.ntiles;
   const int NP = sh_pair_count(d.E);
   auto tile_of = [&](int t) -> ShTile {
-    ShTile tl = g.tiles[t];
+    ShTile tl = t == pair ? tile_first : g.tiles[t];
 #ifdef SH_DEBUG
     const bool ok = SH_INDEX_OK(tl.h, d.H, g.status, SH_SITE_V_TILE) && SH_INDEX_OK(tl.e, NP, g.status, SH_SITE_V_TILE) &&
                     SH_INDEX_OK(tl.nrows, 257, g.status, SH_SITE_V_TILE) &&
@@ -210,6 +215,7 @@ sh_tc_vpair_kernel(const __grid_constant__ CUtensorMap mapW, TcVPairArgs g) {
         const float g0 = g.gate[so], g1 = g.gate[so + 1];
         ga = i0 < i1 ? g0 : g1;                            // a = the lower expert index of the pair
         gb = i0 < i1 ? g1 : g0;
+        if (g.scale != 0.f) { ga *= g.scale; gb *= g.scale; }
       }
       if (!mbar_wait(&acc_full[b], (it >> 1) & 1, g.status, dead)) break;
       tc_fence_after();
@@ -245,7 +251,7 @@ sh_tc_vpair_kernel(const __grid_constant__ CUtensorMap mapW, TcVPairArgs g) {
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();
-  if (threadIdx.x == 0) sh_stamp_end(d.stamps, SH_K_V);
+  if (threadIdx.x == 0 && g.stamp_id >= 0) sh_stamp_end(d.stamps, g.stamp_id);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc_pair(tmem, 512);
