@@ -36,10 +36,10 @@ BF16_CONFIGS = ["small_bf16", "c4_262m_bf16", "long_ctx_bf16", "wide_skew_bf16"]
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel (MB), from the one-kernel ncu
 # captures summarised under profiles/ (the file named beside each workload)
 DRAM_TRAFFIC_MB = {
-    "c4_262m_bf16": {"gate": 16.93, "qk": 18.91, "v": 21.66, "attn": 25.23, "o": 13.17},        # profiles/c4_262m_bf16_forward_kernels.md
-    "long_ctx_bf16": {"gate": 33.76, "sort": 0.64, "qk": 36.36, "v": 43.66, "attn": 52.01, "o": 38.26},   # profiles/long_ctx_bf16_forward_kernels.md
-    "small_bf16": {"gate": 8.49, "qk": 8.69, "v": 11.84, "attn": 6.34, "o": 3.18},             # profiles/small_bf16_forward_kernels.md
-    "wide_skew_bf16": {"gate": 85.45, "sort": 4.37, "qk": 108.96, "v": 518.50, "attn": 143.16, "o": 621.99},   # profiles/wide_skew_bf16_forward_kernels.md
+    "c4_262m_bf16": {"gate": 16.93, "qk": 18.91, "v": 21.67, "attn": 25.23, "o": 13.17},        # profiles/c4_262m_bf16_forward_kernels.md
+    "long_ctx_bf16": {"gate": 33.76, "sort": 0.64, "qk": 36.43, "v": 43.65, "attn": 52.41, "o": 38.80},   # profiles/long_ctx_bf16_forward_kernels.md
+    "small_bf16": {"gate": 8.50, "qk": 8.69, "v": 11.84, "attn": 6.34, "o": 3.18},             # profiles/small_bf16_forward_kernels.md
+    "wide_skew_bf16": {"gate": 84.90, "sort": 4.39, "qk": 109.21, "v": 600.48, "attn": 143.04, "o": 618.35},   # profiles/wide_skew_bf16_forward_kernels.md
 }
 KERNEL_STAGE = {"gate": "gate_topk_sort", "sort": "gate_topk_sort", "qk_a": "qk_proj", "qk_b": "qk_proj", "v": "v_experts",
                 "attn": "attention", "o": "o_experts"}
