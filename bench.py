@@ -292,6 +292,30 @@ def measure_config(cfg, args, rank, world, peaks, flush, barrier, steps, min_sec
     b.record(stream)
     torch.cuda.synchronize()
     res["warm_ms"] = a.elapsed_time(b) / steps
+    # the same with the pass captured once in a CUDA graph and replayed (the caller's option: the library's
+    # launches, side streams included, are capturable): one host call per pass instead of ~15, so the
+    # figure is the device's back-to-back time even where the host cannot keep ahead
+    res["graph_ms"] = None
+    try:
+        gstream = torch.cuda.Stream()
+        with torch.cuda.stream(gstream):
+            layer.sh_forward(x, out)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gstream):
+                layer.sh_forward(x, out)
+            for _ in range(3):
+                graph.replay()
+            a.record(gstream)
+            for _ in range(steps):
+                graph.replay()
+            b.record(gstream)
+        torch.cuda.synchronize()
+        res["graph_ms"] = a.elapsed_time(b) / steps
+        del graph
+    except Exception as e:                                   # (reported as null; the launch path does not depend on it)
+        res["graph_error"] = str(e)[:200]
+        torch.cuda.synchronize()
 
     res["timeline"] = kernel_timeline(layer, x, out, flush)
     # serialised stage times (ordinary launches, one stream, CUDA events at the stage boundaries): what each
@@ -407,6 +431,7 @@ def main():
             "frac_of_bf16_peak_measured": useful_tflops / (world * peaks["tflops"]),
             "frac_of_bf16_peak_nominal_2250": useful_tflops / (world * 2250.0),
             "ms_per_step_l2_warm": warm_ms,
+            "ms_per_step_l2_warm_graph_replay": m.get("graph_ms"),
             "useful_tflops_l2_warm": world * fl["total"] / (warm_ms * 1e-3) / 1e12,
             "kernel_spans_us": {k: [round(s, 2), round(e, 2)] for k, (s, e) in sorted(tl.items(), key=lambda kv: kv[1][0])},
             "stage_ms_serialised": {n: float(v) for n, v in zip(STAGES + ["total"], m["stage_ms_serialised"])},
@@ -515,6 +540,7 @@ def main():
                     per[name] = dict(ms_per_step=line["ms_per_step"], useful_tflops=line["useful_tflops"] / world,
                                      frac_of_bf16_peak_measured=line["frac_of_bf16_peak_measured"],
                                      ms_per_step_l2_warm=line["ms_per_step_l2_warm"],
+                                     ms_per_step_l2_warm_graph_replay=line["ms_per_step_l2_warm_graph_replay"],
                                      dominant_kernel=line["roofline"]["kernel"], dominant_kernel_ms=line["roofline"]["ms"],
                                      dominant_kernel_frac=line["roofline"]["frac"])
                 continue
@@ -528,7 +554,8 @@ def main():
                 roof = roofline_from_timeline(c, mc["timeline"], flc, peaks)
                 per[name] = dict(ms_per_step=msc, useful_tflops=flc["total"] / (msc * 1e-3) / 1e12,
                                  frac_of_bf16_peak_measured=flc["total"] / (msc * 1e-3) / 1e12 / peaks["tflops"],
-                                 ms_per_step_l2_warm=red[nrep], dominant_kernel=roof["kernel"], dominant_kernel_ms=roof["ms"],
+                                 ms_per_step_l2_warm=red[nrep], ms_per_step_l2_warm_graph_replay=mc.get("graph_ms"),
+                                 dominant_kernel=roof["kernel"], dominant_kernel_ms=roof["ms"],
                                  dominant_kernel_frac=roof["frac"],
                                  kernel_spans_us={k: [round(s, 2), round(e, 2)] for k, (s, e) in sorted(mc["timeline"].items(), key=lambda kv: kv[1][0])})
             del mc
