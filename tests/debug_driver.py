@@ -37,6 +37,12 @@ def main(case: str) -> None:
         # the shapes the 2:4-sparse output projection serves (or, with SH_O_MASKED, the masked kernel on them)
         for cfg in tp.SPARSE_O_CONFIGS:
             tp.full_check(inputs.make_inputs(cfg), check_stage_buffers=False)
+    elif case == "moe_qk":
+        # key / query experts on the pair-tiled kernel: both sides bucketed by expert pair, every list entry,
+        # tile field and expert index range-checked
+        for moe_q, moe_k in ((True, False), (False, True), (True, True)):
+            cfg = inputs.LayerConfig("moe_qk_dbg", inputs.DTYPE_BF16, 2, 300, 256, 2, 128, 8, 2, seed=741, zipf_bias=1.2, moe_q=moe_q, moe_k=moe_k)
+            tp.full_check(inputs.make_inputs(cfg))
     elif case == "index_selftest":
         inp = inputs.make_inputs(inputs.CONFIGS["small_bf16"], batch=1)
         layer = binding.layer_from_inputs(inp)

@@ -36,6 +36,10 @@ def test_sparse_output_projection_shapes_with_index_checks_and_against_the_maske
     run_case("sparse_o", {"SH_V_BY_EXPERT": "1"})
 
 
+def test_key_and_query_experts_with_index_checks():
+    run_case("moe_qk")
+
+
 def test_index_checks_stay_silent_on_edge_shapes():
     run_case("edges")
 
