@@ -259,6 +259,10 @@ int sh_noalloc_gate_topk(int dtype, int n_tokens, int d_model, int n_heads, int 
 /* Device pointer and size of an intermediate buffer inside the workspace (contents are
  * those of the last sh_forward / sh_gate_topk once the stream has drained).  Element type:
  * fp32 for SH_F32, fp16 for SH_BF16 (Q, K, V, AHAT); int32 / fp32 for the gate buffers.
+ * The offsets and lists buffers hold what the last call left there: after sh_gate_topk the
+ * per-(side, head, expert) lists that call returns; after an sh_forward with bf16 storage only
+ * what that pass's kernels needed - the source side alone, and for a k = 2 layer the tokens
+ * of a head bucketed by their PAIR of selected experts instead of by expert.
  * Testing aid: lets a failing output be traced to the stage that produced it. */
 int sh_debug_buffer(sh_layer* layer, int which, void** dev_ptr, size_t* bytes);
 
