@@ -256,6 +256,19 @@ int sh_noalloc_gate_topk(int dtype, int n_tokens, int d_model, int n_heads, int 
                          const void* x, const void* w_gate, const float* bias, int32_t* idx,
                          float* gate, int32_t* offsets, int32_t* lists, void* stream);
 
+/* Backward pass, fp32 configuration of the plain layer (sh_create + sh_configure(SH_F32): two gates,
+ * dense Q/K, no cache, no positional term; anything else: SH_ERR_UNSUPPORTED).  The paper gives no
+ * backward formulas - its training differentiates the forward equations of Sec. 2.2 automatically -
+ * so this is the chain rule for those equations with the expert selection held fixed.  Call it after
+ * sh_forward(layer, x, ...) on the SAME x (it reads the Q, K, V, Ahat, selections and gates that pass
+ * left in the workspace; otherwise SH_ERR_NOT_CONFIGURED).  dout [batch, seq, d_model] fp32 = dL/dout.
+ * Every result is a device buffer of the caller, fp32, OVERWRITTEN: dx [batch, seq, d_model]; dWq, dWk
+ * [H, d_model, d_head]; dWv [H, E, d_model, d_head]; dWo [H, E, d_head, d_model]; dWs, dWd [H, d_model, E]
+ * (the layouts sh_set_weights takes).  CUDA-core kernels with fp32 atomics: sums over tokens arrive in
+ * any order, so two calls agree to rounding, not bit for bit.  Work enqueued on `stream`. */
+int sh_backward(sh_layer* layer, const void* x, const float* dout, float* dx, float* dWq, float* dWk,
+                float* dWv, float* dWo, float* dWs, float* dWd, void* stream);
+
 /* Device pointer and size of an intermediate buffer inside the workspace (contents are
  * those of the last sh_forward / sh_gate_topk once the stream has drained).  Element type:
  * fp32 for SH_F32, fp16 for SH_BF16 (Q, K, V, AHAT); int32 / fp32 for the gate buffers.

@@ -22,7 +22,7 @@ ERROR_NAMES = {-1: "SH_ERR_INVALID_ARG", -2: "SH_ERR_UNSUPPORTED", -3: "SH_ERR_N
 BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 
 EXPORTS = ["sh_create", "sh_create_shared", "sh_create_moe_qk", "sh_create_dense", "sh_configure", "sh_configure_xl", "sh_workspace_bytes", "sh_set_workspace",
-           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_set_xl_positions", "sh_forward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
+           "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_set_xl_positions", "sh_forward", "sh_backward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
            "sh_noalloc_gate_topk", "sh_debug_buffer", "sh_last_status", "sh_status_block", "sh_clear_status", "sh_check_guards",
            "sh_selftest", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
 STAMP_KERNELS = ["gate", "sort", "qk_a", "qk_b", "v", "attn", "o"]
@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_set_weights.argtypes = [vp] * 10
     lib.sh_forward.restype = i32
     lib.sh_forward.argtypes = [vp, vp, vp, vp]
+    lib.sh_backward.restype = i32
+    lib.sh_backward.argtypes = [vp] * 11
     lib.sh_forward_timed.restype = i32
     lib.sh_forward_timed.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float)]
     lib.sh_forward_stamped.restype = i32
@@ -209,6 +211,16 @@ class Layer:
 
     def sh_selftest(self, which: int, arg: int) -> None:
         _check(lib.sh_selftest(self.handle, which, arg, _stream()))
+
+    def sh_backward(self, x: torch.Tensor, dout: torch.Tensor) -> dict:
+        """Gradients of sum(out * dout) with respect to x and every weight (fp32 configuration; call sh_forward(x) first)."""
+        d_model, H, D, E, k = self.dims
+        dev = x.device
+        z = lambda *shape: torch.empty(shape, dtype=torch.float32, device=dev)
+        g = dict(dx=z(self.batch, self.seq, d_model), dWq=z(H, d_model, D), dWk=z(H, d_model, D), dWv=z(H, E, d_model, D),
+                 dWo=z(H, E, D, d_model), dWs=z(H, d_model, E), dWd=z(H, d_model, E))
+        _check(lib.sh_backward(self.handle, _ptr(x), _ptr(dout), *[_ptr(g[n]) for n in ("dx", "dWq", "dWk", "dWv", "dWo", "dWs", "dWd")], _stream()))
+        return g
 
     def sh_gate_topk(self, x: torch.Tensor):
         d_model, H, D, E, k = self.dims

@@ -8,6 +8,7 @@
 
 #include "sh_internal.cuh"
 #include "sh_simt.cuh"
+#include "sh_backward.cuh"
 
 static thread_local char g_err[512] = "";
 
@@ -98,6 +99,8 @@ static void layout_workspace(sh_layer* L) {
   // query / key experts (sh_create_moe_qk): [H, E, D, M] like the value experts
   o.wq_e = take(L->moe_q ? HD * d.E * d.M * in : 16);
   o.wk_e = take(L->moe_k ? HD * d.E * d.M * in : 16);      // pair number of every (token, head), source side
+  // fp32 configuration: scratch of the backward pass (dQ, dK, dV, dAhat [N, H, D] and the gate gradients [2, N, H, k])
+  o.bw = take(L->dtype == SH_F32 && !L->dense ? ((size_t)4 * d.N * HD + (size_t)2 * d.N * d.H * d.k) * 4 : 16);
   o.stamps = take(sizeof(ShStampBlock));
   o.total = off;
 }
@@ -555,8 +558,53 @@ extern "C" int sh_forward(sh_layer* L, const void* x, void* out, void* stream) {
   if ((uintptr_t)x % 16 != 0 || (uintptr_t)out % 16 != 0) { sh_set_error("x and out must be 16-byte aligned"); return SH_ERR_INVALID_ARG; }
   cudaStream_t st = (cudaStream_t)stream;
   L->launches = 0;
+  L->fwd_x = x;
   if (L->dtype == SH_F32) return forward_simt<float, float>(L, SH_STAGE_ALL, x, out, st);
   return sh_tc_forward(L, x, out, st);
+}
+
+extern "C" int sh_backward(sh_layer* L, const void* x, const float* dout, float* dx, float* dWq, float* dWk, float* dWv,
+                           float* dWo, float* dWs, float* dWd, void* stream) {
+  g_err[0] = 0;
+  int rc = check_ready(L);
+  if (rc != SH_OK) return rc;
+  if (L->dtype != SH_F32 || L->dense || L->d.sides != 2 || L->d.Tc > 0 || L->rope || L->xl_positions || L->moe_q || L->moe_k) {
+    sh_set_error("sh_backward serves the fp32 configuration of the plain layer (two gates, dense Q/K, no cache, no positional term)");
+    return SH_ERR_UNSUPPORTED;
+  }
+  if (!x || !dout || !dx || !dWq || !dWk || !dWv || !dWo || !dWs || !dWd) { sh_set_error("sh_backward: NULL argument"); return SH_ERR_INVALID_ARG; }
+  if (L->fwd_x != x) { sh_set_error("sh_backward needs the intermediates of sh_forward on the same x: call sh_forward(layer, x, ...) first"); return SH_ERR_NOT_CONFIGURED; }
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t nhd = (size_t)d.N * d.H * d.D;
+  ShBwArgs a{};
+  a.d = d; a.x = (const float*)x; a.dy = dout;
+  a.q = (const float*)(ws + L->o.q); a.k = (const float*)(ws + L->o.k); a.v = (const float*)(ws + L->o.v);
+  a.ahat = (const float*)(ws + L->o.ahat);
+  a.idx = (const int*)(ws + L->o.idx); a.gate = (const float*)(ws + L->o.gate);
+  a.wqk = (const float*)(ws + L->o.wqk); a.wv = (const float*)(ws + L->o.wv); a.wo = (const float*)(ws + L->o.wo);
+  a.wgate = (const float*)(ws + L->o.wgate);
+  float* scratch = (float*)(ws + L->o.bw);
+  a.dq = scratch; a.dk = scratch + nhd; a.dv = scratch + 2 * nhd; a.dahat = scratch + 3 * nhd; a.dgate = scratch + 4 * nhd;
+  a.dx = dx; a.dWq = dWq; a.dWk = dWk; a.dWv = dWv; a.dWo = dWo; a.dWs = dWs; a.dWd = dWd;
+  SH_CUDA_CHECK(cudaMemsetAsync(a.dk, 0, 2 * nhd * 4, st));                                   // dK, dV: summed by atomics
+  SH_CUDA_CHECK(cudaMemsetAsync(dx, 0, (size_t)d.N * d.M * 4, st));
+  SH_CUDA_CHECK(cudaMemsetAsync(dWq, 0, (size_t)d.H * d.M * d.Dt * 4, st));
+  SH_CUDA_CHECK(cudaMemsetAsync(dWk, 0, (size_t)d.H * d.M * d.Dt * 4, st));
+  SH_CUDA_CHECK(cudaMemsetAsync(dWv, 0, (size_t)d.H * d.E * d.M * d.Dt * 4, st));
+  SH_CUDA_CHECK(cudaMemsetAsync(dWo, 0, (size_t)d.H * d.E * d.Dt * d.M * 4, st));
+  SH_CUDA_CHECK(cudaMemsetAsync(dWs, 0, (size_t)d.H * d.M * d.E * 4, st));
+  SH_CUDA_CHECK(cudaMemsetAsync(dWd, 0, (size_t)d.H * d.M * d.E * 4, st));
+  sh_bw_o_kernel<<<d.N * d.H, 128, 0, st>>>(a);
+  const long rows = (long)d.B * d.H * d.T;
+  sh_bw_attn_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(a);
+  sh_bw_v_kernel<<<d.N * d.H, 128, 0, st>>>(a);
+  sh_bw_qk_kernel<<<d.N, 128, (size_t)2 * d.H * d.D * 4, st>>>(a);
+  sh_bw_gate_kernel<<<d.N, 128, 0, st>>>(a);
+  SH_CUDA_CHECK(cudaGetLastError());
+  L->launches = 5;
+  return SH_OK;
 }
 
 extern "C" int sh_forward_timed(sh_layer* L, const void* x, void* out, void* stream, float* stage_ms) {

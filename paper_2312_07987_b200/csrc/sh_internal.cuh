@@ -89,7 +89,7 @@ __device__ __forceinline__ void sh_stamp_end(unsigned long long* s, int k) { if 
 
 struct ShWorkspace {
   size_t status, wqk, wgate, gbias, wv, wo, q, k, v, ahat, idx, gate, blockcnt, blockoff,
-         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, gid, wq_e, wk_e, stamps, total;
+         offsets, lists, lgate, tiles, ntiles, rope, vearly, vearly_cnt, xl_emb, xl_r, xl_uv, xl_r16, xl_vr, xl_uk, xl_bias, wos, gid, wq_e, wk_e, bw, stamps, total;
 };
 
 // Words of the 256-byte status block at the start of the workspace.
@@ -115,6 +115,7 @@ struct sh_layer {
   size_t ws_bytes = 0;
   ShWorkspace o{};
   bool weights_set = false;
+  const void* fwd_x = nullptr;   // input of the last forward pass (sh_backward wants the same one)
   bool rope = false;       // rotary position embeddings on Q, K (table in the workspace)
   bool xl_positions = false;   // Transformer-XL relative-position term (fp32 configuration; tables in the workspace)
   int launches = 0;
