@@ -316,7 +316,7 @@ int sh_selftest(sh_layer* layer, int which, uint64_t arg, void* stream);
  * index read from memory is range-checked before it is used (a failed check records SH_ERR_BOUNDS
  * and the access is skipped), and launch-structure switches are read from the environment when the
  * weights are set (SH_NO_PDL, SH_NO_OVERLAP, SH_QK_ONE_GRID, SH_QK_SINGLE, SH_O_SINGLE,
- * SH_NO_PERSISTENT, SH_SORT_SEPARATE, SH_ATTN_ADJACENT, SH_SIMT_STAGES: A/B and test aids).
+ * SH_NO_PERSISTENT, SH_SORT_SEPARATE, SH_NO_FRONT, SH_ATTN_ADJACENT, SH_SIMT_STAGES: A/B and test aids).
  * 0 for the release library, which has neither. */
 int sh_is_debug_build(void);
 

@@ -99,6 +99,7 @@ enum {
   SH_ST_BOUNDS = 8,       // 8..11: the first failed index check of a debug build (site, value, limit, block)
   SH_ST_SCHED = 16,       // 16, 17: tile counter and finished-claimer counter of the dense Q/K projection
   SH_ST_GRIDBAR = 24,     // 24, 25: grid barrier of the fused gate + sort kernel
+  SH_ST_SORTED = 26,      // one-grid front: 128-token blocks whose selections, list entries and tiles are in memory
   SH_ST_GUARD_BAD = 32    // damaged guard words counted by sh_check_guards
 };
 

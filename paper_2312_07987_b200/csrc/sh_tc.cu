@@ -16,6 +16,7 @@
 #include "sh_tc_xlbias.cuh"
 #include "sh_tc_oproj_sp.cuh"
 #include "sh_tc_vpair.cuh"
+#include "sh_tc_front.cuh"
 
 using namespace shtc;
 
@@ -77,17 +78,38 @@ static int encode_3d_f16(CUtensorMap* map, const void* base, uint64_t inner, uin
   return SH_OK;
 }
 
+// The same tensor in boxes of 32 rows of 32 elements with the 64-byte swizzle: the tiles one epilogue
+// warp of the one-grid front stores.
+static int encode_3d_f16_store32(CUtensorMap* map, const void* base, uint64_t inner, uint64_t n1, uint64_t n2) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { sh_set_error("cuTensorMapEncodeTiled is not available from the driver"); return SH_ERR_CUDA; }
+  cuuint64_t dims[3] = {inner, n1, n2};
+  cuuint64_t strides[2] = {inner * 2, inner * n1 * 2};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { sh_set_error("cuTensorMapEncodeTiled (3-D, store) failed with CUresult %d", (int)r); return SH_ERR_CUDA; }
+  return SH_OK;
+}
+
 struct TcState {
   CUtensorMap map_q, map_k, map_v;
+  CUtensorMap map_q_st, map_k_st;   // Q and K as the one-grid front's epilogue stores them
   CUtensorMap map_wqk, map_wqk128, map_wv, map_wq_e, map_wk_e, map_wo, map_wo256, map_wos, map_ahat, map_wgate;
   CUtensorMap map_q2d, map_r16;  // score-bias GEMM of the Transformer-XL position term: Q as [B*H*T, D], R16 as [H*T, D]
   CUtensorMap map_x;             // tensor map of the last x pointer seen (x_cached)
+  CUtensorMap map_x64;           // the same tensor in 64-token boxes (gate tile of the one-grid front, 64 tokens per CTA)
+  CUtensorMap map_wgate_half;    // gate weights in boxes of gate_gp / 2 rows (each CTA of a pair loads half)
   const void* x_cached = nullptr;
   int gate_gp;          // gate columns padded to a multiple of 16; 0 = CUDA-core gate kernel (more than 256 gate columns)
   int qk_bn;            // column tile of the dense projection: 256 (CTA pairs / persistent) when 2*H*D allows, else 128
   int o_pairs_max;      // clusters of the CTA-pair output projection the device holds at once (0: not asked yet, -1: none)
   int qk_pairs_max;     // the same for the dense Q/K projection
   int gate_coop;        // 1: the gate kernel can be launched cooperatively (fused sort), -1: it cannot
+  int front = 0;        // one-grid front (sh_tc_front_kernel): 0 = not asked yet, 1 = usable, -1 = not
+  int front_stages = 0, front_smem = 0, front_pairs = 0, front_sort_bytes = 0;
   // Launch-structure switches.  The release library fixes them here; a library built with SH_DEBUG
   // reads them from the environment once, in sh_tc_prepare, for A/B runs and for the tests that
   // drive the less-travelled launch paths.
@@ -101,6 +123,7 @@ struct TcState {
   bool o_sparse = true;     // sparse-A CTA-pair output projection where the shape allows (sh_o_sparse_ok)
   bool persistent = true;   // persistent Q/K and value-expert GEMMs (else one CTA per tile)
   bool fused_sort = true;   // sort fused into the gate kernel when it needs at most half of the SMs
+  bool one_grid_front = true;   // gate, selection, sort and the dense Q/K projection as one cooperative grid where the shape allows
   bool attn_balanced = true;
   int simt_mask = 0;        // SH_DEBUG only: stages forced onto the CUDA-core kernels
   cudaStream_t side = nullptr, side2 = nullptr;   // Q/K grids A and B
@@ -216,6 +239,7 @@ int sh_tc_prepare(sh_layer* L) {
   S->v_pairs = !getenv("SH_V_BY_EXPERT");
   S->persistent = !getenv("SH_NO_PERSISTENT");
   S->fused_sort = !getenv("SH_SORT_SEPARATE");
+  S->one_grid_front = !getenv("SH_NO_FRONT");
   S->attn_balanced = !getenv("SH_ATTN_ADJACENT");
   if (const char* env = getenv("SH_SIMT_STAGES")) S->simt_mask = atoi(env);   // bit mask gate=1, qk=2, v=4, attention=8, o=16
 #endif
@@ -266,10 +290,13 @@ int sh_tc_prepare(sh_layer* L) {
   if (!L->dense && (d.G + 15) / 16 * 16 <= 256) {
     S->gate_gp = (d.G + 15) / 16 * 16;
     if ((rc = sh_tc_encode_2d(&S->map_wgate, 0, ws + L->o.wgate, d.M, d.G, (uint64_t)d.M * 2, 64, S->gate_gp))) return rc;
+    if ((rc = sh_tc_encode_2d(&S->map_wgate_half, 0, ws + L->o.wgate, d.M, d.G, (uint64_t)d.M * 2, 64, S->gate_gp / 2))) return rc;
   }
   if ((rc = encode_3d_f16(&S->map_q, ws + L->o.q, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = encode_3d_f16(&S->map_k, ws + L->o.k, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = encode_3d_f16(&S->map_v, ws + L->o.v, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
+  if ((rc = encode_3d_f16_store32(&S->map_q_st, ws + L->o.q, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
+  if ((rc = encode_3d_f16_store32(&S->map_k_st, ws + L->o.k, d.D, d.T, (uint64_t)d.B * d.H))) return rc;
   if ((rc = sh_tc_encode_2d(&S->map_ahat, 1, ws + L->o.ahat, HD, d.N, (uint64_t)HD * 2, 64, 128))) return rc;
   if (!L->dense && d.Tc > 0) {
     if ((rc = sh_tc_encode_2d(&S->map_q2d, 1, ws + L->o.q, d.D, (uint64_t)d.B * d.H * d.T, (uint64_t)d.D * 2, 64, 128))) return rc;
@@ -285,6 +312,7 @@ static int x_map(sh_layer* L, const void* x, const CUtensorMap** out) {
   if (S->x_cached != x) {
     const ShDims& d = L->d;
     if (int rc = sh_tc_encode_2d(&S->map_x, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 128)) return rc;
+    if (int rc = sh_tc_encode_2d(&S->map_x64, 0, x, d.M, d.N, (uint64_t)d.M * 2, 64, 64)) return rc;
     S->x_cached = x;
   }
   *out = &S->map_x;
@@ -433,6 +461,107 @@ static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const T
   return SH_OK;
 }
 
+// ---- one-grid front ------------------------------------------------------------------------------
+// Whether sh_tc_front_kernel serves this layer's forward passes, decided once per prepared layer: the
+// plain bf16 layer with dense Q/K whose projection width is a multiple of 256, at most two 128-token
+// blocks per CTA pair the device holds, shared memory for the operand ring plus the selection's
+// scratch (six ring stages, else five), and a device that launches clusters cooperatively.
+static bool front_plan(sh_layer* L) {
+  TcState* S = (TcState*)L->tc;
+  if (S->front != 0) return S->front > 0;
+  S->front = -1;
+  const ShDims& d = L->d;
+  if (!S->one_grid_front || L->dense || L->moe_q || L->moe_k || S->simt_mask || !S->gate_gp || S->qk_bn != 256 ||
+      !S->persistent || !S->qk_pair)
+    return false;
+  const bool vp = use_v_pairs(L);
+  ShDims ds = d;
+  ds.sides = 1;
+  if (vp) { ds.sides = 1; ds.E = sh_pair_count(d.E); ds.k = 1; ds.G = d.H * ds.E; }
+  const int GH = vp ? ds.G : d.G;
+  S->front_sort_bytes = (int)(vp ? sh_sort_smem_bytes(ds) : sh_sort_smem_bytes(d));
+  int dev = 0, coop = 0, optin = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || !coop) {
+    cudaGetLastError();
+    return false;
+  }
+  // (five ring stages: six measured the same, and the sixth's 32 KB hold the epilogue's staging tiles and
+  //  the selection's scratch)
+  S->front_stages = 5;
+  S->front_smem = FrontSmem<5>::total(S->gate_gp, GH, S->front_sort_bytes);
+  if (S->front_smem > optin) return false;
+  if (set_smem(sh_tc_front_kernel<5>, S->front_smem) != SH_OK) return false;
+  int pairs = max_pairs(sh_tc_front_kernel<5>, FRONT_THREADS, S->front_smem);
+  if (pairs > L->sm_count / 2) pairs = L->sm_count / 2;
+  if (pairs <= 0 || d.nblk > 2 * pairs) return false;
+  S->front_pairs = pairs;
+  S->front = 1;
+  return true;
+}
+
+// Launches the one-grid front on `st`.  A device that refuses the cooperative cluster launch turns
+// the plan off (the caller then takes the separate kernels).
+static int tc_front(sh_layer* L, const void* x, cudaStream_t st) {
+  TcState* S = (TcState*)L->tc;
+  const ShDims& d = L->d;
+  char* ws = L->ws;
+  const int HD = d.H * d.D;
+  int rc;
+  const CUtensorMap* map_x;
+  if ((rc = x_map(L, x, &map_x))) return rc;
+  int* status = (int*)(ws + L->o.status);
+  TcFrontArgs fa{};
+  TcGemmArgs& q = fa.q;
+  q.d = d; q.K = d.M; q.ncols = 2 * HD; q.nrows = d.N;
+  q.out0 = ws + L->o.q; q.out1 = ws + L->o.k; q.out2 = ws + L->o.v;
+  q.qscale = 1.4426950408889634f / sqrtf((float)d.Dt);
+  q.b_row0 = 0;
+  q.status = status; q.sched = status + SH_ST_SCHED; q.claimers = 0;
+  q.rope = L->rope ? (const float2*)(ws + L->o.rope) : nullptr;
+  q.stamp_id = SH_K_QK_A;
+  TcGateArgs& g = fa.g;
+  g.d = d; g.Gp = S->gate_gp; g.gbias = (const float*)(ws + L->o.gbias);
+  g.idx = (int*)(ws + L->o.idx); g.gate = (float*)(ws + L->o.gate);
+  g.blockcnt = (int*)(ws + L->o.blockcnt);
+  const bool vp = use_v_pairs(L);
+  g.vpairs = vp ? 1 : 0;
+  g.NP = sh_pair_count(d.E); g.GH = vp ? d.H * g.NP : d.G; g.gid = (int*)(ws + L->o.gid);
+  g.zero_v = vp ? nullptr : (void*)(ws + L->o.v);          // (the pair-tiled kernel stores every value row once)
+  g.zero_out = nullptr;
+  g.status = status;
+  g.fused = 1;
+  g.sort_sides = 1;                                        // only the value experts read sorted lists in a forward pass
+  g.tile_rows_src = vp ? 256 : d.tile_rows_src;
+  g.max_tiles = d.max_tiles;
+  g.offsets = (int*)(ws + L->o.offsets); g.lists = (int*)(ws + L->o.lists); g.lgate = (float*)(ws + L->o.lgate);
+  g.tiles = (ShTile*)(ws + L->o.tiles); g.ntiles = (int*)(ws + L->o.ntiles);
+  g.gridbar = status + SH_ST_GRIDBAR;
+  fa.R = d.nblk <= S->front_pairs ? 64 : 128;
+  fa.gate_pairs = fa.R == 64 ? d.nblk : (d.nblk + 1) / 2;
+  fa.sort_bytes = S->front_sort_bytes;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2u * (unsigned)S->front_pairs); cfg.blockDim = dim3(FRONT_THREADS);
+  cfg.dynamicSmemBytes = (size_t)S->front_smem; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;
+  attr[1].val.cooperative = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  const CUtensorMap& map_g = fa.R == 64 ? S->map_x64 : *map_x;
+  fa.tma_epi = d.T % 32 == 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, sh_tc_front_kernel<5>, *map_x, map_g, S->map_wqk128, S->map_wgate_half, S->map_q_st, S->map_k_st, fa);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    S->front = -1;
+    sh_set_error("cooperative cluster launch of the one-grid front failed: %s", cudaGetErrorString(e));
+    return SH_ERR_CUDA;
+  }
+  L->launches += 1;
+  return SH_OK;
+}
+
 using QkPS = QkPairSmem<6>;
 
 // Clusters of the CTA-pair Q/K kernel the device holds at once (looked up once per layer; -1: none).
@@ -447,7 +576,7 @@ static int qk_pairs_max(TcState* S) {
 
 // The launches of one forward pass after grid A of a split Q/K projection is out (see sh_tc_forward).
 static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t st, const CUtensorMap& map_x, bool overlap,
-                           int qkA, int qkB, TcGemmArgs& qg);
+                           int qkA, int qkB, TcGemmArgs& qg, bool front);
 
 int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   TcState* S = (TcState*)L->tc;
@@ -461,7 +590,15 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
 
   sh_mark(L, 0, st);
   // stage-timed runs (sh_forward_timed) stay serial so that the stage boundaries mean something
-  const bool overlap = S->side && !L->ev && !(simt & SH_STAGE_QK);
+  // one grid for gate, selection, sort and Q/K where the shape allows; otherwise (and on a device that
+  // refuses the launch) the separate kernels below
+  bool front = false;
+  if (!L->ev && front_plan(L)) {
+    rc = tc_front(L, x, st);
+    if (rc == SH_OK) front = true;
+    else if (S->front > 0) return rc;
+  }
+  const bool overlap = S->side && !L->ev && !(simt & SH_STAGE_QK) && !front;
   if (overlap) {
     SH_CUDA_CHECK(cudaEventRecord(S->ev_fork, st));
     SH_CUDA_CHECK(cudaStreamWaitEvent(S->side, S->ev_fork, 0));
@@ -496,7 +633,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
   }
   // a layer with query (key) experts projects only its keys (queries) densely; with both, nothing
   const int qk_ncols = (L->moe_q || L->moe_k) ? HD : 2 * HD;
-  if (overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_bn == 256 && S->persistent && S->qk_pair &&
+  if (!front && overlap && !L->dense && !(simt & SH_STAGE_GATE) && S->gate_gp && S->qk_bn == 256 && S->persistent && S->qk_pair &&
       S->qk_two_grids && qk_pairs_max(S) > 0 && !(L->moe_q && L->moe_k)) {
     const int ptiles = ((d.N + 255) / 256) * ((qk_ncols + 255) / 256);
     const int pairs = ptiles < S->qk_pairs_max ? ptiles : S->qk_pairs_max;
@@ -518,7 +655,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
     if ((rc = launch_k_pairs(false, sh_tc_qk_pair_kernel<6>, dim3(2 * qkA), dim3(320), QkPS::TOTAL, S->side, *map_x, S->map_wqk128, qg))) return rc;
     L->launches += 1;
   }
-  rc = tc_forward_rest(L, x, out, st, *map_x, overlap, qkA, qkB, qg);
+  rc = tc_forward_rest(L, x, out, st, *map_x, overlap, qkA, qkB, qg, front);
   if (rc != SH_OK && qkA > 0) {
     // Grid A is out and something after it could not be launched: the tile counter it shares with
     // grid B would keep this pass's claims, and the caller's stream would never join the side
@@ -532,7 +669,7 @@ int sh_tc_forward(sh_layer* L, const void* x, void* out, cudaStream_t st) {
 }
 
 static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t st, const CUtensorMap& map_x, bool overlap,
-                           int qkA, int qkB, TcGemmArgs& qg) {
+                           int qkA, int qkB, TcGemmArgs& qg, bool front) {
   TcState* S = (TcState*)L->tc;
   const ShDims& d = L->d;
   char* ws = L->ws;
@@ -541,7 +678,7 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
   const int simt = S->simt_mask;
   int* status = (int*)(ws + L->o.status);
   const bool pdl = S->pdl && !L->ev;                       // stage-timed runs use ordinary launches
-  if (!L->dense) {
+  if (!L->dense && !front) {
     if ((rc = tc_gate_sort(L, x, out, true, st, qkA > 0))) return rc;
   }
   sh_mark(L, 1, st);
@@ -553,8 +690,8 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     L->launches += 1;
   }
   // ---- Q, K (and V for the dense comparator) ------------------------------------------------
-  if (qkA > 0) {
-    // (launched above, as two grids)
+  if (qkA > 0 || front) {
+    // (launched above: as two grids, or inside the one-grid front)
   } else if (simt & SH_STAGE_QK) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_QK, x, out, st))) return rc;
   } else if (L->moe_q && L->moe_k) {
@@ -606,7 +743,10 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
       const int bound = (d.N * d.H + 255) / 256 + d.H * sh_pair_count(d.E);       // tiles: at most this many
       const unsigned pgrid = 2u * (unsigned)(bound < S->v_pairs_max ? bound : S->v_pairs_max);
       g.scale = 0.f; g.stamp_id = SH_K_V;
+      // (behind the one-grid front: wait for the sort's counter, not for the grid - see sh_tc_vpair_kernel)
+      if (front && pdl) { g.ready = status + SH_ST_SORTED; g.ready_count = d.nblk; }
       if ((rc = launch_k_pairs(pdl, sh_tc_vpair_kernel<6>, dim3(pgrid), dim3(320), VPS::TOTAL, st, S->map_wv, g))) return rc;
+      g.ready = nullptr;
       L->launches += 1;
       // key / query experts: the same kernel with the key (query) experts' weights, the source
       // (destination) side's pair tiles and gates, into the K (Q) buffer; queries carry the score scale

@@ -40,6 +40,8 @@ struct TcVPairArgs {
   __half* v;                 // [B, H, T, D]: the projection's result (V; K or Q of a layer with key / query experts)
   float scale;               // extra factor on the result (the queries' log2(e)/sqrt(d_head)); 0 = none
   int stamp_id;              // SH_K_V, or -1: no stamps (the key / query launches)
+  const int* ready;          // nullptr, or a counter that reaches ready_count when lists, tiles, idx and gate are complete:
+  int ready_count;           //   the kernel then waits for the counter at its start and for the grid before it only at its end
   int* status;
 };
 
@@ -87,12 +89,34 @@ sh_tc_vpair_kernel(const __grid_constant__ CUtensorMap mapW, TcVPairArgs g) {
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
   if (threadIdx.x == 0 && g.stamp_id >= 0) sh_stamp_resident(d.stamps, g.stamp_id);
-  pdl_wait();                                              // the sorted lists and the tile table
+  if (g.ready) {
+    // The kernel before this one (the one-grid front) is wholly resident before any CTA of this one
+    // exists, so waiting for its counter cannot starve it.  Bounded like every wait.
+    if (threadIdx.x == 0) {
+      const uint64_t t0 = global_timer_ns();
+      int seen;
+      do {
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(g.ready) : "memory");
+        if (seen >= g.ready_count) break;
+        if (global_timer_ns() - t0 > SH_WAIT_LIMIT_NS || *(volatile int*)g.status != 0) {
+          if (atomicCAS(g.status, 0, SH_ERR_TIMEOUT) == 0) {
+            g.status[1] = (int)blockIdx.x; g.status[2] = 0; g.status[3] = -1;
+            g.status[4] = seen; g.status[5] = (int)gridDim.x; g.status[6] = (int)blockDim.x;
+          }
+          break;
+        }
+      } while (true);
+    }
+    __syncthreads();
+    if (*(volatile int*)g.status != 0) dead = true;
+  } else {
+    pdl_wait();                                            // the sorted lists and the tile table
+  }
   if (threadIdx.x == 0 && g.stamp_id >= 0) sh_stamp_start(d.stamps, g.stamp_id);
   // (the first tile's entry is fetched beside the tile count, not behind it: every dependent trip to L2
   //  costs this kernel's start 2-3 us while the Q/K projection's operand traffic keeps L2 busy)
   const ShTile tile_first = g.tiles[pair];                // (the table has room for every pair's index)
-  const int ntiles = *g.ntiles;
+  const int ntiles = dead ? 0 : *g.ntiles;
   const int NP = sh_pair_count(d.E);
   auto tile_of = [&](int t) -> ShTile {
     ShTile tl = t == pair ? tile_first : g.tiles[t];
@@ -248,6 +272,7 @@ sh_tc_vpair_kernel(const __grid_constant__ CUtensorMap mapW, TcVPairArgs g) {
       }
     }
   }
+  pdl_wait();                                              // (the next kernel's wait for this grid then covers the grid before it)
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();

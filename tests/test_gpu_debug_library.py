@@ -24,7 +24,12 @@ def run_case(case, extra_env=None):
 
 @pytest.mark.parametrize("env", [{}, {"SH_NO_PDL": "1"}, {"SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_PERSISTENT": "1"},
                                  {"SH_ATTN_ADJACENT": "1"}, {"SH_O_SINGLE": "1"}, {"SH_O_MASKED": "1"}, {"SH_V_BY_EXPERT": "1"}, {"SH_QK_SINGLE": "1"}, {"SH_QK_ONE_GRID": "1"},
-                                 {"SH_SORT_SEPARATE": "1"}, {"SH_SIMT_STAGES": "31"}],
+                                 {"SH_SORT_SEPARATE": "1"}, {"SH_SIMT_STAGES": "31"},
+                                 # the launch structure without the one-grid front (gate + sort and Q/K as kernels of their own)
+                                 {"SH_NO_FRONT": "1"}, {"SH_NO_FRONT": "1", "SH_NO_PDL": "1"},
+                                 {"SH_NO_FRONT": "1", "SH_NO_PDL": "1", "SH_NO_OVERLAP": "1"}, {"SH_NO_FRONT": "1", "SH_QK_SINGLE": "1"},
+                                 {"SH_NO_FRONT": "1", "SH_QK_ONE_GRID": "1"}, {"SH_NO_FRONT": "1", "SH_SORT_SEPARATE": "1"},
+                                 {"SH_NO_FRONT": "1", "SH_NO_PERSISTENT": "1"}],
                          ids=lambda e: "+".join(sorted(e)) or "default")
 def test_launch_structure_switches_keep_the_result(env):
     run_case("switches", env)
@@ -34,6 +39,7 @@ def test_sparse_output_projection_shapes_with_index_checks_and_against_the_maske
     run_case("sparse_o")
     run_case("sparse_o", {"SH_O_MASKED": "1"})
     run_case("sparse_o", {"SH_V_BY_EXPERT": "1"})
+    run_case("sparse_o", {"SH_NO_FRONT": "1"})
 
 
 def test_key_and_query_experts_with_index_checks():
