@@ -123,7 +123,7 @@ struct TcState {
   bool o_sparse = true;     // sparse-A CTA-pair output projection where the shape allows (sh_o_sparse_ok)
   bool persistent = true;   // persistent Q/K and value-expert GEMMs (else one CTA per tile)
   bool fused_sort = true;   // sort fused into the gate kernel when it needs at most half of the SMs
-  bool one_grid_front = true;   // gate, selection, sort and the dense Q/K projection as one cooperative grid where the shape allows
+  bool one_grid_front = true;   // gate, selection, sort and the dense Q/K projection as one grid where the shape allows
   bool attn_balanced = true;
   int simt_mask = 0;        // SH_DEBUG only: stages forced onto the CUDA-core kernels
   cudaStream_t side = nullptr, side2 = nullptr;   // Q/K grids A and B
@@ -465,7 +465,7 @@ static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const T
 // Whether sh_tc_front_kernel serves this layer's forward passes, decided once per prepared layer: the
 // plain bf16 layer with dense Q/K whose projection width is a multiple of 256, at most two 128-token
 // blocks per CTA pair the device holds, shared memory for the operand ring plus the selection's
-// scratch (six ring stages, else five), and a device that launches clusters cooperatively.
+// scratch, and a device that holds all of the grid's CTA pairs at once.
 static bool front_plan(sh_layer* L) {
   TcState* S = (TcState*)L->tc;
   if (S->front != 0) return S->front > 0;
@@ -480,9 +480,8 @@ static bool front_plan(sh_layer* L) {
   if (vp) { ds.sides = 1; ds.E = sh_pair_count(d.E); ds.k = 1; ds.G = d.H * ds.E; }
   const int GH = vp ? ds.G : d.G;
   S->front_sort_bytes = (int)(vp ? sh_sort_smem_bytes(ds) : sh_sort_smem_bytes(d));
-  int dev = 0, coop = 0, optin = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || !coop) {
+  int dev = 0, optin = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
     cudaGetLastError();
     return false;
   }
@@ -500,8 +499,8 @@ static bool front_plan(sh_layer* L) {
   return true;
 }
 
-// Launches the one-grid front on `st`.  A device that refuses the cooperative cluster launch turns
-// the plan off (the caller then takes the separate kernels).
+// Launches the one-grid front on `st`.  A device that refuses the launch turns the plan off (the
+// caller then takes the separate kernels).
 static int tc_front(sh_layer* L, const void* x, cudaStream_t st) {
   TcState* S = (TcState*)L->tc;
   const ShDims& d = L->d;
@@ -543,19 +542,21 @@ static int tc_front(sh_layer* L, const void* x, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2u * (unsigned)S->front_pairs); cfg.blockDim = dim3(FRONT_THREADS);
   cfg.dynamicSmemBytes = (size_t)S->front_smem; cfg.stream = st;
-  cudaLaunchAttribute attr[2];
+  // An ordinary cluster launch of no more CTA pairs than the device holds at once (front_plan asked the
+  // occupancy calculator), not a cooperative one: the profiler's counter passes fail every cooperative
+  // cluster launch on this driver.  The kernel's grid-wide barrier is a bounded wait, so CTAs that other
+  // work keeps off the SMs for longer than the limit end the pass with SH_ERR_TIMEOUT, not with a hang.
+  cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeCooperative;
-  attr[1].val.cooperative = 1;
-  cfg.attrs = attr; cfg.numAttrs = 2;
+  cfg.attrs = attr; cfg.numAttrs = 1;
   const CUtensorMap& map_g = fa.R == 64 ? S->map_x64 : *map_x;
   fa.tma_epi = d.T % 32 == 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, sh_tc_front_kernel<5>, *map_x, map_g, S->map_wqk128, S->map_wgate_half, S->map_q_st, S->map_k_st, fa);
   if (e != cudaSuccess) {
     cudaGetLastError();
     S->front = -1;
-    sh_set_error("cooperative cluster launch of the one-grid front failed: %s", cudaGetErrorString(e));
+    sh_set_error("cluster launch of the one-grid front failed: %s", cudaGetErrorString(e));
     return SH_ERR_CUDA;
   }
   L->launches += 1;

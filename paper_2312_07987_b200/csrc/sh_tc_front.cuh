@@ -17,7 +17,7 @@
 //     that selects (R = 64: the leader, across the cluster) and hand the accumulator back;
 //   * 512 selection threads of that CTA pick the top k per (token, side, head), publish the block's
 //     histogram, meet the other selecting CTAs at a grid-wide barrier (a counter in global memory,
-//     bounded wait; the launch is cooperative, so all CTAs are resident) and place the block's tokens
+//     bounded wait; the grid has no more CTA pairs than the device holds at once) and place the block's tokens
 //     (sh_sort_block); block 0 also writes offsets and the tile table;
 //   * meanwhile producers, issuer and epilogue go on with 256 x 256 projection tiles claimed from a
 //     global counter, exactly as in sh_tc_qk_pair_kernel.
