@@ -465,7 +465,7 @@ static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const T
 // Whether sh_tc_front_kernel serves this layer's forward passes, decided once per prepared layer: the
 // plain bf16 layer with dense Q/K whose projection width is a multiple of 256, at most two 128-token
 // blocks per CTA pair the device holds, shared memory for the operand ring plus the selection's
-// scratch, and a device that holds all of the grid's CTA pairs at once.
+// scratch, and a device that launches cooperatively and holds all of the grid's CTA pairs at once.
 static bool front_plan(sh_layer* L) {
   TcState* S = (TcState*)L->tc;
   if (S->front != 0) return S->front > 0;
@@ -480,8 +480,9 @@ static bool front_plan(sh_layer* L) {
   if (vp) { ds.sides = 1; ds.E = sh_pair_count(d.E); ds.k = 1; ds.G = d.H * ds.E; }
   const int GH = vp ? ds.G : d.G;
   S->front_sort_bytes = (int)(vp ? sh_sort_smem_bytes(ds) : sh_sort_smem_bytes(d));
-  int dev = 0, optin = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+  int dev = 0, coop = 0, optin = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || !coop) {
     cudaGetLastError();
     return false;
   }
@@ -542,13 +543,12 @@ static int tc_front(sh_layer* L, const void* x, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2u * (unsigned)S->front_pairs); cfg.blockDim = dim3(FRONT_THREADS);
   cfg.dynamicSmemBytes = (size_t)S->front_smem; cfg.stream = st;
-  // An ordinary cluster launch of no more CTA pairs than the device holds at once (front_plan asked the
-  // occupancy calculator), not a cooperative one: the profiler's counter passes fail every cooperative
-  // cluster launch on this driver.  The kernel's grid-wide barrier is a bounded wait, so CTAs that other
-  // work keeps off the SMs for longer than the limit end the pass with SH_ERR_TIMEOUT, not with a hang.
+  // A cooperative launch (the grid's CTAs meet at a barrier: all of them have to be resident, whatever
+  // else runs on the device); the cluster shape is the kernel's own (__cluster_dims__) - given as a
+  // launch attribute beside the cooperative one, every launch failed under the profiler on this driver.
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   const CUtensorMap& map_g = fa.R == 64 ? S->map_x64 : *map_x;
   fa.tma_epi = d.T % 32 == 0;
@@ -556,7 +556,7 @@ static int tc_front(sh_layer* L, const void* x, cudaStream_t st) {
   if (e != cudaSuccess) {
     cudaGetLastError();
     S->front = -1;
-    sh_set_error("cluster launch of the one-grid front failed: %s", cudaGetErrorString(e));
+    sh_set_error("cooperative launch of the one-grid front failed: %s", cudaGetErrorString(e));
     return SH_ERR_CUDA;
   }
   L->launches += 1;

@@ -17,7 +17,7 @@
 //     that selects (R = 64: the leader, across the cluster) and hand the accumulator back;
 //   * 512 selection threads of that CTA pick the top k per (token, side, head), publish the block's
 //     histogram, meet the other selecting CTAs at a grid-wide barrier (a counter in global memory,
-//     bounded wait; the grid has no more CTA pairs than the device holds at once) and place the block's tokens
+//     bounded wait; the launch is cooperative, so all CTAs are resident) and place the block's tokens
 //     (sh_sort_block); block 0 also writes offsets and the tile table;
 //   * meanwhile producers, issuer and epilogue go on with 256 x 256 projection tiles claimed from a
 //     global counter, exactly as in sh_tc_qk_pair_kernel.
@@ -61,7 +61,7 @@ __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
 }
 
 template <int STAGES>
-__global__ void __launch_bounds__(FRONT_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FRONT_THREADS, 1)
 sh_tc_front_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapAg,
                    const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapWg,
                    const __grid_constant__ CUtensorMap mapQo, const __grid_constant__ CUtensorMap mapKo, TcFrontArgs fa) {
