@@ -453,12 +453,11 @@ static int launch_pgemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const 
 }
 
 template <int BN, int STAGES, int MODE, int A_BF16, int B_BF16, int MT = 1>
-static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, dim3 grid, cudaStream_t st) {
+static int launch_gemm(const CUtensorMap& mapA, const CUtensorMap& mapB, const TcGemmArgs& g, dim3 grid, cudaStream_t st, bool pdl = false) {
   auto kern = sh_tc_gemm_kernel<BN, STAGES, MODE, A_BF16, B_BF16, MT>;
   constexpr int smem = GemmSmem<BN, STAGES, MT>::TOTAL;
   if (int rc = set_smem(kern, smem)) return rc;
-  kern<<<grid, 192, smem, st>>>(mapA, mapB, g);
-  return SH_OK;
+  return launch_k(pdl, kern, grid, dim3(192), smem, st, mapA, mapB, g);
 }
 
 // ---- one-grid front ------------------------------------------------------------------------------
@@ -779,11 +778,11 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
       dim3 grid(d.tile_rows_src == 256 ? d.max_tiles / 2 + d.H * d.E : d.max_tiles, 1);
       if (d.tile_rows_src == 256) {
         if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 2>(map_x, S->map_wv, g, grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count, st, pdl)
-                                           : launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
-        else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st);
+                                           : launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st, pdl);
+        else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st, pdl);
       } else {
-        if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
-        else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st);
+        if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st, pdl);
+        else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st, pdl);
       }
       if (rc) return rc;
       L->launches += 1;

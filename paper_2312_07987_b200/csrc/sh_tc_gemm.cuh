@@ -118,6 +118,7 @@ sh_tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constan
   const ShDims& d = g.d;
   int th = 0, te = 0, row0, nrows;
   if (GATHER) {
+    pdl_wait();                                        // (a no-op in an ordinary launch) the tile table and the lists are the kernel's before this one
     if ((int)blockIdx.x >= *g.ntiles) return;          // whole CTA leaves before any barrier
     const ShTile tl = tile_checked(g.tiles[blockIdx.x], d, g.status);
     th = tl.h; te = tl.e; row0 = tl.row0; nrows = tl.nrows;
