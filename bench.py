@@ -353,9 +353,30 @@ def measure_config(cfg, args, rank, world, peaks, flush, barrier, steps, min_sec
         b.record(pipe.s_out)
         pipe.wait()
         barrier()
-        res["e2e_ms"] = a.elapsed_time(b)
+        res["e2e_ms_f32_result"] = a.elapsed_time(b)
         res["h2d"] = int(x.numel() * x.element_size())
-        res["d2h"] = int(out.numel() * 4)
+        res["d2h_f32_result"] = int(out.numel() * 4)
+        # the same with the result rounded to fp16 on its way out of the output projection (sh_set_output_f16):
+        # half the bytes on the way back, which is what bounds a host-fed step
+        layer.sh_set_output_f16(True)
+        outh16 = [torch.empty(inp.x.shape, dtype=torch.float16).pin_memory() for _ in range(2)]
+        pipe16 = pipeline.HostFedLayer(layer, x)
+        for i in range(4):
+            pipe16.step(xh[i & 1], outh16[i & 1])
+        pipe16.wait()
+        r16 = ref.to(torch.float16)
+        assert torch.equal(outh16[1], r16) or float((outh16[1].float() - ref).abs().max()) < 1e-2 * float(ref.abs().max()), \
+            "pipelined fp16 result differs from the direct one"
+        barrier()
+        a.record(pipe16.s_in)
+        for i in range(steps):
+            pipe16.step(xh[i & 1], outh16[i & 1])
+        b.record(pipe16.s_out)
+        pipe16.wait()
+        barrier()
+        res["e2e_ms"] = a.elapsed_time(b)
+        res["d2h"] = int(out.numel() * 2)
+        layer.sh_set_output_f16(False)
     assert layer.sh_last_status() == 0, "device status word set during the timed region"
     res["inp"], res["x"], res["out"] = inp, x, out
     layer.close()
@@ -413,8 +434,8 @@ def main():
 
     # ---- max over ranks (every repeat mean, so that the median is of the slowest rank's times) ----
     nrep = int(sharding.max_over_ranks([-float(len(m["repeat_means"]))], device="cuda")[0] * -1)   # fewest repeats any rank made
-    reduced = sharding.max_over_ranks(m["repeat_means"][:nrep] + [m["e2e_ms"], m["warm_ms"]], device="cuda")
-    repeat_means, e2e_ms, warm_ms = reduced[:nrep], reduced[nrep], reduced[nrep + 1]
+    reduced = sharding.max_over_ranks(m["repeat_means"][:nrep] + [m["e2e_ms"], m["warm_ms"], m["e2e_ms_f32_result"]], device="cuda")
+    repeat_means, e2e_ms, warm_ms, e2e_ms_f32 = reduced[:nrep], reduced[nrep], reduced[nrep + 1], reduced[nrep + 2]
 
     line = None
     if rank == 0:
@@ -444,7 +465,10 @@ def main():
             "gpu_launches": m["launches"] * args.steps * len(repeat_means),
             "launches_per_step": m["launches"],
             "e2e": {"value": world * N * args.steps / (e2e_ms * 1e-3), "unit": "tokens/s",
-                    "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
+                    "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"],
+                    "result_dtype": "f16 (sh_set_output_f16: the fp32 result rounded once by the output projection's epilogue)",
+                    "with_f32_result": {"value": world * N * args.steps / (e2e_ms_f32 * 1e-3), "unit": "tokens/s",
+                                        "d2h_bytes_per_step": m["d2h_f32_result"]}},
             "roofline": roofline_from_timeline(cfg, tl, fl, peaks),
             "clocks": clocks,
         }

@@ -312,6 +312,15 @@ int sh_check_guards(sh_layer* layer, void* stream);
  * Enqueues one kernel on `stream`. */
 int sh_selftest(sh_layer* layer, int which, uint64_t arg, void* stream);
 
+/* Output precision of sh_forward for a layer configured with bf16 storage (Sec. 2.2, the MoE output
+ * equation is summed in fp32 on chip either way): enable != 0 makes every later sh_forward (and
+ * sh_forward_stamped / sh_forward_timed) write `out` as IEEE fp16 [batch, seq_out, d_model] - each
+ * fp32 result rounded once, to nearest even - instead of fp32; the buffer is then half the size and
+ * must still be 16-byte aligned.  A host-fed caller halves its device-to-host bytes this way.
+ * Host call, no launch.  SH_ERR_UNSUPPORTED for the fp32 configuration and the dense comparator;
+ * sh_backward and the fp32 configuration always use fp32. */
+int sh_set_output_f16(sh_layer* layer, int enable);
+
 /* 1 if the library was built with -DSH_DEBUG: every token-list entry, tile-table field and expert
  * index read from memory is range-checked before it is used (a failed check records SH_ERR_BOUNDS
  * and the access is skipped), and launch-structure switches are read from the environment when the

@@ -24,7 +24,7 @@ BUF = dict(Q=0, K=1, V=2, AHAT=3, IDX=4, GATE=5, OFFSETS=6, LISTS=7)
 EXPORTS = ["sh_create", "sh_create_shared", "sh_create_moe_qk", "sh_create_dense", "sh_configure", "sh_configure_xl", "sh_workspace_bytes", "sh_set_workspace",
            "sh_set_weights", "sh_set_causal", "sh_set_rope", "sh_set_xl_positions", "sh_forward", "sh_backward", "sh_forward_timed", "sh_forward_stamped", "sh_gate_topk",
            "sh_noalloc_gate_topk", "sh_debug_buffer", "sh_last_status", "sh_status_block", "sh_clear_status", "sh_check_guards",
-           "sh_selftest", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
+           "sh_selftest", "sh_set_output_f16", "sh_is_debug_build", "sh_launch_count", "sh_last_error", "sh_destroy"]
 STAMP_KERNELS = ["gate", "sort", "qk_a", "qk_b", "v", "attn", "o"]
 
 
@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     lib.sh_debug_buffer.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(sz)]
     lib.sh_last_status.restype = i32
     lib.sh_last_status.argtypes = [vp, vp]
+    lib.sh_set_output_f16.restype = i32
+    lib.sh_set_output_f16.argtypes = [vp, i32]
     lib.sh_launch_count.restype = i32
     lib.sh_launch_count.argtypes = [vp]
     lib.sh_last_error.restype = ctypes.c_char_p
@@ -177,10 +179,16 @@ class Layer:
     def sh_set_rope(self, base: float) -> None:
         _check(lib.sh_set_rope(self.handle, float(base), _stream()))
 
+    def sh_set_output_f16(self, enable: bool) -> None:
+        """sh_forward writes fp16 instead of fp32 from now on (bf16 storage configuration only)."""
+        _check(lib.sh_set_output_f16(self.handle, 1 if enable else 0))
+        self.out_dtype = torch.float16 if enable else torch.float32
+
     def sh_forward(self, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         assert x.is_cuda and x.is_contiguous()
         if out is None:
-            out = torch.empty((x.shape[0], self.seq_out, x.shape[2]), dtype=torch.float32, device=x.device)
+            out = torch.empty((x.shape[0], self.seq_out, x.shape[2]), dtype=getattr(self, "out_dtype", torch.float32), device=x.device)
+        assert out.dtype == getattr(self, "out_dtype", torch.float32), "out must have the layer's output dtype (see sh_set_output_f16)"
         _check(lib.sh_forward(self.handle, _ptr(x), _ptr(out), _stream()))
         return out
 

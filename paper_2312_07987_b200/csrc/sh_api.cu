@@ -497,6 +497,18 @@ extern "C" int sh_set_causal(sh_layer* L, int causal) {
   return SH_OK;
 }
 
+extern "C" int sh_set_output_f16(sh_layer* L, int enable) {
+  g_err[0] = 0;
+  if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }
+  if (L->dtype < 0) { sh_set_error("sh_set_output_f16 needs a configured layer"); return SH_ERR_NOT_CONFIGURED; }
+  if (enable && (L->dtype != SH_BF16 || L->dense)) {
+    sh_set_error("fp16 output exists for the bf16 storage configuration of the SwitchHead layer only");
+    return SH_ERR_UNSUPPORTED;
+  }
+  L->out_f16 = enable != 0;
+  return SH_OK;
+}
+
 extern "C" int sh_set_xl_positions(sh_layer* L, const float* Wr, const float* u, const float* v, void* stream) {
   g_err[0] = 0;
   if (!L) { sh_set_error("layer is NULL"); return SH_ERR_INVALID_ARG; }

@@ -111,6 +111,7 @@ struct sh_layer {
   ShDims d{};
   bool dense = false;
   bool moe_q = false, moe_k = false;   // query / key projections are experts too (destination / source side selection)
+  bool out_f16 = false;                // sh_set_output_f16: sh_forward writes its result as fp16 (bf16 storage, tensor-core output projection)
   int dtype = -1;
   char* ws = nullptr;
   size_t ws_bytes = 0;

@@ -842,6 +842,10 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
   }
   sh_mark(L, 4, st);
   // ---- output experts ----------------------------------------------------------------------------
+  if (L->out_f16 && ((simt & SH_STAGE_O) || L->dense)) {
+    sh_set_error("fp16 output is written by the tensor-core output-expert kernels only");
+    return SH_ERR_UNSUPPORTED;
+  }
   if (simt & SH_STAGE_O) {
     if ((rc = sh_simt_run_bf16(L, SH_STAGE_O, x, out, st))) return rc;
   } else if (!L->dense) {
@@ -849,7 +853,7 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
     a.d = d;
     const size_t side1 = d.sides == 2 ? (size_t)d.N * d.H * d.k : 0;   // shared selection: the one side there is
     a.idx = (const int*)(ws + L->o.idx) + side1; a.gate = (const float*)(ws + L->o.gate) + side1;
-    a.out = (float*)out; a.status = status;
+    a.out = (float*)out; a.out_f16 = L->out_f16 ? 1 : 0; a.status = status;
     // Up to four selections per (token, head) the CTA-pair kernels serve (their builder threads keep a
     // token's selections in registers).  With more, the single-CTA kernel, which reads the selections
     // from shared memory and multiplies by the gate after the UMMA; a device that cannot hold a two-CTA

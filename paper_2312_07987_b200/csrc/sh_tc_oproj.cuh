@@ -36,11 +36,23 @@ struct TcOprojArgs {
   ShDims d;
   const int* idx;        // destination side: [N, H, k]
   const float* gate;     // destination side: [N, H, k]
-  float* out;            // [N, M]
+  float* out;            // [N, M] fp32, or (out_f16) [N, M] fp16 at the same address
+  int out_f16;           // 1: the result rows are rounded to fp16 once, on their way out
   int a_slots;           // 32 KB weight stages in the ring: 3 or 2
   int nwork;             // nblk * ceil(M / 256)
   int* status;
 };
+
+// Four consecutive features of one result row (element index elem of [N, M]): fp32, or rounded to fp16.
+__device__ __forceinline__ void oproj_put4(float* out, size_t elem, float4 v, int out_f16) {
+  if (out_f16) {
+    const __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
+    *reinterpret_cast<uint2*>(reinterpret_cast<__half*>(out) + elem) =
+        make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+  } else {
+    *reinterpret_cast<float4*>(out + elem) = v;
+  }
+}
 
 template <int D>
 struct OprojSmem {
@@ -226,7 +238,7 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
       const int col0 = fc * 256 + half * 128;
       if (ok && col0 < d.M) {
         float* stg = reinterpret_cast<float*>(sgen + stg_off) + (warp - 2) * 1024;
-        float* obase = g.out + (size_t)(row0 + q * 32) * d.M + col0;
+        const size_t obase = (size_t)(row0 + q * 32) * d.M + col0;
         const int rows_here = min(32, nrows - q * 32);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -241,8 +253,7 @@ sh_tc_oproj_kernel(const __grid_constant__ CUtensorMap mapAhat, const __grid_con
           for (int r4 = 0; r4 < 32; r4 += 4) {
             const int r = r4 + (lane >> 3), ch = lane & 7;
             if (r < rows_here)
-              *reinterpret_cast<float4*>(obase + (size_t)r * d.M + c * 32 + 4 * ch) =
-                  *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2));
+              oproj_put4(g.out, obase + (size_t)r * d.M + c * 32 + 4 * ch, *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2)), g.out_f16);
           }
         }
       }

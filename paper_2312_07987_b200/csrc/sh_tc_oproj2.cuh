@@ -50,8 +50,8 @@ struct OprojPairSmem {
 
 // One 32-column chunk of a unit's accumulator: TMEM -> registers -> 32 x 32 transpose in shared
 // memory (token-per-lane -> 128-byte row segments) -> 16-byte coalesced stores.  One warp; stg = its
-// 4 KB of staging; obase = out + (first of the warp's 32 tokens) * M + the unit's first feature.
-__device__ __forceinline__ void oproj_store_chunk(uint32_t taddr, int c, float* stg, float* obase, int M, int rows_here, bool cols_live, int lane) {
+// 4 KB of staging; obase = element index in out of (first of the warp's 32 tokens, the unit's first feature).
+__device__ __forceinline__ void oproj_store_chunk(uint32_t taddr, int c, float* stg, float* out, size_t obase, int out_f16, int M, int rows_here, bool cols_live, int lane) {
   uint32_t v[32];
   tmem_ld32(taddr + c * 32, v);
   tmem_ld_wait();
@@ -65,8 +65,7 @@ __device__ __forceinline__ void oproj_store_chunk(uint32_t taddr, int c, float* 
     for (int r4 = 0; r4 < 32; r4 += 4) {
       const int r = r4 + (lane >> 3), ch = lane & 7;
       if (r < rows_here)
-        *reinterpret_cast<float4*>(obase + (size_t)r * M + c * 32 + 4 * ch) =
-            *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2));
+        oproj_put4(out, obase + (size_t)r * M + c * 32 + 4 * ch, *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2)), out_f16);
     }
   }
 }
@@ -281,10 +280,10 @@ sh_tc_oproj_pair_kernel(const __grid_constant__ CUtensorMap mapWo, TcOprojArgs g
       const int rows_here = min(32, nout - row0 - q * 32); // <= 0: these rows are past the end
       if (!mbar_wait(&d_full[buf], (un >> 1) & 1, g.status, dead)) break;
       tc_fence_after();
-      float* obase = g.out + (size_t)(row0 + q * 32) * d.M + fc * 256;
+      const size_t obase = (size_t)(row0 + q * 32) * d.M + fc * 256;
 #pragma unroll 1
       for (int c = 0; c < 8; ++c) {
-        oproj_store_chunk(tmem + lane_off + buf * 256, c, stg, obase, d.M, rows_here, fc * 256 + c * 32 < d.M, lane);
+        oproj_store_chunk(tmem + lane_off + buf * 256, c, stg, g.out, obase, g.out_f16, d.M, rows_here, fc * 256 + c * 32 < d.M, lane);
         if (c == 7) {                                      // everything has been read: hand the accumulator back
           tc_fence_before();
           __syncwarp();

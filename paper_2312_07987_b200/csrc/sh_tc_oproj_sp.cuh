@@ -343,7 +343,7 @@ sh_tc_oproj_sp_kernel(const __grid_constant__ CUtensorMap mapWos, TcOprojArgs g,
       if (more) codes_of(w + npairs);                      // (fetched before the wait: an L2 round trip)
       if (!mbar_wait(&d_full[buf], (un >> 1) & 1, g.status, dead)) break;
       tc_fence_after();
-      float* obase = g.out + (size_t)(row0 + q * 32) * d.M + fc * 256;
+      const size_t obase = (size_t)(row0 + q * 32) * d.M + fc * 256;
       const uint32_t taddr = tmem + lane_off + buf * 256;
 #pragma unroll 1
       for (int c = 0; c < 8; ++c) {
@@ -361,8 +361,7 @@ sh_tc_oproj_sp_kernel(const __grid_constant__ CUtensorMap mapWos, TcOprojArgs g,
           for (int r4 = 0; r4 < 32; r4 += 4) {
             const int r = r4 + (lane >> 3), ch = lane & 7;
             if (r < rows_here)
-              *reinterpret_cast<float4*>(obase + (size_t)r * d.M + c * 32 + 4 * ch) =
-                  *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2));
+              oproj_put4(g.out, obase + (size_t)r * d.M + c * 32 + 4 * ch, *reinterpret_cast<const float4*>(stg + r * 32 + ((ch ^ (r & 7)) << 2)), g.out_f16);
           }
         }
         if (c == 7) {

@@ -22,7 +22,8 @@ class HostFedLayer:
         self.layer = layer
         dev = like_x.device
         self.x_dev = [torch.empty_like(like_x) for _ in range(2)]
-        self.out_dev = [torch.empty(like_x.shape, dtype=torch.float32, device=dev) for _ in range(2)]
+        # (the layer's output dtype: fp32, or fp16 after sh_set_output_f16 - half the bytes on the way back)
+        self.out_dev = [torch.empty(like_x.shape, dtype=getattr(layer, "out_dtype", torch.float32), device=dev) for _ in range(2)]
         self.s_in, self.s_compute, self.s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
         mk = lambda: [torch.cuda.Event() for _ in range(2)]
         self.ev_in, self.ev_computed, self.ev_out = mk(), mk(), mk()

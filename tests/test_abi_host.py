@@ -62,6 +62,9 @@ def test_call_order_and_argument_errors():
     assert lib.sh_set_rope(None, 10000.0, None) == -1
     assert lib.sh_set_causal(None, 0) == -1 and lib.sh_set_causal(h, 0) == 0 and lib.sh_set_causal(h, 1) == 0
     assert lib.sh_set_rope(h, 10000.0, None) == -3                   # configured, but no workspace yet
+    assert lib.sh_set_output_f16(None, 1) == -1
+    assert lib.sh_set_output_f16(h, 1) == -2                         # fp32 configuration: unsupported
+    assert lib.sh_set_output_f16(h, 0) == 0
     assert lib.sh_set_rope(h, -1.0, None) in (-3, -1)
     h2 = ctypes.c_void_p(lib.sh_create(128, 2, 32, 4, 2))
     assert lib.sh_set_rope(h2, 10000.0, None) == -3                  # not configured

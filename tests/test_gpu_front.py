@@ -101,3 +101,41 @@ def test_two_layers_run_their_passes_at_the_same_time():
         assert torch.equal(oa, ya) and torch.equal(ob, yb)
     la.close()
     lb.close()
+
+
+# (batch, seq, d_model, heads, d_head, experts, k): the 2:4-sparse output projection | the CTA-pair kernel (k = 3) |
+#  the single-CTA kernel (k = 4, 16 experts), a ragged last tile
+F16_OUT_SHAPES = [(4, 512, 1024, 4, 128, 4, 2), (6, 256, 512, 2, 64, 5, 3), (2, 515, 512, 3, 128, 16, 4)]
+
+
+@pytest.mark.parametrize("B,T,M,H,D,E,k", F16_OUT_SHAPES)
+def test_fp16_output_is_the_fp32_output_rounded_once(B, T, M, H, D, E, k):
+    cfg = inputs.LayerConfig("f16out_bf16", inputs.DTYPE_BF16, B, T, M, H, D, E, k, seed=907)
+    inp = inputs.make_inputs(cfg)
+    layer, x, y32 = pu.run_layer(inp)
+    y32 = y32.clone()
+    layer.sh_set_output_f16(True)
+    y16 = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert layer.sh_last_status() == 0 and y16.dtype == torch.float16
+    if k == 2:        # (k >= 3: the value rows are summed in arrival order, two passes differ in the last bits)
+        assert torch.equal(y16, y32.to(torch.float16))
+    ref = pu.oracle_for(inp)
+    err = pu.rel_rms_err(y16.float().cpu().numpy(), ref["y"])
+    assert err < pu.TOL_Y[cfg.dtype], f"fp16 output: max-abs error / rms = {err:.3e}"
+    layer.sh_set_output_f16(False)
+    y = layer.sh_forward(x)
+    torch.cuda.synchronize()
+    assert y.dtype == torch.float32
+    if k == 2:
+        assert torch.equal(y, y32)
+    layer.sh_check_guards()
+    layer.close()
+
+
+def test_fp16_output_is_refused_where_no_kernel_writes_it():
+    cfg = inputs.LayerConfig("f16out_f32", inputs.DTYPE_F32, 1, 64, 128, 2, 32, 4, 2, seed=908)
+    layer, x, y = pu.run_layer(inputs.make_inputs(cfg))
+    with pytest.raises(binding.SwitchHeadError):
+        layer.sh_set_output_f16(True)
+    layer.close()
