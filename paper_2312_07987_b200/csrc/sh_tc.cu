@@ -781,8 +781,10 @@ static int tc_forward_rest(sh_layer* L, const void* x, void* out, cudaStream_t s
                                            : launch_gemm<128, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st, pdl);
         else rc = launch_gemm<64, 4, GEMM_V, 1, 1, 2>(map_x, S->map_wv, g, grid, st, pdl);
       } else {
-        if (d.D == 128) rc = launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st, pdl);
-        else rc = launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st, pdl);
+        // (128-row tiles of a small workload: the persistent kernel too - one prologue per SM instead of one per tile)
+        const unsigned pg = grid.x < (unsigned)L->sm_count ? grid.x : (unsigned)L->sm_count;
+        if (d.D == 128) rc = S->persistent ? launch_pgemm<128, 4, PG_V, 1>(map_x, S->map_wv, g, pg, st, pdl) : launch_gemm<128, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st, pdl);
+        else rc = S->persistent ? launch_pgemm<64, 4, PG_V, 1>(map_x, S->map_wv, g, pg, st, pdl) : launch_gemm<64, 4, GEMM_V, 1, 1>(map_x, S->map_wv, g, grid, st, pdl);
       }
       if (rc) return rc;
       L->launches += 1;
