@@ -13,14 +13,18 @@
 //     SM pulls x from HBM), or two blocks, one per CTA (R = 128: up to 148 blocks).  cta_group::2 UMMA
 //     with M = 256, N = Gp: each CTA loads its rows of x and half of the gate weights.  With R = 64 the
 //     upper half of a CTA's operand tile is whatever the ring held: those accumulator rows are never read.
-//   * the projection's epilogue warps move the logits (plus bias) into the shared memory of the CTA
-//     that selects (R = 64: the leader, across the cluster) and hand the accumulator back;
+//   * the projection's epilogue warps move the logits, column by column, into the shared memory of the
+//     CTA that selects (R = 64: the leader, for the other CTA's rows across the cluster) and hand the
+//     accumulator back; the selection threads add the bias, which they staged while they waited;
 //   * 512 selection threads of that CTA pick the top k per (token, side, head), publish the block's
 //     histogram, meet the other selecting CTAs at a grid-wide barrier (a counter in global memory,
 //     bounded wait; the launch is cooperative, so all CTAs are resident) and place the block's tokens
 //     (sh_sort_block); block 0 also writes offsets and the tile table;
 //   * meanwhile producers, issuer and epilogue go on with 256 x 256 projection tiles claimed from a
-//     global counter, exactly as in sh_tc_qk_pair_kernel.
+//     global counter, as in sh_tc_qk_pair_kernel - on a ring of five stages (six measure the same; the
+//     sixth's shared memory holds the selection's scratch), and with an epilogue that stores through
+//     2 KB shared-memory tiles and TMA: row-by-row 16-byte stores kept the load / store unit busy a third
+//     of the time, and the selection warps beside them ran microseconds longer.
 //
 // Warp roles (736 threads): warp 0 lane 0 = weight producer (leader: also tile claimer), warp 6 lane 0
 // = x producer, warp 1 = TMEM allocation and (leader) UMMA issuer, warps 2..5 = epilogue, warps 7..22 =
