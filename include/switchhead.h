@@ -68,9 +68,10 @@ enum {
 };
 
 /* Create a layer description.  Host-only, no CUDA call.
- * Requires 1 <= k <= n_experts <= 32, n_heads >= 1, 1 <= d_head <= 256 (bf16 storage: <= 128; the
- * paper's 132 and 168 run in the fp32 configuration), d_model a positive multiple of 64.
- * d_head is stored padded with zero columns to 64 or 128 (bf16 storage) or to 32, 64, 128 or 256 (fp32): the padding changes no result (the scale stays 1/sqrt(d_head)),
+ * Requires 1 <= k <= n_experts <= 32, n_heads >= 1, 1 <= d_head <= 256, d_model a positive multiple of 64.
+ * (bf16 storage with d_head above 128 - the paper's 132 and 168 - runs every stage on the CUDA-core
+ * kernels: correct and slow, the plain layer only; the tensor-core kernels serve d_head <= 128.)
+ * d_head is stored padded with zero columns to 64, 128 or 256 (bf16 storage) or to 32, 64, 128 or 256 (fp32): the padding changes no result (the scale stays 1/sqrt(d_head)),
  * it costs the time of the padded size, and the Q, K, V, Ahat debug buffers have the padded
  * width.  Returns NULL on error (see sh_last_error). */
 sh_layer* sh_create(int d_model, int n_heads, int d_head, int n_experts, int k);

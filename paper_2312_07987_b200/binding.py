@@ -251,7 +251,7 @@ class Layer:
         if name in ("Q", "K", "V", "AHAT"):
             t = raw.view(torch.float32 if self.dtype == SH_F32 else torch.float16)
             # d_head is stored padded with zero columns (64 / 128 on the bf16 path, 32 / 64 / 128 on fp32)
-            Dp = (64 if D <= 64 else 128) if self.dtype != SH_F32 else (32 if D <= 32 else 64 if D <= 64 else 128 if D <= 128 else 256)
+            Dp = (64 if D <= 64 else 128 if D <= 128 else 256) if self.dtype != SH_F32 else (32 if D <= 32 else 64 if D <= 64 else 128 if D <= 128 else 256)
             t = t.view(self.batch, H, self.seq, Dp) if name != "AHAT" else t.view(self.batch * self.seq, H, Dp)
             return t[..., :D]
         return raw.view(torch.float32 if name == "GATE" else torch.int32)

@@ -156,9 +156,10 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
     sh_set_error("bf16 path needs d_model %% 128 == 0 (got d_model=%d)", d0.M);
     return SH_ERR_UNSUPPORTED;
   }
-  if (dtype == SH_BF16 && d0.Dt > 128) {
-    // (the tensor-core attention kernel keeps S and O of two query tiles in the 512 TMEM columns: d_head <= 128)
-    sh_set_error("bf16 path supports d_head up to 128 (got %d); the fp32 configuration takes up to 256", d0.Dt);
+  if (dtype == SH_BF16 && d0.Dt > 128 && (L->dense || cache_len > 0)) {
+    // (the tensor-core attention kernel keeps S and O of two query tiles in the 512 TMEM columns: d_head <= 128;
+    //  above that a bf16 layer runs on the CUDA-core kernels - see sh_tc_prepare - which this build keeps to the plain layer)
+    sh_set_error("bf16 storage with d_head above 128 (got %d): the plain layer without a cache only; the fp32 configuration takes every form", d0.Dt);
     return SH_ERR_UNSUPPORTED;
   }
   if (cache_len > 0 && L->dense) { sh_set_error("the dense comparator has no cache"); return SH_ERR_UNSUPPORTED; }
@@ -181,7 +182,7 @@ static int configure_common(sh_layer* L, int dtype, int batch, int seq, int cach
   }
   // d_head is stored padded with zero columns: to 64 or 128 on the tensor-core path, to 32, 64 or
   // 128 on the fp32 path (zero columns of W_Q, W_K, W_V and zero rows of W_O change no result)
-  L->d.D = dtype == SH_BF16 ? (d0.Dt <= 64 ? 64 : 128) : (d0.Dt <= 32 ? 32 : d0.Dt <= 64 ? 64 : d0.Dt <= 128 ? 128 : 256);
+  L->d.D = dtype == SH_BF16 ? (d0.Dt <= 64 ? 64 : d0.Dt <= 128 ? 128 : 256) : (d0.Dt <= 32 ? 32 : d0.Dt <= 64 ? 64 : d0.Dt <= 128 ? 128 : 256);
   const int T = cache_len + seq;                           // tokens of a sequence the layer sees: cache, then chunk
   const long long slots = (long long)batch * T * d0.H * d0.k;
   if (slots >= (1ll << 31) || (long long)batch * T * d0.M >= (1ll << 40)) {

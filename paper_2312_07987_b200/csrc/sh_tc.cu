@@ -243,6 +243,10 @@ int sh_tc_prepare(sh_layer* L) {
   S->attn_balanced = !getenv("SH_ATTN_ADJACENT");
   if (const char* env = getenv("SH_SIMT_STAGES")) S->simt_mask = atoi(env);   // bit mask gate=1, qk=2, v=4, attention=8, o=16
 #endif
+  // d_head above 128 (stored as 256: the paper's 132 and 168): S and O of two query tiles no longer fit the 512
+  // tensor-memory columns and the expert kernels are built for 64 / 128 columns, so every stage of such a layer
+  // runs on the CUDA-core kernels (bf16 weights and x, fp16 intermediates, fp32 sums) - correct, not fast
+  if (d.D > 128) S->simt_mask = SH_STAGE_GATE | SH_STAGE_QK | SH_STAGE_V | SH_STAGE_ATTN | SH_STAGE_O;
   // 256-column tiles (CTA pairs, or the persistent single-CTA kernel) need the projection's width to
   // be a multiple of 256; other widths take the one-CTA-per-tile kernel with 128-column tiles
   S->qk_bn = (nproj * HD) % 256 == 0 ? 256 : 128;

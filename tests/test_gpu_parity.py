@@ -259,13 +259,21 @@ def test_padded_d_head(dtype, D, T):
 
 @pytest.mark.parametrize("D,T", [(132, 70), (168, 40), (256, 33)])
 def test_d_head_above_128_in_the_fp32_configuration(D, T):
-    # the paper's 262M Wikitext-103 model (d_head 132) and its MAC-matched models (168); bf16 storage stops at 128
+    # the paper's 262M Wikitext-103 model (d_head 132) and its MAC-matched models (168)
     cfg = inputs.LayerConfig("dbig", inputs.DTYPE_F32, 2, T, 128, 2, D, 4, 2, seed=80 + D)
+    full_check(inputs.make_inputs(cfg))
+
+
+@pytest.mark.parametrize("D,T,k", [(132, 300, 2), (168, 140, 3), (256, 65, 2)])
+def test_d_head_above_128_with_bf16_storage(D, T, k):
+    # stored as 256 columns: every stage on the CUDA-core kernels (bf16 weights and x, fp16 intermediates); the
+    # plain layer only - a cache or the dense comparator is refused
+    cfg = inputs.LayerConfig("dbig_bf16", inputs.DTYPE_BF16, 2, T, 256, 2, D, 5, k, seed=90 + D)
     full_check(inputs.make_inputs(cfg))
     L = binding.Layer(256, 2, D, 4, 2)
     with pytest.raises(binding.SwitchHeadError) as e:
-        L.sh_configure(binding.SH_BF16, 1, 64)
-    assert "up to 128" in str(e.value)
+        L.sh_configure(binding.SH_BF16, 1, 128, cache_len=128)
+    assert "above 128" in str(e.value)
     L.close()
 
 
